@@ -1,0 +1,219 @@
+/*
+ * clasp.h -- C ABI of the B200 (sm_100a) layer-skip search library.
+ *
+ * The library implements the "layer optimisation" stage of CLaSp's three-stage
+ * self-speculative decoding loop (Sec. 3.1): after each verification it searches,
+ * by the approximate dynamic programme of Eq. 2 / Algorithm 1, for the set of M
+ * decoder layers whose removal keeps the last verified token's top hidden state
+ * closest (cosine) to the full model's, and it provides the full-model (verify)
+ * and layer-skipped (draft) forwards that share its kernels.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory of the current device, allocated
+ *     and owned by the caller; the library never allocates or frees device
+ *     memory.  "host" pointers are ordinary host memory.
+ *   - All work is enqueued on the stream given to clasp_create; results are
+ *     valid after the caller synchronises that stream.  No call synchronises
+ *     unless its comment says so.
+ *   - Matrices are row-major [out_features, in_features] in the model dtype
+ *     (CLASP_BF16: bfloat16, CLASP_FP32: float).  Norm weights are float.
+ *   - The KV cache of one layer is two arrays [max_ctx, n_kv_heads, head_dim] in
+ *     the model dtype; keys are stored AFTER rotary embedding.
+ *   - Hidden states / residual stream are float everywhere.
+ *   - Layers are f_0..f_{L-1};  h_0 = embedding,  h_{l+1} = f_l(h_l)  (Sec. 3.4).
+ *   - Every function returns CLASP_OK (0) or a negative CLASP_ERR_*; nothing
+ *     throws, aborts or traps on the device.  Every device-side wait is bounded;
+ *     one that runs out records a code readable by clasp_last_device_status.
+ */
+#ifndef CLASP_H_
+#define CLASP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CLASP_OK 0
+#define CLASP_ERR_INVALID_ARG (-1)  /* null pointer, negative size, M > L ...            */
+#define CLASP_ERR_SHAPE (-2)        /* a shape the kernels do not support                 */
+#define CLASP_ERR_CAPACITY (-3)     /* exceeds max_ctx / max_rows / workspace size        */
+#define CLASP_ERR_DTYPE (-4)        /* unknown dtype                                      */
+#define CLASP_ERR_CUDA (-5)         /* a CUDA runtime / driver call failed                */
+#define CLASP_ERR_TIMEOUT (-6)      /* a bounded device-side wait gave up                 */
+#define CLASP_ERR_NOT_LOADED (-7)   /* a layer or the head has not been loaded            */
+
+#define CLASP_FP32 0
+#define CLASP_BF16 1
+
+/* choice table entries (Algorithm 1: which parent g[i][j] was copied from) */
+#define CLASP_CHOICE_APPLY 0   /* g[i][j] = f_{i-1}(g[i-1][j])   */
+#define CLASP_CHOICE_SKIP 1    /* g[i][j] = g[i-1][j-1]          */
+#define CLASP_CHOICE_NONE 255  /* cell not defined (j > i) or "not forced" */
+
+typedef struct clasp_ctx clasp_ctx;
+
+typedef struct clasp_config {
+  int32_t L;            /* decoder layers                                         */
+  int32_t d_model;      /* multiple of 8                                          */
+  int32_t n_q_heads;    /* multiple of n_kv_heads                                 */
+  int32_t n_kv_heads;
+  int32_t head_dim;     /* 64 or 128                                              */
+  int32_t d_ffn;        /* multiple of 8                                          */
+  int32_t vocab;
+  int32_t dtype;        /* CLASP_FP32 | CLASP_BF16: weights, KV cache             */
+  float rms_eps;
+  float rope_theta;
+  int32_t max_ctx;      /* KV cache capacity in positions                         */
+  int32_t max_rows;     /* most rows any call pushes through a layer:
+                           clasp_verify n, clasp_dp_search M*T                    */
+  int32_t max_M;        /* most skipped layers a search is asked for              */
+  int32_t max_T;        /* most objective positions of a search                   */
+  int32_t max_head_rows;/* most rows sent through the LM head in one call         */
+  int32_t flags;        /* CLASP_FLAG_*                                           */
+} clasp_config;
+
+#define CLASP_FLAG_FORCE_SIMT 1 /* bf16 model: use the CUDA-core GEMM instead of the
+                                   tcgen05 one (diagnostics; both are device code) */
+
+/* Device pointers to the nine tensors of one decoder layer (borrowed). */
+typedef struct clasp_layer_weights {
+  const float* attn_norm; /* [d_model]                    */
+  const void* wq;         /* [n_q_heads*head_dim, d_model] */
+  const void* wk;         /* [n_kv_heads*head_dim, d_model] */
+  const void* wv;         /* [n_kv_heads*head_dim, d_model] */
+  const void* wo;         /* [d_model, n_q_heads*head_dim] */
+  const float* mlp_norm;  /* [d_model]                    */
+  const void* w_gate;     /* [d_ffn, d_model]             */
+  const void* w_up;       /* [d_ffn, d_model]             */
+  const void* w_down;     /* [d_model, d_ffn]             */
+} clasp_layer_weights;
+
+/* Device pointers to one layer's KV cache (borrowed). */
+typedef struct clasp_kv_layer {
+  void* k; /* [max_ctx, n_kv_heads, head_dim], after RoPE */
+  void* v; /* [max_ctx, n_kv_heads, head_dim]             */
+} clasp_kv_layer;
+
+/* Bytes of device workspace clasp_create needs for this configuration (0 on a
+ * bad configuration).  Host-only; launches nothing. */
+size_t clasp_workspace_bytes(const clasp_config* cfg);
+
+/* Create a context.  `workspace` is device memory of at least
+ * clasp_workspace_bytes(cfg) bytes, 256-byte aligned, owned by the caller and
+ * kept alive until clasp_destroy; the library zeroes the parts that need it
+ * (on `cuda_stream`).  `cuda_stream` is a cudaStream_t (may be NULL = default
+ * stream).  The context keeps host-side descriptors only. */
+int clasp_create(const clasp_config* cfg, void* workspace, size_t workspace_bytes,
+                 void* cuda_stream, clasp_ctx** out);
+void clasp_destroy(clasp_ctx* ctx);
+
+/* Register the weights of layers first..first+count-1 (Sec. 3.4: the decoder
+ * layers f_l the search and the forwards apply).  `w` is a HOST array of
+ * `count` structs holding DEVICE pointers; the tensors are borrowed, must stay
+ * alive and unchanged while the context uses them, and must be 16-byte aligned. */
+int clasp_load_layers(clasp_ctx* ctx, int32_t first, int32_t count, const clasp_layer_weights* w);
+
+/* Register the embedding table [vocab, d_model], the final norm weight
+ * [d_model] (float) and the LM head [vocab, d_model]; device, borrowed. */
+int clasp_load_head(clasp_ctx* ctx, const void* embed, const float* final_norm, const void* lm_head);
+
+/* Layer-skip search (Eq. 2, Algorithm 1; j-loop batched as in Sec. 3.6).
+ *
+ *   hidden_states  device, float: the full model's states x_0..x_L of the T
+ *                  objective positions; element (l, t, c) is at
+ *                  hidden_states[l*layer_stride + t*token_stride + c].
+ *   kv             HOST array of L structs of DEVICE pointers; read-only here.
+ *   ctx_len        C: cache positions [0, C) are visible to every state.
+ *   pos0           absolute position of the first objective row (normally C).
+ *   T, M           objective rows (paper: 1) and number of layers to skip.
+ *   skip_mask      device, uint8[L], out: 1 = layer skipped by the draft model.
+ *   scores         device, float[(L+1)*(M+1)], out: D(i, j) of Eq. 2, NaN where
+ *                  j > i.  For T > 1 the mean of the T per-row cosines.
+ *   margins        device or NULL, same shape: cosine(apply) - cosine(skip)
+ *                  where both candidates exist, NaN elsewhere.
+ *   g_final        device or NULL, float[T*d_model], out: g[L][M].
+ *   forced_choice  device or NULL, uint8[(L+1)*(M+1)]: where an entry is not
+ *                  CLASP_CHOICE_NONE the search takes that decision instead of
+ *                  comparing cosines (test hook: follow an oracle's path).
+ *
+ * Step i pushes the states g[i-1][1..min(i-1,M)] through layer i-1 in one batch,
+ * so each layer's weights are read from HBM once; each state attends to the
+ * cache plus its own freshly computed keys, never to another state, and the
+ * cache is not written.  M == 0 writes an all-zero mask and D(i,0) = 1 only.
+ * Errors: INVALID_ARG (null, M > L, T < 1), CAPACITY (M > max_M, T > max_T,
+ * M*T > max_rows, ctx_len + T > max_ctx), NOT_LOADED. */
+int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_stride,
+                    int64_t token_stride, const clasp_kv_layer* kv, int32_t ctx_len, int32_t pos0,
+                    int32_t T, int32_t M, uint8_t* skip_mask, float* scores, float* margins,
+                    float* g_final, const uint8_t* forced_choice);
+
+/* Full-model forward over n tokens at positions pos0..pos0+n-1 (the verify
+ * model of Sec. 3.1; also the prompt prefill and plain autoregressive steps).
+ *
+ *   tokens       device, int32[n].
+ *   kv           HOST array of L structs; K/V of the n positions are WRITTEN for
+ *                every layer, positions [0, pos0) are read.
+ *   n_head_rows  the last n_head_rows rows go through final norm + LM head.
+ *   argmax_out   device, int32[n_head_rows]: greedy token per row, lowest
+ *                index on ties.  May be NULL when n_head_rows == 0.
+ *   hidden_out   device or NULL, float[n*(L+1)*d_model]: element (t, l, c) at
+ *                hidden_out[(t*(L+1) + l)*d_model + c] = residual stream
+ *                entering layer l (l = L: after the last layer, before the
+ *                final norm) -- the objective the search needs (Sec. 3.4).
+ * Errors: CAPACITY (n > max_rows, pos0 + n > max_ctx, n_head_rows > max_head_rows). */
+int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0,
+                 const clasp_kv_layer* kv, int32_t n_head_rows, int32_t* argmax_out,
+                 float* hidden_out);
+
+/* One token through the layer-skipped draft model (Sec. 3.1, Sec. 3.3).
+ *
+ *   skip_mask_host  HOST uint8[L], 1 = skip the layer entirely (no weights read,
+ *                   no K/V written).
+ *   token_in        device, int32[1] (may be the previous call's token_out).
+ *   token_out       device, int32[1]: greedy next token.
+ *   top1_prob_out   device or NULL, float[1]: softmax probability of token_out. */
+int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int32_t* token_in,
+                        int32_t pos, const clasp_kv_layer* kv, int32_t* token_out,
+                        float* top1_prob_out);
+
+/* Greedy acceptance (Sec. 3.1, verification stage).  HOST pointers, no GPU
+ * work: draft[K] are the drafted tokens, full_argmax[K+1] the full model's
+ * greedy tokens for the rows [pending, draft_1..draft_K].  Writes the number a
+ * of leading drafts that match and the a+1 committed tokens (the accepted
+ * drafts followed by the full model's own token). */
+int clasp_accept(const int32_t* draft, const int32_t* full_argmax, int32_t K,
+                 int32_t* n_accepted, int32_t* committed /* [K+1] */);
+
+/* One decoder layer applied to S independent states of T rows each (the batch
+ * of Sec. 3.6).  x_in/x_out: device float, row (s*T+t) at x + row*stride.
+ * Row t of a state sits at position pos0+t, sees cache [0, ctx_len) and rows
+ * 0..t of its own state.  write_kv != 0 requires S == 1 and stores the rows'
+ * K/V into the cache at pos0..pos0+T-1 (they are also what the rows attend to).
+ * Exposed so that a single layer can be checked against the oracle. */
+int clasp_layer_forward(clasp_ctx* ctx, int32_t layer, const float* x_in, int64_t in_stride,
+                        int32_t S, int32_t T, int32_t ctx_len, int32_t pos0,
+                        const clasp_kv_layer* kv_layer, int32_t write_kv, float* x_out,
+                        int64_t out_stride);
+
+/* y[r, n] = sum_k x[r, k] * w[n, k]  (float out) through the same weight-
+ * streaming GEMM the layers use; x: device, model dtype, [R, K] contiguous;
+ * w: device, model dtype, [N, K]; y: device float [R, N].  Test hook. */
+int clasp_gemm_xwT(clasp_ctx* ctx, const void* x, const void* w, int32_t R, int32_t N, int32_t K,
+                   float* y);
+
+/* Synchronises the context's stream and returns the device status word:
+ * CLASP_OK, or CLASP_ERR_TIMEOUT if a bounded wait inside a kernel gave up
+ * since the last call (the word is then cleared), or CLASP_ERR_CUDA. */
+int clasp_last_device_status(clasp_ctx* ctx);
+
+/* Number of kernel launches the context has enqueued so far (host counter). */
+int64_t clasp_launch_count(const clasp_ctx* ctx);
+
+const char* clasp_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CLASP_H_ */

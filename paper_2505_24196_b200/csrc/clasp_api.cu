@@ -1,0 +1,719 @@
+// C ABI of the layer-skip search library: context, argument checks and the host-side
+// launch sequences.  Every arithmetic step runs in the kernels of kernels.cuh and
+// gemm_tc.cuh; this file only sequences launches on the caller's stream.
+#include "../../include/clasp.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <tuple>
+#include <vector>
+
+#include "gemm_tc.cuh"
+#include "kernels.cuh"
+
+namespace {
+
+using bf16 = __nv_bfloat16;
+constexpr int NSPLIT_MAX = 16;       // key splits of the attention kernel
+constexpr int MAX_COUNTERS = 4096;   // tiles of one GEMM launch that may use split-K
+constexpr size_t PARTIAL_FLOATS = (size_t)296 * 2 * 128 * 128 + (1 << 20);
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+struct LayerMaps {
+  CUtensorMap wq, wk, wv, wo, w_gate, w_up, w_down;
+};
+
+struct Workspace {
+  int* status;
+  int* counters;
+  void* xn;
+  float* qkv;
+  void* own_k;
+  void* own_v;
+  void* attn;
+  float* x1;
+  void* act;
+  float* G;
+  float* hping;
+  float* hpong;
+  float* grow[2];
+  uint8_t* choice;
+  float2* rope;
+  float* att_acc;
+  float2* att_ml;
+  float* logits;
+  float* partial;
+  size_t bytes;
+};
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+bool config_ok(const clasp_config* c) {
+  if (!c) return false;
+  if (c->L < 1 || c->d_model < 8 || c->d_model % 8 || c->d_ffn < 8 || c->d_ffn % 8) return false;
+  if (c->n_kv_heads < 1 || c->n_q_heads < c->n_kv_heads || c->n_q_heads % c->n_kv_heads) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->vocab < 1 || c->max_ctx < 1 || c->max_rows < 1 || c->max_head_rows < 1) return false;
+  if (c->max_M < 0 || c->max_M > c->L || c->max_T < 1) return false;
+  if (c->dtype != CLASP_FP32 && c->dtype != CLASP_BF16) return false;
+  return true;
+}
+
+// Lays the workspace out; with base == nullptr only the size is computed.
+Workspace carve(const clasp_config& c, uint8_t* base) {
+  Workspace w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> void* {
+    void* p = base ? base + off : nullptr;
+    off += align_up(bytes, 256);
+    return p;
+  };
+  const size_t esz = c.dtype == CLASP_BF16 ? 2 : 4;
+  const size_t R = c.max_rows, d = c.d_model;
+  const size_t qd = (size_t)c.n_q_heads * c.head_dim, kvd = (size_t)c.n_kv_heads * c.head_dim;
+  const size_t grows = (size_t)(c.max_M + 1) * c.max_T;
+  w.status = (int*)take(256);
+  w.counters = (int*)take(MAX_COUNTERS * sizeof(int));
+  w.xn = take(R * d * esz);
+  w.qkv = (float*)take(R * (qd + 2 * kvd) * 4);
+  w.own_k = take(R * kvd * esz);
+  w.own_v = take(R * kvd * esz);
+  w.attn = take(R * qd * esz);
+  w.x1 = (float*)take(R * d * 4);
+  w.act = take(R * (size_t)c.d_ffn * esz);
+  w.G = (float*)take(R * d * 4);
+  w.hping = (float*)take(R * d * 4);
+  w.hpong = (float*)take(R * d * 4);
+  w.grow[0] = (float*)take(grows * d * 4);
+  w.grow[1] = (float*)take(grows * d * 4);
+  w.choice = (uint8_t*)take((size_t)(c.L + 1) * (c.max_M + 1));
+  w.rope = (float2*)take(R * (c.head_dim / 2) * sizeof(float2));
+  w.att_acc = (float*)take(R * c.n_q_heads * NSPLIT_MAX * (size_t)c.head_dim * 4);
+  w.att_ml = (float2*)take(R * c.n_q_heads * NSPLIT_MAX * sizeof(float2));
+  w.logits = (float*)take((size_t)c.max_head_rows * c.vocab * 4);
+  w.partial = (float*)take(PARTIAL_FLOATS * 4);
+  w.bytes = off;
+  return w;
+}
+
+}  // namespace
+
+struct clasp_ctx {
+  clasp_config cfg;
+  cudaStream_t stream;
+  Workspace ws;
+  std::vector<clasp_layer_weights> layers;
+  std::vector<uint8_t> loaded;
+  std::vector<LayerMaps> maps;
+  const void* embed = nullptr;
+  const float* final_norm = nullptr;
+  const void* lm_head = nullptr;
+  CUtensorMap lm_head_map;
+  bool use_tc = false;
+  EncodeTiledFn encode = nullptr;
+  std::map<std::tuple<const void*, int, int>, CUtensorMap> xmaps;
+  int64_t launches = 0;
+  int cta_cap = 296;
+  int smem_budget = 110 * 1024;
+  int num_sms = 148;
+};
+
+namespace {
+
+#define CUDA_TRY(expr)                              \
+  do {                                              \
+    cudaError_t e__ = (expr);                       \
+    if (e__ != cudaSuccess) return CLASP_ERR_CUDA;  \
+  } while (0)
+
+int launch_check(clasp_ctx* ctx, int n = 1) {
+  ctx->launches += n;
+  return cudaGetLastError() == cudaSuccess ? CLASP_OK : CLASP_ERR_CUDA;
+}
+
+// 2-D bf16 tensor map over a row-major [rows, cols] matrix, box [box_rows x 64 cols],
+// 128-byte swizzle, zero fill outside the matrix.
+int make_map(clasp_ctx* ctx, const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)clasp::tc::BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides,
+                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? CLASP_OK : CLASP_ERR_CUDA;
+}
+
+struct GemmCall {
+  const void* x = nullptr;  // [R, K] operand dtype, contiguous
+  int R = 0, K = 0;
+  int n_mats = 1;
+  const void* w[3] = {nullptr, nullptr, nullptr};
+  const CUtensorMap* wmap[3] = {nullptr, nullptr, nullptr};
+  int N[3] = {0, 0, 0};
+  int col_off[3] = {0, 0, 0};
+  int epi = clasp::EPI_STORE;
+  const void* w2 = nullptr;  // SwiGLU: the "up" matrix
+  const CUtensorMap* w2map = nullptr;
+  float* yf = nullptr;
+  int64_t ldy = 0;
+  const float* resid = nullptr;
+  int64_t ldr = 0;
+  void* yo = nullptr;
+  int64_t ldo = 0;
+};
+
+template <typename TW, int EPI>
+int gemm_simt_one(clasp_ctx* ctx, const GemmCall& g, int m) {
+  constexpr int WARPS = 8, RB = 4;
+  const int N = g.N[m];
+  dim3 grid((N + WARPS - 1) / WARPS), block(WARPS * 32);
+  clasp::gemm_simt_kernel<TW, EPI, RB><<<grid, block, 0, ctx->stream>>>(
+      (const TW*)g.x, g.K, (const TW*)g.w[m], (const TW*)g.w2, g.R, N, g.K,
+      g.yf ? g.yf + g.col_off[m] : nullptr, g.ldy, g.resid ? g.resid + g.col_off[m] : nullptr, g.ldr,
+      g.yo ? (TW*)g.yo + g.col_off[m] : nullptr, g.ldo);
+  return launch_check(ctx);
+}
+
+template <typename TW>
+int gemm_simt(clasp_ctx* ctx, const GemmCall& g) {
+  for (int m = 0; m < g.n_mats; ++m) {
+    int rc;
+    if (g.epi == clasp::EPI_STORE) rc = gemm_simt_one<TW, clasp::EPI_STORE>(ctx, g, m);
+    else if (g.epi == clasp::EPI_RESID) rc = gemm_simt_one<TW, clasp::EPI_RESID>(ctx, g, m);
+    else rc = gemm_simt_one<TW, clasp::EPI_SWIGLU>(ctx, g, m);
+    if (rc) return rc;
+  }
+  return CLASP_OK;
+}
+
+int gemm_tc(clasp_ctx* ctx, const GemmCall& g) {
+  using namespace clasp::tc;
+  const int dual = g.epi == clasp::EPI_SWIGLU ? 1 : 0;
+  const int rb_max = dual ? 128 : 256;
+  int tiles_total = 0, n_total = 0;
+  Params p{};
+  for (int m = 0; m < 3; ++m) {
+    p.N[m] = m < g.n_mats ? g.N[m] : 0;
+    p.tiles[m] = (p.N[m] + BM - 1) / BM;
+    p.col_off[m] = m < g.n_mats ? g.col_off[m] : 0;
+    tiles_total += p.tiles[m];
+    if (m < g.n_mats && g.col_off[m] + g.N[m] > n_total) n_total = g.col_off[m] + g.N[m];
+  }
+  p.K = g.K;
+  p.k_chunks = (g.K + BK - 1) / BK;
+  // splits: a function of (N, K) only, so a row's sum never depends on the batch
+  int splits = ctx->cta_cap / tiles_total;
+  const int max_splits = p.k_chunks / 4 > 1 ? p.k_chunks / 4 : 1;
+  if (splits > max_splits) splits = max_splits;
+  if (splits < 1) splits = 1;
+  if (splits > 1 && tiles_total > MAX_COUNTERS) splits = 1;
+  p.dual = dual;
+  p.n_mats = g.n_mats;
+  p.epi = g.epi;
+  p.n_total = n_total;
+  p.ldy = g.ldy;
+  p.ldr = g.ldr;
+  p.ldo = g.ldo;
+  p.counters = ctx->ws.counters;
+  p.status = ctx->ws.status;
+  p.partial = ctx->ws.partial;
+  for (int r0 = 0; r0 < g.R; r0 += rb_max) {
+    const int Rb = g.R - r0 < rb_max ? g.R - r0 : rb_max;
+    p.R = Rb;
+    p.BN = Rb <= 16 ? 16 : (Rb + 15) / 16 * 16;
+    p.splits = splits;
+    if ((size_t)splits * (dual + 1) * Rb * n_total > PARTIAL_FLOATS) p.splits = 1;
+    const int stage_bytes = A_TILE_BYTES * (dual + 1) + p.BN * BK * 2;
+    int stages = ctx->smem_budget / stage_bytes;
+    if (stages > 8) stages = 8;
+    if (stages < 2) stages = 2;
+    const int per_cta = (p.k_chunks + p.splits - 1) / p.splits;
+    if (stages > per_cta) stages = per_cta < 1 ? 1 : per_cta;
+    p.stages = stages;
+    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    const bf16* xb = (const bf16*)g.x + (size_t)r0 * g.K;
+    auto key = std::make_tuple((const void*)xb, g.K, Rb * 1024 + p.BN);
+    auto it = ctx->xmaps.find(key);
+    if (it == ctx->xmaps.end()) {
+      CUtensorMap mp;
+      if (make_map(ctx, xb, Rb, g.K, p.BN, &mp)) return CLASP_ERR_CUDA;
+      it = ctx->xmaps.emplace(key, mp).first;
+    }
+    p.yf = g.yf ? g.yf + (size_t)r0 * g.ldy : nullptr;
+    p.resid = g.resid ? g.resid + (size_t)r0 * g.ldr : nullptr;
+    p.yo = g.yo ? (bf16*)g.yo + (size_t)r0 * g.ldo : nullptr;
+    const CUtensorMap* a0 = g.wmap[0];
+    const CUtensorMap* a1 = dual ? g.w2map : (g.n_mats > 1 ? g.wmap[1] : g.wmap[0]);
+    const CUtensorMap* a2 = g.n_mats > 2 ? g.wmap[2] : g.wmap[0];
+    dim3 grid(tiles_total, p.splits), block(THREADS);
+    gemm_tc_kernel<<<grid, block, smem, ctx->stream>>>(*a0, *a1, *a2, it->second, p);
+    int rc = launch_check(ctx);
+    if (rc) return rc;
+  }
+  return CLASP_OK;
+}
+
+int gemm(clasp_ctx* ctx, const GemmCall& g) {
+  if (g.R <= 0) return CLASP_OK;
+  if (ctx->cfg.dtype == CLASP_FP32) return gemm_simt<float>(ctx, g);
+  if (ctx->use_tc) return gemm_tc(ctx, g);
+  return gemm_simt<bf16>(ctx, g);
+}
+
+int attn_nsplit(int C) {
+  int n = (C + 255) / 256;
+  if (n < 1) n = 1;
+  if (n > NSPLIT_MAX) n = NSPLIT_MAX;
+  return n;
+}
+
+template <typename TW>
+int rmsnorm(clasp_ctx* ctx, const float* x, int64_t ldx, const float* w, int R, void* y) {
+  clasp::rmsnorm_kernel<TW><<<R, 256, 0, ctx->stream>>>(x, ldx, w, ctx->cfg.d_model, ctx->cfg.rms_eps, (TW*)y);
+  return launch_check(ctx);
+}
+
+int rope_table(clasp_ctx* ctx, int T, int pos0) {
+  const int half = ctx->cfg.head_dim / 2, n = T * half;
+  clasp::rope_table_kernel<<<(n + 255) / 256, 256, 0, ctx->stream>>>(ctx->ws.rope, T, half, pos0,
+                                                                     (double)ctx->cfg.rope_theta);
+  return launch_check(ctx);
+}
+
+// One decoder layer over S states x T rows (rope table for (T, pos0) already built).
+// own K/V of the rows go to the cache at pos0.. when write_kv, else to scratch.
+template <typename TW>
+int run_layer(clasp_ctx* ctx, int l, const float* x, int64_t ldx, int S, int T, int C, int pos0,
+              const clasp_kv_layer& kv, bool write_kv, float* out, int64_t ldo) {
+  const clasp_config& c = ctx->cfg;
+  Workspace& ws = ctx->ws;
+  const clasp_layer_weights& W = ctx->layers[l];
+  const bool tc = ctx->use_tc && c.dtype == CLASP_BF16;
+  const LayerMaps* mp = tc ? &ctx->maps[l] : nullptr;
+  const int R = S * T, d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+  const int qkvd = qd + 2 * kvd;
+  int rc;
+  if ((rc = rmsnorm<TW>(ctx, x, ldx, W.attn_norm, R, ws.xn))) return rc;
+  {
+    GemmCall g;
+    g.x = ws.xn; g.R = R; g.K = d; g.n_mats = 3;
+    g.w[0] = W.wq; g.w[1] = W.wk; g.w[2] = W.wv;
+    if (tc) { g.wmap[0] = &mp->wq; g.wmap[1] = &mp->wk; g.wmap[2] = &mp->wv; }
+    g.N[0] = qd; g.N[1] = kvd; g.N[2] = kvd;
+    g.col_off[0] = 0; g.col_off[1] = qd; g.col_off[2] = qd + kvd;
+    g.epi = clasp::EPI_STORE; g.yf = ws.qkv; g.ldy = qkvd;
+    if ((rc = gemm(ctx, g))) return rc;
+  }
+  TW* own_k = write_kv ? (TW*)kv.k : (TW*)ws.own_k;
+  TW* own_v = write_kv ? (TW*)kv.v : (TW*)ws.own_v;
+  const int64_t own_base = write_kv ? pos0 : 0;
+  clasp::rope_split_kernel<TW><<<R, 256, 0, ctx->stream>>>(ws.qkv, qkvd, ws.rope, T, c.n_q_heads, c.n_kv_heads,
+                                                           c.head_dim, own_k, own_v, own_base);
+  if ((rc = launch_check(ctx))) return rc;
+  {
+    const int nsplit = attn_nsplit(C);
+    int chunk = (C + nsplit - 1) / nsplit;
+    chunk = (chunk + 31) / 32 * 32;
+    if (chunk < 32) chunk = 32;
+    const int64_t warps = (int64_t)R * c.n_q_heads * nsplit;
+    const int wpb = 4;
+    const unsigned blocks = (unsigned)((warps + wpb - 1) / wpb);
+    const size_t smem = (size_t)wpb * c.head_dim * sizeof(float);
+    if (c.head_dim == 128) {
+      clasp::attn_partial_kernel<TW, 128><<<blocks, wpb * 32, smem, ctx->stream>>>(
+          ws.qkv, qkvd, (const TW*)kv.k, (const TW*)kv.v, C, own_k, own_v, own_base, R, T, c.n_q_heads,
+          c.n_kv_heads, nsplit, chunk, ws.att_acc, ws.att_ml);
+      if ((rc = launch_check(ctx))) return rc;
+      clasp::attn_merge_kernel<TW, 128><<<R * c.n_q_heads, 128, 0, ctx->stream>>>(
+          ws.att_acc, ws.att_ml, R, c.n_q_heads, nsplit, (TW*)ws.attn);
+    } else {
+      clasp::attn_partial_kernel<TW, 64><<<blocks, wpb * 32, smem, ctx->stream>>>(
+          ws.qkv, qkvd, (const TW*)kv.k, (const TW*)kv.v, C, own_k, own_v, own_base, R, T, c.n_q_heads,
+          c.n_kv_heads, nsplit, chunk, ws.att_acc, ws.att_ml);
+      if ((rc = launch_check(ctx))) return rc;
+      clasp::attn_merge_kernel<TW, 64><<<R * c.n_q_heads, 64, 0, ctx->stream>>>(
+          ws.att_acc, ws.att_ml, R, c.n_q_heads, nsplit, (TW*)ws.attn);
+    }
+    if ((rc = launch_check(ctx))) return rc;
+  }
+  {
+    GemmCall g;
+    g.x = ws.attn; g.R = R; g.K = qd; g.n_mats = 1; g.w[0] = W.wo;
+    if (tc) g.wmap[0] = &mp->wo;
+    g.N[0] = d; g.epi = clasp::EPI_RESID; g.yf = ws.x1; g.ldy = d; g.resid = x; g.ldr = ldx;
+    if ((rc = gemm(ctx, g))) return rc;
+  }
+  if ((rc = rmsnorm<TW>(ctx, ws.x1, d, W.mlp_norm, R, ws.xn))) return rc;
+  {
+    GemmCall g;
+    g.x = ws.xn; g.R = R; g.K = d; g.n_mats = 1; g.w[0] = W.w_gate; g.w2 = W.w_up;
+    if (tc) { g.wmap[0] = &mp->w_gate; g.w2map = &mp->w_up; }
+    g.N[0] = c.d_ffn; g.epi = clasp::EPI_SWIGLU; g.yo = ws.act; g.ldo = c.d_ffn;
+    if ((rc = gemm(ctx, g))) return rc;
+  }
+  {
+    GemmCall g;
+    g.x = ws.act; g.R = R; g.K = c.d_ffn; g.n_mats = 1; g.w[0] = W.w_down;
+    if (tc) g.wmap[0] = &mp->w_down;
+    g.N[0] = d; g.epi = clasp::EPI_RESID; g.yf = out; g.ldy = ldo; g.resid = ws.x1; g.ldr = d;
+    if ((rc = gemm(ctx, g))) return rc;
+  }
+  return CLASP_OK;
+}
+
+int run_layer_any(clasp_ctx* ctx, int l, const float* x, int64_t ldx, int S, int T, int C, int pos0,
+                  const clasp_kv_layer& kv, bool write_kv, float* out, int64_t ldo) {
+  if (ctx->cfg.dtype == CLASP_FP32)
+    return run_layer<float>(ctx, l, x, ldx, S, T, C, pos0, kv, write_kv, out, ldo);
+  return run_layer<bf16>(ctx, l, x, ldx, S, T, C, pos0, kv, write_kv, out, ldo);
+}
+
+bool layers_ready(const clasp_ctx* ctx) {
+  for (uint8_t b : ctx->loaded)
+    if (!b) return false;
+  return true;
+}
+
+// final norm + LM head + argmax over `rows` rows of x (float, stride ldx)
+int run_head(clasp_ctx* ctx, const float* x, int64_t ldx, int rows, int32_t* argmax_out, float* top1) {
+  const clasp_config& c = ctx->cfg;
+  int rc;
+  if (c.dtype == CLASP_FP32) rc = rmsnorm<float>(ctx, x, ldx, ctx->final_norm, rows, ctx->ws.xn);
+  else rc = rmsnorm<bf16>(ctx, x, ldx, ctx->final_norm, rows, ctx->ws.xn);
+  if (rc) return rc;
+  GemmCall g;
+  g.x = ctx->ws.xn; g.R = rows; g.K = c.d_model; g.n_mats = 1; g.w[0] = ctx->lm_head;
+  g.wmap[0] = &ctx->lm_head_map; g.N[0] = c.vocab; g.epi = clasp::EPI_STORE;
+  g.yf = ctx->ws.logits; g.ldy = c.vocab;
+  if ((rc = gemm(ctx, g))) return rc;
+  clasp::argmax_kernel<<<rows, 1024, 0, ctx->stream>>>(ctx->ws.logits, c.vocab, argmax_out, top1);
+  return launch_check(ctx);
+}
+
+int embed_rows(clasp_ctx* ctx, const int32_t* tokens, int n, float* out, int64_t ldo) {
+  const clasp_config& c = ctx->cfg;
+  if (c.dtype == CLASP_FP32)
+    clasp::embed_kernel<float><<<n, 256, 0, ctx->stream>>>(tokens, (const float*)ctx->embed, c.d_model, c.vocab, out, ldo);
+  else
+    clasp::embed_kernel<bf16><<<n, 256, 0, ctx->stream>>>(tokens, (const bf16*)ctx->embed, c.d_model, c.vocab, out, ldo);
+  return launch_check(ctx);
+}
+
+}  // namespace
+
+// =============================================================== C ABI
+
+extern "C" {
+
+size_t clasp_workspace_bytes(const clasp_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return carve(*cfg, nullptr).bytes;
+}
+
+int clasp_create(const clasp_config* cfg, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                 clasp_ctx** out) {
+  if (!out) return CLASP_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!cfg || !workspace) return CLASP_ERR_INVALID_ARG;
+  if (cfg->dtype != CLASP_FP32 && cfg->dtype != CLASP_BF16) return CLASP_ERR_DTYPE;
+  if (!config_ok(cfg)) return CLASP_ERR_SHAPE;
+  if (((uintptr_t)workspace & 255) != 0) return CLASP_ERR_INVALID_ARG;
+  Workspace ws = carve(*cfg, (uint8_t*)workspace);
+  if (workspace_bytes < ws.bytes) return CLASP_ERR_CAPACITY;
+  int dev = 0, n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev < 1) return CLASP_ERR_CUDA;
+  CUDA_TRY(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+  clasp_ctx* ctx = new clasp_ctx();
+  ctx->cfg = *cfg;
+  ctx->stream = (cudaStream_t)cuda_stream;
+  ctx->ws = ws;
+  ctx->layers.resize(cfg->L);
+  ctx->loaded.assign(cfg->L, 0);
+  ctx->num_sms = prop.multiProcessorCount;
+  ctx->use_tc = cfg->dtype == CLASP_BF16 && !(cfg->flags & CLASP_FLAG_FORCE_SIMT);
+  if (ctx->use_tc) {
+    if (prop.major != 10) {  // the tcgen05 kernel exists for sm_100a only
+      delete ctx;
+      return CLASP_ERR_CUDA;
+    }
+    ctx->maps.resize(cfg->L);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) {
+      delete ctx;
+      return CLASP_ERR_CUDA;
+    }
+    ctx->encode = (EncodeTiledFn)fn;
+    if (cudaFuncSetAttribute(clasp::tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             220 * 1024) != cudaSuccess) {
+      delete ctx;
+      return CLASP_ERR_CUDA;
+    }
+    ctx->cta_cap = 2 * ctx->num_sms;
+    if (const char* e = getenv("CLASP_GEMM_CTA_CAP")) ctx->cta_cap = atoi(e) > 0 ? atoi(e) : ctx->cta_cap;
+    if (const char* e = getenv("CLASP_GEMM_SMEM_KB")) {
+      const int kb = atoi(e);
+      if (kb >= 40 && kb <= 216) ctx->smem_budget = kb * 1024;
+    }
+  }
+  if (cudaMemsetAsync(ws.status, 0, 256, ctx->stream) != cudaSuccess ||
+      cudaMemsetAsync(ws.counters, 0, MAX_COUNTERS * sizeof(int), ctx->stream) != cudaSuccess) {
+    delete ctx;
+    return CLASP_ERR_CUDA;
+  }
+  *out = ctx;
+  return CLASP_OK;
+}
+
+void clasp_destroy(clasp_ctx* ctx) { delete ctx; }
+
+int clasp_load_layers(clasp_ctx* ctx, int32_t first, int32_t count, const clasp_layer_weights* w) {
+  if (!ctx || !w || first < 0 || count < 0 || first + count > ctx->cfg.L) return CLASP_ERR_INVALID_ARG;
+  const clasp_config& c = ctx->cfg;
+  const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+  for (int k = 0; k < count; ++k) {
+    const clasp_layer_weights& lw = w[k];
+    const void* ptrs[9] = {lw.attn_norm, lw.wq, lw.wk, lw.wv, lw.wo, lw.mlp_norm, lw.w_gate, lw.w_up, lw.w_down};
+    for (const void* p : ptrs)
+      if (!p || ((uintptr_t)p & 15)) return CLASP_ERR_INVALID_ARG;
+    ctx->layers[first + k] = lw;
+    if (ctx->use_tc) {
+      LayerMaps& m = ctx->maps[first + k];
+      int rc = 0;
+      rc |= make_map(ctx, lw.wq, qd, d, clasp::tc::BM, &m.wq);
+      rc |= make_map(ctx, lw.wk, kvd, d, clasp::tc::BM, &m.wk);
+      rc |= make_map(ctx, lw.wv, kvd, d, clasp::tc::BM, &m.wv);
+      rc |= make_map(ctx, lw.wo, d, qd, clasp::tc::BM, &m.wo);
+      rc |= make_map(ctx, lw.w_gate, c.d_ffn, d, clasp::tc::BM, &m.w_gate);
+      rc |= make_map(ctx, lw.w_up, c.d_ffn, d, clasp::tc::BM, &m.w_up);
+      rc |= make_map(ctx, lw.w_down, d, c.d_ffn, clasp::tc::BM, &m.w_down);
+      if (rc) return CLASP_ERR_CUDA;
+    }
+    ctx->loaded[first + k] = 1;
+  }
+  return CLASP_OK;
+}
+
+int clasp_load_head(clasp_ctx* ctx, const void* embed, const float* final_norm, const void* lm_head) {
+  if (!ctx || !embed || !final_norm || !lm_head) return CLASP_ERR_INVALID_ARG;
+  if (((uintptr_t)embed & 15) || ((uintptr_t)final_norm & 15) || ((uintptr_t)lm_head & 15))
+    return CLASP_ERR_INVALID_ARG;
+  ctx->embed = embed;
+  ctx->final_norm = final_norm;
+  ctx->lm_head = lm_head;
+  if (ctx->use_tc && make_map(ctx, lm_head, ctx->cfg.vocab, ctx->cfg.d_model, clasp::tc::BM, &ctx->lm_head_map))
+    return CLASP_ERR_CUDA;
+  return CLASP_OK;
+}
+
+int clasp_layer_forward(clasp_ctx* ctx, int32_t layer, const float* x_in, int64_t in_stride, int32_t S,
+                        int32_t T, int32_t ctx_len, int32_t pos0, const clasp_kv_layer* kv_layer,
+                        int32_t write_kv, float* x_out, int64_t out_stride) {
+  if (!ctx || !x_in || !x_out || !kv_layer || !kv_layer->k || !kv_layer->v) return CLASP_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->cfg.L || S < 1 || T < 1 || ctx_len < 0 || pos0 < 0) return CLASP_ERR_INVALID_ARG;
+  if (write_kv && S != 1) return CLASP_ERR_INVALID_ARG;
+  if (in_stride < ctx->cfg.d_model || out_stride < ctx->cfg.d_model) return CLASP_ERR_INVALID_ARG;
+  if ((int64_t)S * T > ctx->cfg.max_rows || ctx_len > ctx->cfg.max_ctx || pos0 + T > ctx->cfg.max_ctx)
+    return CLASP_ERR_CAPACITY;
+  if (!ctx->loaded[layer]) return CLASP_ERR_NOT_LOADED;
+  int rc = rope_table(ctx, T, pos0);
+  if (rc) return rc;
+  return run_layer_any(ctx, layer, x_in, in_stride, S, T, ctx_len, pos0, *kv_layer, write_kv != 0, x_out,
+                       out_stride);
+}
+
+int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_stride, int64_t token_stride,
+                    const clasp_kv_layer* kv, int32_t ctx_len, int32_t pos0, int32_t T, int32_t M,
+                    uint8_t* skip_mask, float* scores, float* margins, float* g_final,
+                    const uint8_t* forced_choice) {
+  if (!ctx || !hidden_states || !kv || !skip_mask || !scores) return CLASP_ERR_INVALID_ARG;
+  const clasp_config& c = ctx->cfg;
+  const int L = c.L, d = c.d_model;
+  if (M < 0 || M > L || T < 1 || ctx_len < 0 || pos0 < 0) return CLASP_ERR_INVALID_ARG;
+  if (M > c.max_M || T > c.max_T || (int64_t)M * T > c.max_rows || ctx_len > c.max_ctx ||
+      (int64_t)pos0 + T > c.max_ctx)
+    return CLASP_ERR_CAPACITY;
+  for (int l = 0; l < L; ++l)
+    if (!kv[l].k || !kv[l].v) return CLASP_ERR_INVALID_ARG;
+  if (M > 0 && !layers_ready(ctx)) return CLASP_ERR_NOT_LOADED;
+  Workspace& ws = ctx->ws;
+  const int ncell = (L + 1) * (M + 1);
+  clasp::fill_tables_kernel<<<(ncell + 255) / 256, 256, 0, ctx->stream>>>(scores, margins, ws.choice, ncell);
+  int rc = launch_check(ctx);
+  if (rc) return rc;
+  if ((rc = rope_table(ctx, T, pos0))) return rc;
+  const int64_t Td = (int64_t)T * d;
+  {
+    clasp::DpStepArgs a0{};  // g[0][0] = x_0, D[0][0] = 1: the b == 0 path of a step over x_0 itself
+    a0.x_i = hidden_states; a0.x_tok_stride = token_stride; a0.G = ws.G; a0.g_prev = ws.grow[0];
+    a0.g_next = ws.grow[0]; a0.D = scores; a0.margin = nullptr; a0.choice = ws.choice; a0.forced = nullptr;
+    a0.T = T; a0.d = d; a0.ell = 0; a0.i = 0; a0.M = M;
+    clasp::dp_step_kernel<<<1, 256, 0, ctx->stream>>>(a0);
+    if ((rc = launch_check(ctx))) return rc;
+  }
+  int cur = 0;
+  for (int i = 1; i <= L; ++i) {
+    const int ell = (i - 1 < M) ? i - 1 : M;
+    float* g_prev = ws.grow[cur];
+    float* g_next = ws.grow[cur ^ 1];
+    if (ell > 0) {
+      // all candidate states j = 1..ell through layer i-1 in one batch (Sec. 3.6)
+      rc = run_layer_any(ctx, i - 1, g_prev + Td, d, ell, T, ctx_len, pos0, kv[i - 1], false, ws.G, d);
+      if (rc) return rc;
+    }
+    clasp::DpStepArgs a{};
+    a.x_i = hidden_states + (int64_t)i * layer_stride;
+    a.x_tok_stride = token_stride;
+    a.G = ws.G;
+    a.g_prev = g_prev;
+    a.g_next = g_next;
+    a.D = scores + (int64_t)i * (M + 1);
+    a.margin = margins ? margins + (int64_t)i * (M + 1) : nullptr;
+    a.choice = ws.choice + (int64_t)i * (M + 1);
+    a.forced = forced_choice ? forced_choice + (int64_t)i * (M + 1) : nullptr;
+    a.T = T; a.d = d; a.ell = ell; a.i = i; a.M = M;
+    const int blocks = 1 + ell + (i <= M ? 1 : 0);
+    clasp::dp_step_kernel<<<blocks, 256, 0, ctx->stream>>>(a);
+    if ((rc = launch_check(ctx))) return rc;
+    cur ^= 1;
+  }
+  clasp::backtrack_kernel<<<1, 32, 0, ctx->stream>>>(ws.choice, L, M, skip_mask);
+  if ((rc = launch_check(ctx))) return rc;
+  if (g_final) {
+    clasp::copy_rows_kernel<<<T, 256, 0, ctx->stream>>>(ws.grow[cur] + (int64_t)M * Td, d, g_final, d, d);
+    if ((rc = launch_check(ctx))) return rc;
+  }
+  return CLASP_OK;
+}
+
+int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0, const clasp_kv_layer* kv,
+                 int32_t n_head_rows, int32_t* argmax_out, float* hidden_out) {
+  if (!ctx || !tokens || !kv || n < 1 || pos0 < 0 || n_head_rows < 0 || n_head_rows > n)
+    return CLASP_ERR_INVALID_ARG;
+  if (n_head_rows > 0 && !argmax_out) return CLASP_ERR_INVALID_ARG;
+  const clasp_config& c = ctx->cfg;
+  if (n > c.max_rows || (int64_t)pos0 + n > c.max_ctx || n_head_rows > c.max_head_rows) return CLASP_ERR_CAPACITY;
+  for (int l = 0; l < c.L; ++l)
+    if (!kv[l].k || !kv[l].v) return CLASP_ERR_INVALID_ARG;
+  if (!layers_ready(ctx) || !ctx->embed) return CLASP_ERR_NOT_LOADED;
+  const int d = c.d_model, L = c.L;
+  int rc;
+  if ((rc = rope_table(ctx, n, pos0))) return rc;
+  const float* x;
+  int64_t ldx;
+  if (hidden_out) {
+    const int64_t ld = (int64_t)(L + 1) * d;
+    if ((rc = embed_rows(ctx, tokens, n, hidden_out, ld))) return rc;
+    for (int l = 0; l < L; ++l) {
+      rc = run_layer_any(ctx, l, hidden_out + (int64_t)l * d, ld, 1, n, pos0, pos0, kv[l], true,
+                         hidden_out + (int64_t)(l + 1) * d, ld);
+      if (rc) return rc;
+    }
+    x = hidden_out + (int64_t)L * d;
+    ldx = ld;
+  } else {
+    float* a = ctx->ws.hping;
+    float* b = ctx->ws.hpong;
+    if ((rc = embed_rows(ctx, tokens, n, a, d))) return rc;
+    for (int l = 0; l < L; ++l) {
+      if ((rc = run_layer_any(ctx, l, a, d, 1, n, pos0, pos0, kv[l], true, b, d))) return rc;
+      float* t = a; a = b; b = t;
+    }
+    x = a;
+    ldx = d;
+  }
+  if (n_head_rows > 0)
+    return run_head(ctx, x + (int64_t)(n - n_head_rows) * ldx, ldx, n_head_rows, argmax_out, nullptr);
+  return CLASP_OK;
+}
+
+int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int32_t* token_in, int32_t pos,
+                        const clasp_kv_layer* kv, int32_t* token_out, float* top1_prob_out) {
+  if (!ctx || !skip_mask_host || !token_in || !kv || !token_out || pos < 0) return CLASP_ERR_INVALID_ARG;
+  const clasp_config& c = ctx->cfg;
+  if ((int64_t)pos + 1 > c.max_ctx) return CLASP_ERR_CAPACITY;
+  if (!layers_ready(ctx) || !ctx->embed) return CLASP_ERR_NOT_LOADED;
+  const int d = c.d_model;
+  int rc;
+  if ((rc = rope_table(ctx, 1, pos))) return rc;
+  float* a = ctx->ws.hping;
+  float* b = ctx->ws.hpong;
+  if ((rc = embed_rows(ctx, token_in, 1, a, d))) return rc;
+  for (int l = 0; l < c.L; ++l) {
+    if (skip_mask_host[l]) continue;  // skipped layer: state passes through, nothing read or written
+    if (!kv[l].k || !kv[l].v) return CLASP_ERR_INVALID_ARG;
+    if ((rc = run_layer_any(ctx, l, a, d, 1, 1, pos, pos, kv[l], true, b, d))) return rc;
+    float* t = a; a = b; b = t;
+  }
+  return run_head(ctx, a, d, 1, token_out, top1_prob_out);
+}
+
+int clasp_accept(const int32_t* draft, const int32_t* full_argmax, int32_t K, int32_t* n_accepted,
+                 int32_t* committed) {
+  if (K < 0 || !full_argmax || !n_accepted || !committed || (K > 0 && !draft)) return CLASP_ERR_INVALID_ARG;
+  int a = 0;
+  while (a < K && draft[a] == full_argmax[a]) ++a;
+  for (int k = 0; k < a; ++k) committed[k] = draft[k];
+  committed[a] = full_argmax[a];
+  *n_accepted = a;
+  return CLASP_OK;
+}
+
+int clasp_gemm_xwT(clasp_ctx* ctx, const void* x, const void* w, int32_t R, int32_t N, int32_t K, float* y) {
+  if (!ctx || !x || !w || !y || R < 1 || N < 1 || K < 8 || K % 8) return CLASP_ERR_INVALID_ARG;
+  if (((uintptr_t)x & 15) || ((uintptr_t)w & 15)) return CLASP_ERR_INVALID_ARG;
+  GemmCall g;
+  g.x = x; g.R = R; g.K = K; g.n_mats = 1; g.w[0] = w; g.N[0] = N; g.epi = clasp::EPI_STORE;
+  g.yf = y; g.ldy = N;
+  CUtensorMap mp;
+  if (ctx->use_tc) {
+    if (make_map(ctx, w, N, K, clasp::tc::BM, &mp)) return CLASP_ERR_CUDA;
+    g.wmap[0] = &mp;
+    ctx->xmaps.clear();  // caller-owned operand buffers come and go: do not keep stale maps
+  }
+  return gemm(ctx, g);
+}
+
+int clasp_last_device_status(clasp_ctx* ctx) {
+  if (!ctx) return CLASP_ERR_INVALID_ARG;
+  int st = 0;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return CLASP_ERR_CUDA;
+  if (cudaMemcpy(&st, ctx->ws.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return CLASP_ERR_CUDA;
+  if (st != 0) {
+    cudaMemset(ctx->ws.status, 0, sizeof(int));
+    cudaMemset(ctx->ws.counters, 0, MAX_COUNTERS * sizeof(int));
+    return CLASP_ERR_TIMEOUT;
+  }
+  return CLASP_OK;
+}
+
+int64_t clasp_launch_count(const clasp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* clasp_strerror(int code) {
+  switch (code) {
+    case CLASP_OK: return "ok";
+    case CLASP_ERR_INVALID_ARG: return "invalid argument";
+    case CLASP_ERR_SHAPE: return "unsupported shape";
+    case CLASP_ERR_CAPACITY: return "capacity exceeded";
+    case CLASP_ERR_DTYPE: return "unsupported dtype";
+    case CLASP_ERR_CUDA: return "CUDA error";
+    case CLASP_ERR_TIMEOUT: return "device-side wait timed out";
+    case CLASP_ERR_NOT_LOADED: return "weights not loaded";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

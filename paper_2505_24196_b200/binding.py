@@ -21,7 +21,7 @@ FLAG_FORCE_SIMT = 1
 
 SYMBOLS = ["clasp_workspace_bytes", "clasp_create", "clasp_destroy", "clasp_load_layers", "clasp_load_head",
            "clasp_dp_search", "clasp_verify", "clasp_draft_forward", "clasp_accept", "clasp_layer_forward",
-           "clasp_gemm_xwT", "clasp_last_device_status", "clasp_launch_count", "clasp_strerror"]
+           "clasp_gemm_xwT", "clasp_profile_gemm", "clasp_last_device_status", "clasp_launch_count", "clasp_strerror"]
 
 
 class ClaspConfig(C.Structure):
@@ -83,6 +83,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.clasp_layer_forward.argtypes = [vp, i32, vp, i64, i32, i32, i32, i32, C.POINTER(ClaspKvLayer), i32, vp, i64]
     lib.clasp_gemm_xwT.restype = C.c_int
     lib.clasp_gemm_xwT.argtypes = [vp, vp, vp, i32, i32, i32, vp]
+    lib.clasp_profile_gemm.restype = C.c_int
+    lib.clasp_profile_gemm.argtypes = [vp, i32, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     lib.clasp_last_device_status.restype = C.c_int
     lib.clasp_last_device_status.argtypes = [vp]
     lib.clasp_launch_count.restype = C.c_int64

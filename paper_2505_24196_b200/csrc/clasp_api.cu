@@ -123,6 +123,9 @@ struct clasp_ctx {
   EncodeTiledFn encode = nullptr;
   std::map<std::tuple<const void*, int, int>, CUtensorMap> xmaps;
   int64_t launches = 0;
+  bool profiling = false;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_events;
+  double prof_bytes = 0.0;
   int cta_cap = 296;
   int smem_budget = 110 * 1024;
   int num_sms = 148;
@@ -257,7 +260,19 @@ int gemm_tc(clasp_ctx* ctx, const GemmCall& g) {
     const CUtensorMap* a1 = dual ? g.w2map : (g.n_mats > 1 ? g.wmap[1] : g.wmap[0]);
     const CUtensorMap* a2 = g.n_mats > 2 ? g.wmap[2] : g.wmap[0];
     dim3 grid(tiles_total, p.splits), block(THREADS);
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (ctx->profiling) {
+      if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return CLASP_ERR_CUDA;
+      cudaEventRecord(e0, ctx->stream);
+    }
     gemm_tc_kernel<<<grid, block, smem, ctx->stream>>>(*a0, *a1, *a2, it->second, p);
+    if (ctx->profiling) {
+      cudaEventRecord(e1, ctx->stream);
+      ctx->prof_events.emplace_back(e0, e1);
+      double nk = 0.0;
+      for (int m = 0; m < g.n_mats; ++m) nk += (double)g.N[m] * g.K;
+      ctx->prof_bytes += nk * 2.0 * (dual + 1);
+    }
     int rc = launch_check(ctx);
     if (rc) return rc;
   }
@@ -698,6 +713,32 @@ int clasp_last_device_status(clasp_ctx* ctx) {
     return CLASP_ERR_TIMEOUT;
   }
   return CLASP_OK;
+}
+
+int clasp_profile_gemm(clasp_ctx* ctx, int32_t enable, int64_t* n_launches, double* total_ms,
+                       double* weight_bytes) {
+  if (!ctx) return CLASP_ERR_INVALID_ARG;
+  if (enable) {
+    ctx->profiling = true;
+    return CLASP_OK;
+  }
+  ctx->profiling = false;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return CLASP_ERR_CUDA;
+  double ms = 0.0;
+  int rc = CLASP_OK;
+  for (auto& pr : ctx->prof_events) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, pr.first, pr.second) != cudaSuccess) rc = CLASP_ERR_CUDA;
+    ms += t;
+    cudaEventDestroy(pr.first);
+    cudaEventDestroy(pr.second);
+  }
+  if (n_launches) *n_launches = (int64_t)ctx->prof_events.size();
+  if (total_ms) *total_ms = ms;
+  if (weight_bytes) *weight_bytes = ctx->prof_bytes;
+  ctx->prof_events.clear();
+  ctx->prof_bytes = 0.0;
+  return rc;
 }
 
 int64_t clasp_launch_count(const clasp_ctx* ctx) { return ctx ? ctx->launches : 0; }

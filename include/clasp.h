@@ -203,6 +203,44 @@ int clasp_layer_forward(clasp_ctx* ctx, int32_t layer, const float* x_in, int64_
 int clasp_gemm_xwT(clasp_ctx* ctx, const void* x, const void* w, int32_t R, int32_t N, int32_t K,
                    float* y);
 
+/* Allocation-free variant of clasp_gemm_xwT for bf16 operands (the paper has no
+ * counterpart; it exists for callers that must not allocate).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- an inference
+ * plug-in's enqueue hook, or a serving loop that handed the whole device to a memory
+ * pool at start-up, so that a fresh allocation would fail or force a device-wide
+ * synchronisation in the middle of decoding.  Such a caller cannot create a clasp_ctx
+ * (whose workspace somebody has to allocate) just to run one product.
+ *
+ * What it does: y[r, n] = sum_k x[r, k] * w[n, k] with the same tensor-core kernel and
+ * the same split-K schedule as clasp_gemm_xwT, so the two agree bit for bit.  The
+ * split-K partial sums, the per-tile arrival counters and a status word live in a
+ * fixed array of CLASP_NOALLOC_SCRATCH_BYTES that is part of the library image: every
+ * GPU that loads the library carries it until the process exits.  The call makes no
+ * cudaMalloc, cudaFree or other allocating call; the caller passes inputs and outputs.
+ *
+ *   x  device, bf16 [R, K] contiguous, 16-byte aligned;  1 <= R <= CLASP_NOALLOC_MAX_ROWS
+ *   w  device, bf16 [N, K] contiguous, 16-byte aligned;  K a multiple of 8
+ *   y  device, float [R, N]
+ *   cuda_stream  the cudaStream_t to launch on (NULL = default stream)
+ *   status_out   device int32 or NULL: set to 1 by the kernel if one of its bounded
+ *                waits gave up (y is then unspecified); the caller zeroes it beforehand.
+ *
+ * Limits: shapes whose partial sums (splits * R * N floats) exceed the array, or with
+ * more than 4096 output tiles under split-K, are refused with CLASP_ERR_CAPACITY;
+ * R > CLASP_NOALLOC_MAX_ROWS likewise.  Devices other than sm_100 give CLASP_ERR_CUDA.
+ * First use on each device: the first call made with that device current looks up the
+ * array's device address and the driver's tensor-map encoder and raises the kernel's
+ * shared-memory limit.  Make that first call before any stream capture begins.
+ * Sharing: all calls on a device use the one array and it keeps the previous call's
+ * contents; each call re-zeroes the counters on its stream before launching.  Two
+ * calls that overlap on the GPU (different streams, or different host threads without
+ * ordering) race on it: serialise them. */
+#define CLASP_NOALLOC_SCRATCH_BYTES (4u * 1024u * 1024u + 16u * 1024u + 256u)
+#define CLASP_NOALLOC_MAX_ROWS 256
+int clasp_gemm_xwT_noalloc(const void* x, const void* w, int32_t R, int32_t N, int32_t K, float* y,
+                           void* cuda_stream, int32_t* status_out);
+
 /* Synchronises the context's stream and returns the device status word:
  * CLASP_OK, or CLASP_ERR_TIMEOUT if a bounded wait inside a kernel gave up
  * since the last call (the word is then cleared), or CLASP_ERR_CUDA. */

@@ -21,7 +21,7 @@ FLAG_FORCE_SIMT = 1
 
 SYMBOLS = ["clasp_workspace_bytes", "clasp_create", "clasp_destroy", "clasp_load_layers", "clasp_load_head",
            "clasp_dp_search", "clasp_verify", "clasp_draft_forward", "clasp_accept", "clasp_layer_forward",
-           "clasp_gemm_xwT", "clasp_profile_gemm", "clasp_last_device_status", "clasp_launch_count", "clasp_strerror"]
+           "clasp_gemm_xwT", "clasp_gemm_xwT_noalloc", "clasp_profile_gemm", "clasp_last_device_status", "clasp_launch_count", "clasp_strerror"]
 
 
 class ClaspConfig(C.Structure):
@@ -83,6 +83,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.clasp_layer_forward.argtypes = [vp, i32, vp, i64, i32, i32, i32, i32, C.POINTER(ClaspKvLayer), i32, vp, i64]
     lib.clasp_gemm_xwT.restype = C.c_int
     lib.clasp_gemm_xwT.argtypes = [vp, vp, vp, i32, i32, i32, vp]
+    lib.clasp_gemm_xwT_noalloc.restype = C.c_int
+    lib.clasp_gemm_xwT_noalloc.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     lib.clasp_profile_gemm.restype = C.c_int
     lib.clasp_profile_gemm.argtypes = [vp, i32, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     lib.clasp_last_device_status.restype = C.c_int
@@ -106,6 +108,20 @@ def _check(code: int, what: str):
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
     return None if t is None else t.data_ptr()
+
+
+def gemm_xwT_noalloc(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor,
+                     status_out: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """y = x w^T (bf16 in, float out) through the allocation-free entry point: no context,
+    no workspace; the library's built-in scratch array is used.  The caller owns x, w, y."""
+    R, K = x.shape
+    N = w.shape[0]
+    assert x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16 and y.dtype == torch.float32
+    assert x.is_contiguous() and w.is_contiguous() and y.is_contiguous() and y.shape == (R, N)
+    st = stream if stream is not None else torch.cuda.current_stream(x.device)
+    with torch.cuda.device(x.device):
+        _check(load_library().clasp_gemm_xwT_noalloc(x.data_ptr(), w.data_ptr(), R, N, K, y.data_ptr(),
+                                                     st.cuda_stream, _ptr(status_out)), "clasp_gemm_xwT_noalloc")
 
 
 def make_config(model_cfg, max_ctx: int, max_rows: int, max_M: int, max_T: int = 1,

@@ -11,6 +11,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <tuple>
 #include <vector>
 
@@ -700,6 +701,121 @@ int clasp_gemm_xwT(clasp_ctx* ctx, const void* x, const void* w, int32_t R, int3
     ctx->xmaps.clear();  // caller-owned operand buffers come and go: do not keep stale maps
   }
   return gemm(ctx, g);
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------- allocation-free GEMM
+// Scratch of clasp_gemm_xwT_noalloc: [4 MiB split-K partial sums][4096 tile counters]
+// [status word].  In host code the symbol below is only a stand-in: the device address
+// comes from cudaGetSymbolAddress, once per device, with that device current.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[CLASP_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr size_t NOALLOC_PARTIAL_BYTES = 4u * 1024u * 1024u;
+constexpr int NOALLOC_COUNTERS = 4096;
+constexpr int NOALLOC_MAX_DEVICES = 64;
+struct NoAllocDevice {
+  bool ready = false;
+  unsigned char* scratch = nullptr;
+  EncodeTiledFn encode = nullptr;
+  int cta_cap = 296;
+};
+NoAllocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
+std::mutex g_noalloc_mutex;  // guards the one-time set-up only
+
+int noalloc_setup(int dev, NoAllocDevice** out) {
+  if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return CLASP_ERR_CAPACITY;
+  NoAllocDevice& nd = g_noalloc_dev[dev];
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!nd.ready) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return CLASP_ERR_CUDA;
+    if (prop.major != 10) return CLASP_ERR_CUDA;
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return CLASP_ERR_CUDA;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
+      return CLASP_ERR_CUDA;
+    if (cudaFuncSetAttribute(clasp::tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             220 * 1024) != cudaSuccess)
+      return CLASP_ERR_CUDA;
+    nd.scratch = (unsigned char*)ptr;
+    nd.encode = (EncodeTiledFn)fn;
+    nd.cta_cap = 2 * prop.multiProcessorCount;
+    nd.ready = true;
+  }
+  *out = &nd;
+  return CLASP_OK;
+}
+
+int noalloc_map(EncodeTiledFn encode, const void* ptr, int rows, int cols, int box_rows, CUtensorMap* out) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)clasp::tc::BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? CLASP_OK : CLASP_ERR_CUDA;
+}
+}  // namespace
+
+extern "C" {
+
+int clasp_gemm_xwT_noalloc(const void* x, const void* w, int32_t R, int32_t N, int32_t K, float* y,
+                           void* cuda_stream, int32_t* status_out) {
+  using namespace clasp::tc;
+  if (!x || !w || !y || R < 1 || N < 1 || K < 8 || K % 8) return CLASP_ERR_INVALID_ARG;
+  if (((uintptr_t)x & 15) || ((uintptr_t)w & 15)) return CLASP_ERR_INVALID_ARG;
+  if (R > CLASP_NOALLOC_MAX_ROWS) return CLASP_ERR_CAPACITY;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return CLASP_ERR_CUDA;
+  NoAllocDevice* nd = nullptr;
+  int rc = noalloc_setup(dev, &nd);
+  if (rc) return rc;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  Params p{};
+  const int tiles = (N + BM - 1) / BM;
+  p.N[0] = N; p.tiles[0] = tiles; p.col_off[0] = 0;
+  p.K = K;
+  p.k_chunks = (K + BK - 1) / BK;
+  int splits = nd->cta_cap / tiles;  // the schedule of clasp_gemm_xwT: a function of (N, K) only
+  const int max_splits = p.k_chunks / 4 > 1 ? p.k_chunks / 4 : 1;
+  if (splits > max_splits) splits = max_splits;
+  if (splits < 1) splits = 1;
+  if (splits > 1 && tiles > MAX_COUNTERS) splits = 1;
+  if (splits > 1) {
+    if ((size_t)splits * R * N * sizeof(float) > NOALLOC_PARTIAL_BYTES || tiles > NOALLOC_COUNTERS)
+      return CLASP_ERR_CAPACITY;
+  }
+  p.R = R;
+  p.BN = R <= 16 ? 16 : (R + 15) / 16 * 16;
+  p.splits = splits;
+  p.dual = 0; p.n_mats = 1; p.epi = clasp::EPI_STORE; p.n_total = N;
+  p.yf = y; p.ldy = N;
+  p.partial = (float*)nd->scratch;
+  p.counters = (int*)(nd->scratch + NOALLOC_PARTIAL_BYTES);
+  int* scratch_status = (int*)(nd->scratch + NOALLOC_PARTIAL_BYTES + NOALLOC_COUNTERS * sizeof(int));
+  p.status = status_out ? status_out : scratch_status;
+  const int stage_bytes = A_TILE_BYTES + p.BN * BK * 2;
+  int stages = 110 * 1024 / stage_bytes;
+  if (stages > 8) stages = 8;
+  if (stages < 2) stages = 2;
+  const int per_cta = (p.k_chunks + splits - 1) / splits;
+  if (stages > per_cta) stages = per_cta < 1 ? 1 : per_cta;
+  p.stages = stages;
+  const size_t smem = (size_t)stages * stage_bytes + 1024;
+  CUtensorMap map_w, map_x;
+  if (noalloc_map(nd->encode, w, N, K, BM, &map_w) || noalloc_map(nd->encode, x, R, K, p.BN, &map_x))
+    return CLASP_ERR_CUDA;
+  // the array keeps whatever the previous call left: the counters must start at zero
+  if (cudaMemsetAsync(p.counters, 0, (NOALLOC_COUNTERS + 64) * sizeof(int), stream) != cudaSuccess)
+    return CLASP_ERR_CUDA;
+  dim3 grid(tiles, splits), block(THREADS);
+  gemm_tc_kernel<<<grid, block, smem, stream>>>(map_w, map_w, map_w, map_x, p);
+  return cudaGetLastError() == cudaSuccess ? CLASP_OK : CLASP_ERR_CUDA;
 }
 
 int clasp_last_device_status(clasp_ctx* ctx) {

@@ -21,7 +21,6 @@
 namespace {
 
 using bf16 = __nv_bfloat16;
-constexpr int NSPLIT_MAX = 16;       // key splits of the attention kernel
 constexpr int MAX_COUNTERS = 4096;   // tiles of one GEMM launch that may use split-K
 constexpr size_t PARTIAL_FLOATS = (size_t)296 * 2 * 128 * 128 + (1 << 20);
 
@@ -99,8 +98,9 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
   w.grow[1] = (float*)take(grows * d * 4);
   w.choice = (uint8_t*)take((size_t)(c.L + 1) * (c.max_M + 1));
   w.rope = (float2*)take(R * (c.head_dim / 2) * sizeof(float2));
-  w.att_acc = (float*)take(R * c.n_q_heads * NSPLIT_MAX * (size_t)c.head_dim * 4);
-  w.att_ml = (float2*)take(R * c.n_q_heads * NSPLIT_MAX * sizeof(float2));
+  const size_t att_chunks = clasp::ATT_MAX_CACHE_CHUNKS + (R + clasp::ATT_KEYS - 1) / clasp::ATT_KEYS;
+  w.att_acc = (float*)take(R * c.n_q_heads * att_chunks * (size_t)c.head_dim * 4);
+  w.att_ml = (float2*)take(R * c.n_q_heads * att_chunks * sizeof(float2));
   w.logits = (float*)take((size_t)c.max_head_rows * c.vocab * 4);
   w.partial = (float*)take(PARTIAL_FLOATS * 4);
   w.bytes = off;
@@ -287,11 +287,36 @@ int gemm(clasp_ctx* ctx, const GemmCall& g) {
   return gemm_simt<bf16>(ctx, g);
 }
 
-int attn_nsplit(int C) {
-  int n = (C + 255) / 256;
-  if (n < 1) n = 1;
-  if (n > NSPLIT_MAX) n = NSPLIT_MAX;
-  return n;
+template <typename TW, int HD>
+int attention(clasp_ctx* ctx, int R, int T, int C, const clasp_kv_layer& kv, const TW* own_k, const TW* own_v,
+              int64_t own_base) {
+  const clasp_config& c = ctx->cfg;
+  Workspace& ws = ctx->ws;
+  const int qkvd = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  // chunking is a function of C (cache) and R (own rows) only
+  const int n_sub = (C + clasp::ATT_KEYS - 1) / clasp::ATT_KEYS;
+  const int nsub = n_sub > 0 ? (n_sub + clasp::ATT_MAX_CACHE_CHUNKS - 1) / clasp::ATT_MAX_CACHE_CHUNKS : 1;
+  const int n_cache_chunks = (n_sub + nsub - 1) / nsub;
+  const int n_chunks = n_cache_chunks + (R + clasp::ATT_KEYS - 1) / clasp::ATT_KEYS;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const int pair_blocks = (R * G + clasp::ATT_PAIRS - 1) / clasp::ATT_PAIRS;
+  constexpr int smem = clasp::att_smem_bytes<TW, HD>();
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(clasp::attn_tile_kernel<TW, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+        cudaSuccess)
+      return CLASP_ERR_CUDA;
+    attr_set = true;
+  }
+  dim3 grid(n_chunks, c.n_kv_heads, pair_blocks);
+  clasp::attn_tile_kernel<TW, HD><<<grid, clasp::ATT_WARPS * 32, smem, ctx->stream>>>(
+      ws.qkv, qkvd, ws.rope, (const TW*)kv.k, (const TW*)kv.v, C, own_k, own_v, own_base, R, T, c.n_q_heads,
+      c.n_kv_heads, n_cache_chunks, nsub, n_chunks, ws.att_acc, ws.att_ml);
+  int rc = launch_check(ctx);
+  if (rc) return rc;
+  clasp::attn_merge_kernel<TW, HD><<<R * c.n_q_heads, HD, 0, ctx->stream>>>(ws.att_acc, ws.att_ml, R, c.n_q_heads,
+                                                                          n_chunks, (TW*)ws.attn);
+  return launch_check(ctx);
 }
 
 template <typename TW>
@@ -334,35 +359,12 @@ int run_layer(clasp_ctx* ctx, int l, const float* x, int64_t ldx, int S, int T, 
   TW* own_k = write_kv ? (TW*)kv.k : (TW*)ws.own_k;
   TW* own_v = write_kv ? (TW*)kv.v : (TW*)ws.own_v;
   const int64_t own_base = write_kv ? pos0 : 0;
-  clasp::rope_split_kernel<TW><<<R, 256, 0, ctx->stream>>>(ws.qkv, qkvd, ws.rope, T, c.n_q_heads, c.n_kv_heads,
-                                                           c.head_dim, own_k, own_v, own_base);
+  clasp::kv_store_kernel<TW><<<R, 256, 0, ctx->stream>>>(ws.qkv, qkvd, ws.rope, T, c.n_q_heads, c.n_kv_heads,
+                                                         c.head_dim, own_k, own_v, own_base);
   if ((rc = launch_check(ctx))) return rc;
-  {
-    const int nsplit = attn_nsplit(C);
-    int chunk = (C + nsplit - 1) / nsplit;
-    chunk = (chunk + 31) / 32 * 32;
-    if (chunk < 32) chunk = 32;
-    const int64_t warps = (int64_t)R * c.n_q_heads * nsplit;
-    const int wpb = 4;
-    const unsigned blocks = (unsigned)((warps + wpb - 1) / wpb);
-    const size_t smem = (size_t)wpb * c.head_dim * sizeof(float);
-    if (c.head_dim == 128) {
-      clasp::attn_partial_kernel<TW, 128><<<blocks, wpb * 32, smem, ctx->stream>>>(
-          ws.qkv, qkvd, (const TW*)kv.k, (const TW*)kv.v, C, own_k, own_v, own_base, R, T, c.n_q_heads,
-          c.n_kv_heads, nsplit, chunk, ws.att_acc, ws.att_ml);
-      if ((rc = launch_check(ctx))) return rc;
-      clasp::attn_merge_kernel<TW, 128><<<R * c.n_q_heads, 128, 0, ctx->stream>>>(
-          ws.att_acc, ws.att_ml, R, c.n_q_heads, nsplit, (TW*)ws.attn);
-    } else {
-      clasp::attn_partial_kernel<TW, 64><<<blocks, wpb * 32, smem, ctx->stream>>>(
-          ws.qkv, qkvd, (const TW*)kv.k, (const TW*)kv.v, C, own_k, own_v, own_base, R, T, c.n_q_heads,
-          c.n_kv_heads, nsplit, chunk, ws.att_acc, ws.att_ml);
-      if ((rc = launch_check(ctx))) return rc;
-      clasp::attn_merge_kernel<TW, 64><<<R * c.n_q_heads, 64, 0, ctx->stream>>>(
-          ws.att_acc, ws.att_ml, R, c.n_q_heads, nsplit, (TW*)ws.attn);
-    }
-    if ((rc = launch_check(ctx))) return rc;
-  }
+  if (c.head_dim == 128) rc = attention<TW, 128>(ctx, R, T, C, kv, own_k, own_v, own_base);
+  else rc = attention<TW, 64>(ctx, R, T, C, kv, own_k, own_v, own_base);
+  if (rc) return rc;
   {
     GemmCall g;
     g.x = ws.attn; g.R = R; g.K = qd; g.n_mats = 1; g.w[0] = W.wo;

@@ -156,22 +156,16 @@ __global__ void rope_table_kernel(float2* __restrict__ cs, int T, int half, int 
   cs[idx] = make_float2((float)c, (float)s);
 }
 
-// Rotate q in place (float), rotate k and store k, v in the cache dtype at row
-// (own_base + r) of own_k / own_v ([rows, n_kv, hd]).  One block per row.
+// K/V of the rows: rotate k, round k and v to the cache dtype and store them at row
+// (own_base + r) of own_k / own_v ([rows, n_kv, hd]).  q stays un-rotated in qkv; the
+// attention kernel rotates it while loading.  One block per row.
 template <typename TW>
-__global__ void rope_split_kernel(float* __restrict__ qkv, int64_t ld, const float2* __restrict__ cs,
-                                  int T, int nq, int nkv, int hd, TW* __restrict__ own_k,
-                                  TW* __restrict__ own_v, int64_t own_base) {
+__global__ void kv_store_kernel(const float* __restrict__ qkv, int64_t ld, const float2* __restrict__ cs,
+                                int T, int nq, int nkv, int hd, TW* __restrict__ own_k,
+                                TW* __restrict__ own_v, int64_t own_base) {
   const int r = blockIdx.x, t = r % T, half = hd >> 1;
-  float* row = qkv + (int64_t)r * ld;
+  const float* row = qkv + (int64_t)r * ld;
   const float2* c = cs + (int64_t)t * half;
-  for (int idx = threadIdx.x; idx < nq * half; idx += blockDim.x) {
-    const int h = idx / half, i = idx % half;
-    float* p = row + h * hd;
-    const float a = p[i], b = p[i + half];
-    p[i] = a * c[i].x - b * c[i].y;
-    p[i + half] = b * c[i].x + a * c[i].y;
-  }
   const float* kr = row + nq * hd;
   const float* vr = kr + nkv * hd;
   TW* ko = own_k + (own_base + r) * (int64_t)(nkv * hd);
@@ -186,91 +180,191 @@ __global__ void rope_split_kernel(float* __restrict__ qkv, int64_t ld, const flo
 }
 
 // ---------------------------------------------------------------- attention
-// One warp per (row, query head, key split).  Row r = s*T + t of state s sees the
-// cache keys of its split and -- in the last split -- the rows 0..t of its own
-// state, read from own_k / own_v at row own_base + s*T + t' (Sec. 3.6: the states
-// share one cache and never see each other).  Writes an un-normalised partial
-// (acc[hd], max, sum) per split; splits are merged in index order afterwards, so
-// the result depends on (C, nsplit) only.
+// Grid (key chunk, kv head, pair block).  A CTA stages 64-key tiles of one kv head's K
+// and V in shared memory and runs every (row, query head) pair of that kv head against
+// them, so the cache is read from HBM/L2 once per pair block instead of once per pair.
+// Chunks [0, n_cache_chunks) cover the verified cache, nsub tiles of 64 keys each with an
+// online softmax across the tiles; the remaining chunks cover the rows' own keys, 64
+// flattened rows per chunk, masked so that row (s, t) sees rows (s, t' <= t) only
+// (Sec. 3.6: states share the cache and never see each other).  q is rotated (RoPE) while
+// it is loaded.  Each (pair, chunk) leaves an un-normalised partial (acc[hd], max, sum);
+// attn_merge_kernel adds the chunks in index order, so the result depends on (C, R) only
+// through the fixed chunking and never on timing.
+constexpr int ATT_KEYS = 64;
+constexpr int ATT_WARPS = 8;
+constexpr int ATT_PPW = 8;
+constexpr int ATT_PAIRS = ATT_WARPS * ATT_PPW;
+constexpr int ATT_MAX_CACHE_CHUNKS = 16;
+
 template <typename TW, int HD>
-__global__ void attn_partial_kernel(const float* __restrict__ q, int64_t ldq,
-                                    const TW* __restrict__ ck, const TW* __restrict__ cv, int C,
-                                    const TW* __restrict__ own_k, const TW* __restrict__ own_v,
-                                    int64_t own_base, int R, int T, int nq, int nkv, int nsplit,
-                                    int chunk, float* __restrict__ part_acc,
-                                    float2* __restrict__ part_ml) {
-  constexpr int DPL = HD / 32;  // output dims per lane
-  extern __shared__ float smem_q[];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
-  const int64_t gw = (int64_t)blockIdx.x * wpb + warp;
-  const int64_t total = (int64_t)R * nq * nsplit;
-  if (gw >= total) return;
-  const int sp = (int)(gw % nsplit);
-  const int h = (int)((gw / nsplit) % nq);
-  const int r = (int)(gw / ((int64_t)nsplit * nq));
-  const int s = r / T, t = r % T, kvh = h / (nq / nkv);
-  const int64_t kvld = (int64_t)nkv * HD;
-
-  float* qs = smem_q + warp * HD;
-  const float scale = rsqrtf((float)HD) * 1.4426950408889634f;  // 1/sqrt(hd) * log2(e)
-  for (int c = lane; c < HD; c += 32) qs[c] = q[(int64_t)r * ldq + h * HD + c] * scale;
-  __syncwarp();
-
-  float m = -INFINITY, l = 0.f, acc[DPL];
-#pragma unroll
-  for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
-
-  const int k_begin = sp * chunk, k_end = min(C, (sp + 1) * chunk);
-  const int n_own = (sp == nsplit - 1) ? (t + 1) : 0;
-  const int n_cache = max(0, k_end - k_begin);
-  const int n_total = n_cache + n_own;
-  for (int b0 = 0; b0 < n_total; b0 += 32) {
-    const int idx = b0 + lane;
-    const TW* kp = nullptr;
-    const TW* vp = nullptr;
-    if (idx < n_cache) {
-      kp = ck + (int64_t)(k_begin + idx) * kvld + kvh * HD;
-      vp = cv + (int64_t)(k_begin + idx) * kvld + kvh * HD;
-    } else if (idx < n_total) {
-      const int64_t row = own_base + (int64_t)s * T + (idx - n_cache);
-      kp = own_k + row * kvld + kvh * HD;
-      vp = own_v + row * kvld + kvh * HD;
-    }
-    float sc = -INFINITY;
-    if (kp) {
-      float d0 = 0.f;
-#pragma unroll
-      for (int c = 0; c < HD; c += 8) {
-        float kv8[8];
-        load8(kp + c, kv8);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) d0 = fmaf(kv8[e], qs[c + e], d0);
-      }
-      sc = d0;
-    }
-    const float m_new = fmaxf(m, warp_max(sc));
-    const float corr = exp2f(m - m_new);
-    const float p = kp ? exp2f(sc - m_new) : 0.f;
-    l = l * corr + warp_sum(p);
-#pragma unroll
-    for (int i = 0; i < DPL; ++i) acc[i] *= corr;
-    const int nb = min(32, n_total - b0);
-    for (int kk = 0; kk < nb; ++kk) {
-      const float pk = __shfl_sync(0xffffffffu, p, kk);
-      const TW* vrow = reinterpret_cast<const TW*>(
-          __shfl_sync(0xffffffffffffffffull & 0xffffffffu, (unsigned long long)vp, kk));
-#pragma unroll
-      for (int i = 0; i < DPL; ++i) acc[i] = fmaf(pk, to_float(vrow[lane * DPL + i]), acc[i]);
-    }
-    m = m_new;
-  }
-  float* pa = part_acc + gw * HD;
-#pragma unroll
-  for (int i = 0; i < DPL; ++i) pa[lane * DPL + i] = acc[i];
-  if (lane == 0) part_ml[gw] = make_float2(m, l);
+constexpr int att_smem_bytes() {
+  return ATT_KEYS * (HD + 16 / (int)sizeof(TW)) * (int)sizeof(TW) + ATT_KEYS * HD * (int)sizeof(TW) +
+         ATT_PAIRS * HD * 4 + ATT_WARPS * ATT_KEYS * 4;
 }
 
-// Merge the splits of one (row, head) in index order and round to the operand type.
+template <int DPL> __device__ __forceinline__ void load_dpl(const float* p, float (&f)[DPL]) {
+  if (DPL == 4) { float4 v = *reinterpret_cast<const float4*>(p); f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
+  else { float2 v = *reinterpret_cast<const float2*>(p); f[0] = v.x; f[1] = v.y; }
+}
+template <int DPL> __device__ __forceinline__ void load_dpl(const __nv_bfloat16* p, float (&f)[DPL]) {
+  if (DPL == 4) {
+    uint2 u = *reinterpret_cast<const uint2*>(p);
+    f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
+    f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
+  } else {
+    uint32_t u = *reinterpret_cast<const uint32_t*>(p);
+    f[0] = __uint_as_float(u << 16); f[1] = __uint_as_float(u & 0xffff0000u);
+  }
+}
+
+template <typename TW, int HD>
+__global__ void __launch_bounds__(ATT_WARPS * 32)
+attn_tile_kernel(const float* __restrict__ qkv, int64_t ldq, const float2* __restrict__ cs,
+                 const TW* __restrict__ ck, const TW* __restrict__ cv, int C,
+                 const TW* __restrict__ own_k, const TW* __restrict__ own_v, int64_t own_base,
+                 int R, int T, int nq, int nkv, int n_cache_chunks, int nsub, int n_chunks,
+                 float* __restrict__ part_acc, float2* __restrict__ part_ml) {
+  constexpr int DPL = HD / 32;
+  constexpr int KLD = HD + 16 / (int)sizeof(TW);       // padded K row: conflict-free 16-byte reads
+  constexpr int VEC = 16 / (int)sizeof(TW);            // elements per 16-byte vector
+  constexpr int VPR = HD / VEC;                        // vectors per row
+  extern __shared__ __align__(16) unsigned char att_smem[];
+  TW* k_s = reinterpret_cast<TW*>(att_smem);
+  TW* v_s = k_s + ATT_KEYS * KLD;
+  float* q_s = reinterpret_cast<float*>(v_s + ATT_KEYS * HD);
+  float* p_s = q_s + ATT_PAIRS * HD;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x, kvh = blockIdx.y, pb = blockIdx.z;
+  const int G = nq / nkv, n_pairs = R * G, half = HD / 2;
+  const bool own_chunk = chunk >= n_cache_chunks;
+  const int64_t kvld = (int64_t)nkv * HD;
+  const float scale = rsqrtf((float)HD) * 1.4426950408889634f;  // 1/sqrt(hd) * log2(e)
+
+  // this warp's pairs: p = pb*ATT_PAIRS + pi*ATT_WARPS + warp
+  float m[ATT_PPW], l[ATT_PPW], acc[ATT_PPW][DPL];
+#pragma unroll
+  for (int pi = 0; pi < ATT_PPW; ++pi) {
+    m[pi] = -INFINITY; l[pi] = 0.f;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[pi][i] = 0.f;
+    const int p = pb * ATT_PAIRS + pi * ATT_WARPS + warp;
+    if (p < n_pairs) {
+      const int r = p / G, hq = kvh * G + p % G, t = r % T;
+      const float* qr = qkv + (int64_t)r * ldq + hq * HD;
+      float* qd = q_s + (warp * ATT_PPW + pi) * HD;
+      for (int c = lane; c < half; c += 32) {
+        const float a = qr[c], b = qr[c + half];
+        const float2 w = cs[(int64_t)t * half + c];
+        qd[c] = (a * w.x - b * w.y) * scale;
+        qd[c + half] = (b * w.x + a * w.y) * scale;
+      }
+    }
+  }
+  __syncwarp();
+
+  const int n_tiles = own_chunk ? 1 : nsub;
+  for (int st = 0; st < n_tiles; ++st) {
+    int key0, nkeys;
+    const TW *src_k, *src_v;
+    if (!own_chunk) {
+      key0 = (chunk * nsub + st) * ATT_KEYS;
+      nkeys = min(ATT_KEYS, C - key0);
+      src_k = ck + (int64_t)key0 * kvld + kvh * HD;
+      src_v = cv + (int64_t)key0 * kvld + kvh * HD;
+    } else {
+      key0 = (chunk - n_cache_chunks) * ATT_KEYS;       // first flattened own row of this chunk
+      nkeys = min(ATT_KEYS, R - key0);
+      src_k = own_k + (own_base + key0) * kvld + kvh * HD;
+      src_v = own_v + (own_base + key0) * kvld + kvh * HD;
+    }
+    if (nkeys <= 0) break;                               // uniform across the CTA
+    __syncthreads();                                     // previous tile fully consumed
+    for (int v = threadIdx.x; v < ATT_KEYS * VPR; v += blockDim.x) {
+      const int row = v / VPR, cv16 = v % VPR;
+      uint4 kk = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
+      if (row < nkeys) {
+        kk = *reinterpret_cast<const uint4*>(src_k + (int64_t)row * kvld + cv16 * VEC);
+        vv = *reinterpret_cast<const uint4*>(src_v + (int64_t)row * kvld + cv16 * VEC);
+      }
+      *reinterpret_cast<uint4*>(k_s + row * KLD + cv16 * VEC) = kk;
+      *reinterpret_cast<uint4*>(v_s + row * HD + cv16 * VEC) = vv;
+    }
+    __syncthreads();
+
+#pragma unroll
+    for (int pi = 0; pi < ATT_PPW; ++pi) {
+      const int p = pb * ATT_PAIRS + pi * ATT_WARPS + warp;
+      if (p >= n_pairs) continue;                        // warp-uniform
+      const int r = p / G;
+      bool ok0 = lane < nkeys, ok1 = lane + 32 < nkeys;
+      if (own_chunk) {
+        const int r0 = key0 + lane, r1 = key0 + lane + 32;
+        ok0 = ok0 && (r0 / T == r / T) && (r0 <= r);
+        ok1 = ok1 && (r1 / T == r / T) && (r1 <= r);
+      }
+      if (!__any_sync(0xffffffffu, ok0 || ok1)) continue;
+      const float* qd = q_s + (warp * ATT_PPW + pi) * HD;
+      const TW* k0 = k_s + lane * KLD;
+      const TW* k1 = k_s + (lane + 32) * KLD;
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll 4
+      for (int c = 0; c < HD; c += 8) {
+        float a[8], b[8];
+        load8(k0 + c, a);
+        load8(k1 + c, b);
+        const float4 q0 = *reinterpret_cast<const float4*>(qd + c);
+        const float4 q1 = *reinterpret_cast<const float4*>(qd + c + 4);
+        s0 = fmaf(a[0], q0.x, s0); s0 = fmaf(a[1], q0.y, s0); s0 = fmaf(a[2], q0.z, s0); s0 = fmaf(a[3], q0.w, s0);
+        s0 = fmaf(a[4], q1.x, s0); s0 = fmaf(a[5], q1.y, s0); s0 = fmaf(a[6], q1.z, s0); s0 = fmaf(a[7], q1.w, s0);
+        s1 = fmaf(b[0], q0.x, s1); s1 = fmaf(b[1], q0.y, s1); s1 = fmaf(b[2], q0.z, s1); s1 = fmaf(b[3], q0.w, s1);
+        s1 = fmaf(b[4], q1.x, s1); s1 = fmaf(b[5], q1.y, s1); s1 = fmaf(b[6], q1.z, s1); s1 = fmaf(b[7], q1.w, s1);
+      }
+      if (!ok0) s0 = -INFINITY;
+      if (!ok1) s1 = -INFINITY;
+      const float m_new = fmaxf(m[pi], warp_max(fmaxf(s0, s1)));
+      const float corr = exp2f(m[pi] - m_new);          // m = -inf on the first tile: exp2(-inf) = 0
+      const float p0 = ok0 ? exp2f(s0 - m_new) : 0.f;
+      const float p1 = ok1 ? exp2f(s1 - m_new) : 0.f;
+      l[pi] = l[pi] * corr + warp_sum(p0 + p1);
+      m[pi] = m_new;
+      float* pw = p_s + warp * ATT_KEYS;
+      __syncwarp();
+      pw[lane] = p0;
+      pw[lane + 32] = p1;
+      __syncwarp();
+      float o[DPL];
+#pragma unroll
+      for (int i = 0; i < DPL; ++i) o[i] = acc[pi][i] * corr;
+      const TW* vcol = v_s + lane * DPL;
+#pragma unroll 8
+      for (int k = 0; k < ATT_KEYS; ++k) {
+        float vv[DPL];
+        load_dpl<DPL>(vcol + k * HD, vv);
+        const float pk = pw[k];
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) o[i] = fmaf(pk, vv[i], o[i]);
+      }
+#pragma unroll
+      for (int i = 0; i < DPL; ++i) acc[pi][i] = o[i];
+    }
+  }
+
+#pragma unroll
+  for (int pi = 0; pi < ATT_PPW; ++pi) {
+    const int p = pb * ATT_PAIRS + pi * ATT_WARPS + warp;
+    if (p >= n_pairs) continue;
+    const int r = p / G, hq = kvh * G + p % G;
+    const int64_t idx = ((int64_t)r * nq + hq) * n_chunks + chunk;
+    float* pa = part_acc + idx * HD + lane * DPL;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) pa[i] = acc[pi][i];
+    if (lane == 0) part_ml[idx] = make_float2(m[pi], l[pi]);
+  }
+}
+
+// Merge the chunks of one (row, head) in index order and round to the operand type.
+// A chunk that held no visible key has max = -inf and weight 0.
 template <typename TO, int HD>
 __global__ void attn_merge_kernel(const float* __restrict__ part_acc, const float2* __restrict__ part_ml,
                                   int R, int nq, int nsplit, TO* __restrict__ out) {
@@ -281,6 +375,7 @@ __global__ void attn_merge_kernel(const float* __restrict__ part_acc, const floa
   float num = 0.f, den = 0.f;
   for (int sp = 0; sp < nsplit; ++sp) {
     const float2 ml = part_ml[rh * nsplit + sp];
+    if (ml.x == -INFINITY) continue;
     const float wgt = exp2f(ml.x - mx);
     num = fmaf(wgt, part_acc[(rh * nsplit + sp) * HD + c], num);
     den = fmaf(wgt, ml.y, den);

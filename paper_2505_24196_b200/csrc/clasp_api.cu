@@ -9,6 +9,7 @@
 
 #include <cstdio>
 #include <cstdlib>
+#include <array>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -17,6 +18,7 @@
 
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
+#include "engine.cuh"
 
 namespace {
 
@@ -53,6 +55,23 @@ struct Workspace {
   float2* att_ml;
   float* logits;
   float* partial;
+  // persistent layer engine
+  void* xn_m;
+  float* e_part;
+  float* e_att_acc;
+  float2* e_att_ml;
+  float* ss_a;
+  float* ss_m;
+  float* cosp;
+  float4* tile_best;
+  int* e_counters;
+  clasp::pk::Ctl* ctl;
+  CUtensorMap* wmaps;
+  clasp::pk::Job* jobs;
+  size_t e_part_bytes;
+  int e_chunk_cap;
+  int e_run_len;
+  int e_rcap;
   size_t bytes;
 };
 
@@ -67,6 +86,28 @@ bool config_ok(const clasp_config* c) {
   if (c->max_M < 0 || c->max_M > c->L || c->max_T < 1) return false;
   if (c->dtype != CLASP_FP32 && c->dtype != CLASP_BF16) return false;
   return true;
+}
+
+constexpr int ENGINE_SIZING_CTAS = 148;
+
+// Bytes of split-K partial tiles the layer engine needs with a grid of G CTAs: every CTA owns
+// sk_max_segs slots of (planes x rows x 128) floats in each product.
+size_t engine_part_bytes(const clasp_config& c, int G) {
+  namespace pk = clasp::pk;
+  const long long R = c.max_rows < pk::MAX_ROWS ? c.max_rows : pk::MAX_ROWS;
+  const long long Rh = c.max_head_rows < pk::MAX_ROWS ? c.max_head_rows : pk::MAX_ROWS;
+  const long long d = c.d_model, qd = (long long)c.n_q_heads * c.head_dim, kvd = (long long)c.n_kv_heads * c.head_dim;
+  auto tiles = [](long long n) { return (n + pk::BM - 1) / pk::BM; };
+  auto chunks = [](long long k) { return (k + pk::BK - 1) / pk::BK; };
+  auto need = [&](long long t, long long kc, long long planes, long long rows) {
+    return (size_t)G * pk::sk_max_segs(t, kc, G) * planes * rows * pk::BM * 4;
+  };
+  size_t m = need(tiles(qd) + 2 * tiles(kvd), chunks(d), 1, R);
+  size_t v = need(tiles(d), chunks(qd), 1, R); if (v > m) m = v;
+  v = need(tiles(c.d_ffn), chunks(d), 2, R); if (v > m) m = v;
+  v = need(tiles(d), chunks(c.d_ffn), 1, R); if (v > m) m = v;
+  v = need(tiles(c.vocab), chunks(d), 1, Rh); if (v > m) m = v;
+  return m;
 }
 
 // Lays the workspace out; with base == nullptr only the size is computed.
@@ -103,6 +144,29 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
   w.att_ml = (float2*)take(R * c.n_q_heads * att_chunks * sizeof(float2));
   w.logits = (float*)take((size_t)c.max_head_rows * c.vocab * 4);
   w.partial = (float*)take(PARTIAL_FLOATS * 4);
+  if (c.dtype == CLASP_BF16) {
+    // buffers of the persistent layer engine (sized for a grid of ENGINE_SIZING_CTAS)
+    namespace pk = clasp::pk;
+    const size_t Re = R < (size_t)pk::MAX_ROWS ? R : (size_t)pk::MAX_ROWS;
+    const size_t rcap = align_up(Re, 16);
+    const size_t n_dt = (d + pk::BM - 1) / pk::BM;
+    w.e_rcap = (int)rcap;
+    w.xn_m = take(rcap * d * 2);
+    w.e_part_bytes = engine_part_bytes(c, ENGINE_SIZING_CTAS);
+    w.e_part = (float*)take(w.e_part_bytes);
+    w.e_run_len = pk::ATT_KEYS * ((c.max_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32));
+    w.e_chunk_cap = (c.max_ctx + w.e_run_len - 1) / w.e_run_len + (int)((rcap + pk::ATT_KEYS - 1) / pk::ATT_KEYS);
+    w.e_att_acc = (float*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * c.head_dim * 4);
+    w.e_att_ml = (float2*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * sizeof(float2));
+    w.ss_a = (float*)take(n_dt * rcap * 4);
+    w.ss_m = (float*)take(n_dt * rcap * 4);
+    w.cosp = (float*)take(n_dt * (rcap + pk::MAX_ROWS) * 5 * 4);
+    w.tile_best = (float4*)take((size_t)((c.vocab + pk::BM - 1) / pk::BM) * pk::MAX_ROWS * sizeof(float4));
+    w.e_counters = (int*)take(MAX_COUNTERS * sizeof(int));
+    w.ctl = (pk::Ctl*)take(256);
+    w.wmaps = (CUtensorMap*)take(((size_t)c.L * 7 + 1) * sizeof(CUtensorMap));
+    w.jobs = (pk::Job*)take(((size_t)c.L + 4) * sizeof(pk::Job));
+  }
   w.bytes = off;
   return w;
 }
@@ -130,6 +194,16 @@ struct clasp_ctx {
   int cta_cap = 296;
   int smem_budget = 110 * 1024;
   int num_sms = 148;
+  // persistent layer engine
+  bool use_engine = false;
+  int e_G = 0;              // CTAs of the cooperative grid (one per SM)
+  int e_static_smem = 0;
+  int e_cnt_base[5] = {0, 0, 0, 0, 0};
+  std::vector<CUtensorMap> e_wmaps_host;
+  bool e_wmaps_dirty = true;
+  std::map<int, std::array<CUtensorMap, 4>> e_bmaps;           // by BN
+  std::map<std::pair<int, int>, CUtensorMap> e_headmaps;       // by (row offset, BN)
+  std::vector<clasp::pk::Job> e_jobs;
 };
 
 namespace {
@@ -428,6 +502,158 @@ int embed_rows(clasp_ctx* ctx, const int32_t* tokens, int n, float* out, int64_t
   return launch_check(ctx);
 }
 
+
+// ---------------------------------------------------------------- persistent layer engine
+// Host side of engine.cuh: builds the job list of a call and launches the cooperative
+// kernel once.  Used by the bf16 tensor-core configuration; the per-kernel sequences
+// above remain for the fp32 model, for CLASP_FLAG_FORCE_SIMT and for shapes the engine
+// does not take (more than 128 rows).
+namespace pk = clasp::pk;
+
+int engine_setup(clasp_ctx* ctx) {
+  const clasp_config& c = ctx->cfg;
+  ctx->use_engine = false;
+  if (!ctx->use_tc || getenv("CLASP_NO_ENGINE")) return CLASP_OK;
+  int dev = 0, coop = 0, optin = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  CUDA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+  CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+  if (!coop) return CLASP_OK;
+  const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
+  auto tiles = [](int n) { return (n + pk::BM - 1) / pk::BM; };
+  const int t_qkv = tiles(qd) + 2 * tiles(kvd), t_o = tiles(d), t_gu = tiles(c.d_ffn), t_down = tiles(d);
+  const int t_head = tiles(c.vocab);
+  ctx->e_cnt_base[0] = 0;
+  ctx->e_cnt_base[1] = t_qkv;
+  ctx->e_cnt_base[2] = t_qkv + t_o;
+  ctx->e_cnt_base[3] = t_qkv + t_o + t_gu;
+  ctx->e_cnt_base[4] = t_qkv + t_o + t_gu + t_down;
+  if (ctx->e_cnt_base[4] + t_head > MAX_COUNTERS) return CLASP_OK;
+  cudaFuncAttributes fa;
+  CUDA_TRY(cudaFuncGetAttributes(&fa, pk::engine_kernel));
+  ctx->e_static_smem = (int)fa.sharedSizeBytes;
+  const int dyn_max = optin - ctx->e_static_smem;
+  if (dyn_max < 1024 + 2 * (pk::A_TILE_BYTES + 128 * 128) + pk::SCRATCH_BYTES) return CLASP_OK;
+  CUDA_TRY(cudaFuncSetAttribute(pk::engine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
+  int G = ctx->num_sms;
+  if (const char* e = getenv("CLASP_ENGINE_CTAS")) {
+    const int v = atoi(e);
+    if (v >= 1 && v < G) G = v;
+  }
+  if (engine_part_bytes(c, G) > ctx->ws.e_part_bytes) return CLASP_OK;
+  ctx->e_G = G;
+  ctx->e_wmaps_host.assign((size_t)c.L * 7 + 1, CUtensorMap{});
+  ctx->e_wmaps_dirty = true;
+  ctx->use_engine = true;
+  return CLASP_OK;
+}
+
+// weight + visible K/V bytes one job must move (for the per-launch bandwidth figure)
+double job_bytes(const clasp_ctx* ctx, const pk::Job& J) {
+  const clasp_config& c = ctx->cfg;
+  const double d = c.d_model, qd = (double)c.n_q_heads * c.head_dim, kvd = (double)c.n_kv_heads * c.head_dim;
+  if (J.type == pk::JOB_HEAD) return 2.0 * c.vocab * d;
+  if (J.type != pk::JOB_LAYER) return 0.0;
+  const double keys = J.uniform ? J.C + J.T : J.C;
+  return 2.0 * (d * (qd + 2 * kvd) + qd * d + 3.0 * d * c.d_ffn) + 2.0 * keys * kvd * 2.0;
+}
+
+// Launch the engine over ctx->e_jobs.  Rmax: most rows of any job; head_off: first row of the
+// previous job that the head job (if any) reads.
+int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
+  const clasp_config& c = ctx->cfg;
+  Workspace& ws = ctx->ws;
+  if (ctx->e_jobs.empty()) return CLASP_OK;
+  if (Rmax > pk::MAX_ROWS || (int)ctx->e_jobs.size() > c.L + 4) return CLASP_ERR_CAPACITY;
+  const int d = c.d_model, qd = c.n_q_heads * c.head_dim;
+  const int rows_cap = c.max_rows;
+  const int BN = Rmax <= 16 ? 16 : (Rmax + 15) / 16 * 16;
+  int dev = 0, optin = 0;
+  CUDA_TRY(cudaGetDevice(&dev));
+  CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+  const int slot_bytes = pk::A_TILE_BYTES + BN * pk::BK * 2;
+  int n_slots = (optin - ctx->e_static_smem - 1024 - pk::SCRATCH_BYTES) / slot_bytes;
+  if (n_slots > pk::MAX_SLOTS) n_slots = pk::MAX_SLOTS;
+  if (const char* e = getenv("CLASP_ENGINE_SLOTS")) {
+    const int v = atoi(e);
+    if (v >= 2 && v < n_slots) n_slots = v;
+  }
+  if (n_slots < 2) return CLASP_ERR_CAPACITY;
+  const size_t dyn = 1024 + (size_t)n_slots * slot_bytes + pk::SCRATCH_BYTES;
+
+  auto bm = ctx->e_bmaps.find(BN);
+  if (bm == ctx->e_bmaps.end()) {
+    std::array<CUtensorMap, 4> m;
+    int rc = 0;
+    rc |= make_map(ctx, ws.xn, rows_cap, d, BN, &m[0]);
+    rc |= make_map(ctx, ws.attn, rows_cap, qd, BN, &m[1]);
+    rc |= make_map(ctx, ws.xn_m, rows_cap, d, BN, &m[2]);
+    rc |= make_map(ctx, ws.act, rows_cap, c.d_ffn, BN, &m[3]);
+    if (rc) return CLASP_ERR_CUDA;
+    bm = ctx->e_bmaps.emplace(BN, m).first;
+  }
+  auto hk = std::make_pair(head_off, BN);
+  auto hm = ctx->e_headmaps.find(hk);
+  if (hm == ctx->e_headmaps.end()) {
+    CUtensorMap m;
+    if (make_map(ctx, (const bf16*)ws.xn + (size_t)head_off * d, rows_cap - head_off, d, BN, &m)) return CLASP_ERR_CUDA;
+    hm = ctx->e_headmaps.emplace(hk, m).first;
+  }
+  if (ctx->e_wmaps_dirty) {
+    CUDA_TRY(cudaMemcpyAsync(ws.wmaps, ctx->e_wmaps_host.data(), ctx->e_wmaps_host.size() * sizeof(CUtensorMap),
+                             cudaMemcpyHostToDevice, ctx->stream));
+    ctx->e_wmaps_dirty = false;
+  }
+  CUDA_TRY(cudaMemcpyAsync(ws.jobs, ctx->e_jobs.data(), ctx->e_jobs.size() * sizeof(pk::Job),
+                           cudaMemcpyHostToDevice, ctx->stream));
+  CUDA_TRY(cudaMemsetAsync(ws.ctl, 0, 8, ctx->stream));  // barrier counter and abort flag; status is sticky
+  CUDA_TRY(cudaMemsetAsync(ws.e_counters, 0, MAX_COUNTERS * sizeof(int), ctx->stream));
+
+  pk::Params P{};
+  P.c.L = c.L; P.c.d = d; P.c.qd = qd; P.c.kvd = c.n_kv_heads * c.head_dim; P.c.hd = c.head_dim;
+  P.c.nq = c.n_q_heads; P.c.nkv = c.n_kv_heads; P.c.dffn = c.d_ffn; P.c.vocab = c.vocab; P.c.eps = c.rms_eps;
+  P.c.G = ctx->e_G; P.c.Rcap = ws.e_rcap; P.c.n_dt = (d + pk::BM - 1) / pk::BM; P.c.run_len = ws.e_run_len;
+  P.c.chunk_cap = ws.e_chunk_cap;
+  for (int k = 0; k < 5; ++k) P.c.cnt_base[k] = ctx->e_cnt_base[k];
+  P.c.BN = BN; P.c.n_slots = n_slots; P.c.slot_bytes = slot_bytes;
+  P.b.xn_a = (bf16*)ws.xn; P.b.xn_m = (bf16*)ws.xn_m; P.b.attn = (bf16*)ws.attn; P.b.act = (bf16*)ws.act;
+  P.b.q = ws.qkv; P.b.x1 = ws.x1; P.b.Gbuf = ws.G; P.b.part = ws.e_part; P.b.att_acc = ws.e_att_acc;
+  P.b.att_ml = ws.e_att_ml; P.b.ss_a = ws.ss_a; P.b.ss_m = ws.ss_m; P.b.cosp = ws.cosp;
+  P.b.tile_best = ws.tile_best; P.b.counters = ws.e_counters; P.b.rope = ws.rope;
+  P.jobs = ws.jobs; P.n_jobs = (int)ctx->e_jobs.size(); P.wmaps = ws.wmaps; P.ctl = ws.ctl;
+
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (ctx->profiling) {
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return CLASP_ERR_CUDA;
+    cudaEventRecord(e0, ctx->stream);
+  }
+  void* args[] = {(void*)&bm->second[0], (void*)&bm->second[1], (void*)&bm->second[2], (void*)&bm->second[3],
+                  (void*)&hm->second, (void*)&P};
+  cudaError_t err = cudaLaunchCooperativeKernel((const void*)pk::engine_kernel, dim3(ctx->e_G), dim3(pk::THREADS),
+                                                args, dyn, ctx->stream);
+  if (ctx->profiling) {
+    cudaEventRecord(e1, ctx->stream);
+    ctx->prof_events.emplace_back(e0, e1);
+    for (const pk::Job& J : ctx->e_jobs) ctx->prof_bytes += job_bytes(ctx, J);
+  }
+  ctx->launches += 1;
+  return err == cudaSuccess ? CLASP_OK : CLASP_ERR_CUDA;
+}
+
+// a decoder-layer job with the fields every caller sets the same way
+pk::Job layer_job(clasp_ctx* ctx, int l, int S, int T, int C, bool uniform, const clasp_kv_layer& kv, int64_t pos0) {
+  const clasp_config& c = ctx->cfg;
+  pk::Job J{};
+  J.type = pk::JOB_LAYER; J.layer = l; J.S = S; J.T = T; J.R = S * T; J.C = C; J.uniform = uniform ? 1 : 0;
+  J.norm_in = ctx->layers[l].attn_norm; J.norm_mlp = ctx->layers[l].mlp_norm;
+  J.ck = (const bf16*)kv.k; J.cv = (const bf16*)kv.v;
+  J.ok = uniform ? (bf16*)kv.k : (bf16*)ctx->ws.own_k;
+  J.ov = uniform ? (bf16*)kv.v : (bf16*)ctx->ws.own_v;
+  J.own_base = uniform ? pos0 : 0;
+  (void)c;
+  return J;
+}
+
 }  // namespace
 
 // =============================================================== C ABI
@@ -492,6 +718,12 @@ int clasp_create(const clasp_config* cfg, void* workspace, size_t workspace_byte
     delete ctx;
     return CLASP_ERR_CUDA;
   }
+  if (ctx->use_tc) {
+    if (engine_setup(ctx) != CLASP_OK || cudaMemsetAsync(ws.ctl, 0, 256, ctx->stream) != cudaSuccess) {
+      delete ctx;
+      return CLASP_ERR_CUDA;
+    }
+  }
   *out = ctx;
   return CLASP_OK;
 }
@@ -519,6 +751,12 @@ int clasp_load_layers(clasp_ctx* ctx, int32_t first, int32_t count, const clasp_
       rc |= make_map(ctx, lw.w_up, c.d_ffn, d, clasp::tc::BM, &m.w_up);
       rc |= make_map(ctx, lw.w_down, d, c.d_ffn, clasp::tc::BM, &m.w_down);
       if (rc) return CLASP_ERR_CUDA;
+      if (ctx->use_engine) {
+        CUtensorMap* dst = &ctx->e_wmaps_host[(size_t)(first + k) * 7];
+        dst[0] = m.wq; dst[1] = m.wk; dst[2] = m.wv; dst[3] = m.wo; dst[4] = m.w_gate; dst[5] = m.w_up;
+        dst[6] = m.w_down;
+        ctx->e_wmaps_dirty = true;
+      }
     }
     ctx->loaded[first + k] = 1;
   }
@@ -534,6 +772,10 @@ int clasp_load_head(clasp_ctx* ctx, const void* embed, const float* final_norm, 
   ctx->lm_head = lm_head;
   if (ctx->use_tc && make_map(ctx, lm_head, ctx->cfg.vocab, ctx->cfg.d_model, clasp::tc::BM, &ctx->lm_head_map))
     return CLASP_ERR_CUDA;
+  if (ctx->use_engine) {
+    ctx->e_wmaps_host[(size_t)ctx->cfg.L * 7] = ctx->lm_head_map;
+    ctx->e_wmaps_dirty = true;
+  }
   return CLASP_OK;
 }
 
@@ -549,6 +791,12 @@ int clasp_layer_forward(clasp_ctx* ctx, int32_t layer, const float* x_in, int64_
   if (!ctx->loaded[layer]) return CLASP_ERR_NOT_LOADED;
   int rc = rope_table(ctx, T, pos0);
   if (rc) return rc;
+  if (ctx->use_engine && S * T <= pk::MAX_ROWS && (!write_kv || pos0 == ctx_len)) {
+    pk::Job J = layer_job(ctx, layer, S, T, ctx_len, write_kv != 0, *kv_layer, pos0);
+    J.prep = 1; J.x_in = x_in; J.ldx = in_stride; J.x_out = x_out; J.ldo = out_stride;
+    ctx->e_jobs.assign(1, J);
+    return engine_launch(ctx, S * T, 0);
+  }
   return run_layer_any(ctx, layer, x_in, in_stride, S, T, ctx_len, pos0, *kv_layer, write_kv != 0, x_out,
                        out_stride);
 }
@@ -574,6 +822,40 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
   if (rc) return rc;
   if ((rc = rope_table(ctx, T, pos0))) return rc;
   const int64_t Td = (int64_t)T * d;
+  if (ctx->use_engine && M > 0 && M * T <= pk::MAX_ROWS) {
+    // one cooperative launch for the whole search: step i = (layer i-1 over the candidate
+    // states) + (Eq. 2 select); row 0 of the g table is x_i itself and is never stored
+    clasp::dp_origin_kernel<<<1, 32, 0, ctx->stream>>>(scores, ws.choice);
+    if ((rc = launch_check(ctx))) return rc;
+    ctx->e_jobs.clear();
+    int cur = 0;
+    for (int i = 1; i <= L; ++i) {
+      const int ell = (i - 1 < M) ? i - 1 : M;
+      pk::Job J{};
+      if (ell > 0) {
+        J = layer_job(ctx, i - 1, ell, T, ctx_len, false, kv[i - 1], pos0);
+        J.x_in = ws.grow[cur] + Td; J.ldx = d; J.dp = 1;
+      } else {
+        J.type = pk::JOB_SELECT; J.T = T;
+      }
+      J.i = i; J.ell = ell; J.diag = i <= M ? 1 : 0; J.M = M;
+      J.x_i = hidden_states + (int64_t)i * layer_stride;
+      J.x_im1 = hidden_states + (int64_t)(i - 1) * layer_stride;
+      J.x_tok_stride = token_stride;
+      J.g_prev = ws.grow[cur]; J.g_next = ws.grow[cur ^ 1];
+      J.D = scores + (int64_t)i * (M + 1);
+      J.margin = margins ? margins + (int64_t)i * (M + 1) : nullptr;
+      J.choice = ws.choice + (int64_t)i * (M + 1);
+      J.forced = forced_choice ? forced_choice + (int64_t)i * (M + 1) : nullptr;
+      J.norm_next = i < L ? ctx->layers[i].attn_norm : nullptr;
+      J.g_final = (i == L) ? g_final : nullptr;
+      ctx->e_jobs.push_back(J);
+      cur ^= 1;
+    }
+    if ((rc = engine_launch(ctx, M * T, 0))) return rc;
+    clasp::backtrack_kernel<<<1, 32, 0, ctx->stream>>>(ws.choice, L, M, skip_mask);
+    return launch_check(ctx);
+  }
   {
     clasp::DpStepArgs a0{};  // g[0][0] = x_0, D[0][0] = 1: the b == 0 path of a step over x_0 itself
     a0.x_i = hidden_states; a0.x_tok_stride = token_stride; a0.G = ws.G; a0.g_prev = ws.grow[0];
@@ -630,6 +912,35 @@ int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0,
   const int d = c.d_model, L = c.L;
   int rc;
   if ((rc = rope_table(ctx, n, pos0))) return rc;
+  if (ctx->use_engine && n <= pk::MAX_ROWS) {
+    // embedding gather, then every layer and the head in one cooperative launch
+    float* h0 = hidden_out ? hidden_out : ctx->ws.hping;
+    const int64_t ld = hidden_out ? (int64_t)(L + 1) * d : d;
+    if ((rc = embed_rows(ctx, tokens, n, h0, ld))) return rc;
+    ctx->e_jobs.clear();
+    float* a = ctx->ws.hping;
+    float* b = ctx->ws.hpong;
+    for (int l = 0; l < L; ++l) {
+      pk::Job J = layer_job(ctx, l, 1, n, pos0, true, kv[l], pos0);
+      J.prep = l == 0 ? 1 : 0;
+      if (hidden_out) {
+        J.x_in = hidden_out + (int64_t)l * d; J.x_out = hidden_out + (int64_t)(l + 1) * d;
+      } else {
+        J.x_in = a; J.x_out = b;
+        float* t = a; a = b; b = t;
+      }
+      J.ldx = ld; J.ldo = ld;
+      J.norm_next = l + 1 < L ? ctx->layers[l + 1].attn_norm : (n_head_rows > 0 ? ctx->final_norm : nullptr);
+      ctx->e_jobs.push_back(J);
+    }
+    if (n_head_rows > 0) {
+      pk::Job H{};
+      H.type = pk::JOB_HEAD; H.R = n_head_rows; H.T = 1; H.row_off = n - n_head_rows;
+      H.argmax_out = argmax_out;
+      ctx->e_jobs.push_back(H);
+    }
+    return engine_launch(ctx, n, n_head_rows > 0 ? n - n_head_rows : 0);
+  }
   const float* x;
   int64_t ldx;
   if (hidden_out) {
@@ -670,6 +981,27 @@ int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int
   float* a = ctx->ws.hping;
   float* b = ctx->ws.hpong;
   if ((rc = embed_rows(ctx, token_in, 1, a, d))) return rc;
+  int n_kept = 0;
+  for (int l = 0; l < c.L; ++l) n_kept += skip_mask_host[l] ? 0 : 1;
+  if (ctx->use_engine && n_kept > 0) {
+    ctx->e_jobs.clear();
+    for (int l = 0; l < c.L; ++l) {
+      if (skip_mask_host[l]) continue;  // skipped layer: nothing read, nothing written
+      if (!kv[l].k || !kv[l].v) return CLASP_ERR_INVALID_ARG;
+      pk::Job J = layer_job(ctx, l, 1, 1, pos, true, kv[l], pos);
+      J.prep = ctx->e_jobs.empty() ? 1 : 0;
+      J.x_in = a; J.ldx = d; J.x_out = b; J.ldo = d;
+      float* t = a; a = b; b = t;
+      ctx->e_jobs.push_back(J);
+    }
+    for (size_t k = 0; k + 1 < ctx->e_jobs.size(); ++k)
+      ctx->e_jobs[k].norm_next = ctx->layers[ctx->e_jobs[k + 1].layer].attn_norm;
+    ctx->e_jobs.back().norm_next = ctx->final_norm;
+    pk::Job H{};
+    H.type = pk::JOB_HEAD; H.R = 1; H.T = 1; H.row_off = 0; H.argmax_out = token_out; H.top1_out = top1_prob_out;
+    ctx->e_jobs.push_back(H);
+    return engine_launch(ctx, 1, 0);
+  }
   for (int l = 0; l < c.L; ++l) {
     if (skip_mask_host[l]) continue;  // skipped layer: state passes through, nothing read or written
     if (!kv[l].k || !kv[l].v) return CLASP_ERR_INVALID_ARG;
@@ -825,6 +1157,15 @@ int clasp_last_device_status(clasp_ctx* ctx) {
   int st = 0;
   if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return CLASP_ERR_CUDA;
   if (cudaMemcpy(&st, ctx->ws.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return CLASP_ERR_CUDA;
+  if (ctx->use_engine) {
+    int est = 0;
+    if (cudaMemcpy(&est, &ctx->ws.ctl->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+      return CLASP_ERR_CUDA;
+    if (est != 0) {
+      cudaMemset(ctx->ws.ctl, 0, sizeof(clasp::pk::Ctl));
+      st = 1;
+    }
+  }
   if (st != 0) {
     cudaMemset(ctx->ws.status, 0, sizeof(int));
     cudaMemset(ctx->ws.counters, 0, MAX_COUNTERS * sizeof(int));

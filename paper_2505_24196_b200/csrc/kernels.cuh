@@ -509,6 +509,14 @@ __global__ void fill_tables_kernel(float* D, float* margin, uint8_t* choice, int
   choice[idx] = 255;
 }
 
+// D(0, 0) = 1 and its choice entry: the origin of the table (g[0][0] = x_0)
+__global__ void dp_origin_kernel(float* D, uint8_t* choice) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    D[0] = 1.0f;
+    choice[0] = 0;
+  }
+}
+
 // rows of floats: dst[r, :] = src[r, :] (strided)
 __global__ void copy_rows_kernel(const float* __restrict__ src, int64_t lds, float* __restrict__ dst,
                                  int64_t ldd, int d) {

@@ -258,6 +258,15 @@ int clasp_profile_gemm(clasp_ctx* ctx, int32_t enable, int64_t* n_launches, doub
 /* Number of kernel launches the context has enqueued so far (host counter). */
 int64_t clasp_launch_count(const clasp_ctx* ctx);
 
+/* Step tracing of the persistent layer kernel (measurement aid; no counterpart in the
+ * paper).  `stamps` is DEVICE memory of n_ctas * cap_per_cta uint64 (borrowed until it is
+ * replaced or cleared with NULL): during every following search / verify / draft call the
+ * kernel's CTA c writes the %globaltimer value (ns) of its k-th step boundary to
+ * stamps[c * cap_per_cta + k] (a boundary = entering or leaving a grid-wide barrier; steps
+ * beyond cap_per_cta are not recorded).  *n_ctas (HOST, may be NULL) receives the grid
+ * size, 0 when the context does not use the persistent kernel. */
+int clasp_engine_trace(clasp_ctx* ctx, uint64_t* stamps, int32_t cap_per_cta, int32_t* n_ctas);
+
 const char* clasp_strerror(int code);
 
 #ifdef __cplusplus

@@ -21,7 +21,7 @@ FLAG_FORCE_SIMT = 1
 
 SYMBOLS = ["clasp_workspace_bytes", "clasp_create", "clasp_destroy", "clasp_load_layers", "clasp_load_head",
            "clasp_dp_search", "clasp_verify", "clasp_draft_forward", "clasp_accept", "clasp_layer_forward",
-           "clasp_gemm_xwT", "clasp_gemm_xwT_noalloc", "clasp_profile_gemm", "clasp_last_device_status", "clasp_launch_count", "clasp_strerror"]
+           "clasp_gemm_xwT", "clasp_gemm_xwT_noalloc", "clasp_profile_gemm", "clasp_last_device_status", "clasp_launch_count", "clasp_engine_trace", "clasp_strerror"]
 
 
 class ClaspConfig(C.Structure):
@@ -91,6 +91,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.clasp_last_device_status.argtypes = [vp]
     lib.clasp_launch_count.restype = C.c_int64
     lib.clasp_launch_count.argtypes = [vp]
+    lib.clasp_engine_trace.restype = C.c_int
+    lib.clasp_engine_trace.argtypes = [vp, vp, i32, C.POINTER(i32)]
     lib.clasp_strerror.restype = C.c_char_p
     lib.clasp_strerror.argtypes = [C.c_int]
     _lib = lib
@@ -264,3 +266,13 @@ class Clasp:
 
     def launch_count(self) -> int:
         return self.lib.clasp_launch_count(self.handle)
+
+    def engine_ctas(self) -> int:
+        n = C.c_int32()
+        _check(self.lib.clasp_engine_trace(self.handle, None, 0, C.byref(n)), "clasp_engine_trace")
+        return n.value
+
+    def set_trace(self, stamps: Optional[torch.Tensor], cap_per_cta: int = 0):
+        """stamps: int64 device tensor [n_ctas, cap_per_cta] or None to stop tracing."""
+        self._trace = stamps
+        _check(self.lib.clasp_engine_trace(self.handle, _ptr(stamps), cap_per_cta, None), "clasp_engine_trace")

@@ -68,6 +68,7 @@ struct Workspace {
   clasp::pk::Ctl* ctl;
   CUtensorMap* wmaps;
   clasp::pk::Job* jobs;
+  int* tabs;
   size_t e_part_bytes;
   int e_chunk_cap;
   int e_run_len;
@@ -89,6 +90,8 @@ bool config_ok(const clasp_config* c) {
 }
 
 constexpr int ENGINE_SIZING_CTAS = 148;
+constexpr int ENGINE_MAX_CTAS = 192;
+constexpr size_t ENGINE_TAB_INTS = 5 * (ENGINE_MAX_CTAS + 1) + 2 * (4096 + 5) + 5 * ENGINE_MAX_CTAS;
 
 // Bytes of split-K partial tiles the layer engine needs with a grid of G CTAs: every CTA owns
 // sk_max_segs slots of (planes x rows x 128) floats in each product.
@@ -166,6 +169,7 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
     w.ctl = (pk::Ctl*)take(256);
     w.wmaps = (CUtensorMap*)take(((size_t)c.L * 7 + 1) * sizeof(CUtensorMap));
     w.jobs = (pk::Job*)take(((size_t)c.L + 4) * sizeof(pk::Job));
+    w.tabs = (int*)take(ENGINE_TAB_INTS * sizeof(int));
   }
   w.bytes = off;
   return w;
@@ -199,11 +203,15 @@ struct clasp_ctx {
   int e_G = 0;              // CTAs of the cooperative grid (one per SM)
   int e_static_smem = 0;
   int e_cnt_base[5] = {0, 0, 0, 0, 0};
+  int e_tab_lo[5], e_tab_seg0[5], e_tab_segc[5], e_segmax[5];
+  int e_pf_max = 0;
   std::vector<CUtensorMap> e_wmaps_host;
   bool e_wmaps_dirty = true;
   std::map<int, std::array<CUtensorMap, 4>> e_bmaps;           // by BN
   std::map<std::pair<int, int>, CUtensorMap> e_headmaps;       // by (row offset, BN)
   std::vector<clasp::pk::Job> e_jobs;
+  unsigned long long* e_trace = nullptr;
+  int e_trace_cap = 0;
 };
 
 namespace {
@@ -540,7 +548,41 @@ int engine_setup(clasp_ctx* ctx) {
     const int v = atoi(e);
     if (v >= 1 && v < G) G = v;
   }
-  if (engine_part_bytes(c, G) > ctx->ws.e_part_bytes) return CLASP_OK;
+  if (engine_part_bytes(c, G) > ctx->ws.e_part_bytes || G > ENGINE_MAX_CTAS) return CLASP_OK;
+  // stream-K tables: unit range of every CTA and, per output tile, the CTAs that hold a partial tile
+  {
+    const int kc_d = (d + pk::BK - 1) / pk::BK, kc_q = (qd + pk::BK - 1) / pk::BK, kc_f = (c.d_ffn + pk::BK - 1) / pk::BK;
+    const int n_tiles[5] = {t_qkv, t_o, t_gu, t_down, t_head};
+    const int n_kc[5] = {kc_d, kc_q, kc_d, kc_f, kc_d};
+    std::vector<int> tab;
+    for (int k = 0; k < 5; ++k) {
+      const long long U = (long long)n_tiles[k] * n_kc[k];
+      ctx->e_segmax[k] = pk::sk_max_segs(n_tiles[k], n_kc[k], G);
+      ctx->e_tab_lo[k] = (int)tab.size();
+      std::vector<int> lo(G + 1);
+      for (int cc = 0; cc <= G; ++cc) lo[cc] = (int)(U * cc / G);
+      tab.insert(tab.end(), lo.begin(), lo.end());
+      std::vector<int> seg0(n_tiles[k] + 1, 0), segc;
+      for (int t = 0; t < n_tiles[k]; ++t) {
+        seg0[t] = (int)segc.size();
+        const long long q0 = (long long)t * n_kc[k], q1 = q0 + n_kc[k];
+        for (int cc = 0; cc < G; ++cc)
+          if (lo[cc + 1] > lo[cc] && lo[cc] < q1 && lo[cc + 1] > q0) segc.push_back(cc);
+      }
+      seg0[n_tiles[k]] = (int)segc.size();
+      ctx->e_tab_seg0[k] = (int)tab.size();
+      tab.insert(tab.end(), seg0.begin(), seg0.end());
+      ctx->e_tab_segc[k] = (int)tab.size();
+      tab.insert(tab.end(), segc.begin(), segc.end());
+    }
+    if (tab.size() > ENGINE_TAB_INTS) return CLASP_OK;
+    CUDA_TRY(cudaMemcpyAsync(ctx->ws.tabs, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+    CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+  }
+  if (const char* e = getenv("CLASP_ENGINE_PF")) {
+    const int v = atoi(e);
+    if (v >= 0 && v <= 256) ctx->e_pf_max = v;
+  }
   ctx->e_G = G;
   ctx->e_wmaps_host.assign((size_t)c.L * 7 + 1, CUtensorMap{});
   ctx->e_wmaps_dirty = true;
@@ -615,12 +657,18 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   P.c.G = ctx->e_G; P.c.Rcap = ws.e_rcap; P.c.n_dt = (d + pk::BM - 1) / pk::BM; P.c.run_len = ws.e_run_len;
   P.c.chunk_cap = ws.e_chunk_cap;
   for (int k = 0; k < 5; ++k) P.c.cnt_base[k] = ctx->e_cnt_base[k];
-  P.c.BN = BN; P.c.n_slots = n_slots; P.c.slot_bytes = slot_bytes;
+  P.c.BN = BN; P.c.n_slots = n_slots; P.c.slot_bytes = slot_bytes; P.c.pf_max = ctx->e_pf_max;
+  for (int k = 0; k < 5; ++k) {
+    P.c.tab_lo[k] = ctx->e_tab_lo[k]; P.c.tab_seg0[k] = ctx->e_tab_seg0[k]; P.c.tab_segc[k] = ctx->e_tab_segc[k];
+    P.c.segmax[k] = ctx->e_segmax[k];
+  }
+  P.tabs = ws.tabs;
   P.b.xn_a = (bf16*)ws.xn; P.b.xn_m = (bf16*)ws.xn_m; P.b.attn = (bf16*)ws.attn; P.b.act = (bf16*)ws.act;
   P.b.q = ws.qkv; P.b.x1 = ws.x1; P.b.Gbuf = ws.G; P.b.part = ws.e_part; P.b.att_acc = ws.e_att_acc;
   P.b.att_ml = ws.e_att_ml; P.b.ss_a = ws.ss_a; P.b.ss_m = ws.ss_m; P.b.cosp = ws.cosp;
   P.b.tile_best = ws.tile_best; P.b.counters = ws.e_counters; P.b.rope = ws.rope;
   P.jobs = ws.jobs; P.n_jobs = (int)ctx->e_jobs.size(); P.wmaps = ws.wmaps; P.ctl = ws.ctl;
+  P.trace = ctx->e_trace; P.trace_cap = ctx->e_trace_cap;
 
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (ctx->profiling) {
@@ -1201,6 +1249,14 @@ int clasp_profile_gemm(clasp_ctx* ctx, int32_t enable, int64_t* n_launches, doub
 }
 
 int64_t clasp_launch_count(const clasp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int clasp_engine_trace(clasp_ctx* ctx, uint64_t* stamps, int32_t cap_per_cta, int32_t* n_ctas) {
+  if (!ctx || cap_per_cta < 0) return CLASP_ERR_INVALID_ARG;
+  if (n_ctas) *n_ctas = ctx->use_engine ? ctx->e_G : 0;
+  ctx->e_trace = (unsigned long long*)stamps;
+  ctx->e_trace_cap = stamps ? cap_per_cta : 0;
+  return CLASP_OK;
+}
 
 const char* clasp_strerror(int code) {
   switch (code) {

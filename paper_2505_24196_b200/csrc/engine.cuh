@@ -73,6 +73,12 @@ struct Cfg {
   int BN;          // activation rows padded to a multiple of 16 (MMA N)
   int n_slots;
   int slot_bytes;
+  int pf_max;      // weight tiles a CTA may prefetch into L2 beyond its ring while the ring is full
+  // stream-K tables (ints in Params::tabs), one set per product kind
+  int tab_lo[5];    // [G + 1] first unit of each CTA
+  int tab_seg0[5];  // [tiles + 1] first entry of each tile in the segment list
+  int tab_segc[5];  // segment list: CTA of every partial tile, tile-major, CTA order
+  int segmax[5];    // partial-tile slots per CTA
 };
 
 struct Bufs {
@@ -145,10 +151,14 @@ struct Params {
   const Job* jobs;
   int n_jobs;
   const CUtensorMap* wmaps;  // [L*7 + 1]
+  const int* tabs;
   Ctl* ctl;
+  unsigned long long* trace;  // optional [G, trace_cap] time stamps (ns) of the workers' steps
+  int trace_cap;
 };
 
 struct GemmDesc {
+  int kind;
   int tiles, kc, dual, n_mats, K;
   int mat_tiles[3], mat_N[3];
   int map_base, bmap, cnt_base;
@@ -156,6 +166,7 @@ struct GemmDesc {
 
 __device__ __forceinline__ GemmDesc make_desc(const Cfg& c, int kind, int layer) {
   GemmDesc g;
+  g.kind = kind;
   g.dual = 0; g.n_mats = 1;
   g.mat_N[0] = g.mat_N[1] = g.mat_N[2] = 0;
   if (kind == G_QKV) {
@@ -180,11 +191,11 @@ __device__ __forceinline__ GemmDesc make_desc(const Cfg& c, int kind, int layer)
   return g;
 }
 
-// units [lo, hi) of CTA c
-__device__ __forceinline__ void sk_range(const GemmDesc& g, int G, int c, long long& lo, long long& hi) {
-  const long long U = (long long)g.tiles * g.kc;
-  lo = U * c / G;
-  hi = U * (c + 1) / G;
+// units [lo, hi) of CTA c (host-built table: lo(c) = floor(c U / G))
+__device__ __forceinline__ void sk_range(const Params& p, const GemmDesc& g, int c, int& lo, int& hi) {
+  const int* t = p.tabs + p.c.tab_lo[g.kind];
+  lo = __ldg(t + c);
+  hi = __ldg(t + c + 1);
 }
 // most tiles one CTA can touch in a product (bounds the partial-tile slots per CTA)
 __host__ __device__ inline int sk_max_segs(long long tiles, long long kc, int G) {
@@ -276,21 +287,21 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctl* ct
   return false;
 }
 
-// Grid barrier of the worker threads (all 256 call it).  `epoch` counts barriers.
+// Grid barrier of the worker threads (all 256 call it).  `epoch` counts barriers.  Only one
+// thread fences and signals: the CTA barrier before it orders the other workers' writes first.
 __device__ __forceinline__ bool grid_barrier(const Params& p, Shared* sh, unsigned& epoch, int wtid) {
   ++epoch;
-  fence_proxy_async();  // operands written with ordinary stores are read by TMA afterwards
-  __threadfence();
   worker_sync();
   if (wtid == 0) {
     const unsigned target = epoch * (unsigned)p.c.G;
+    __threadfence();
     atomicAdd(&p.ctl->bar, 1u);
     bool ok = false;
     for (uint32_t it = 0; it < (1u << 24); ++it) {
       if (ld_acquire_u32(&p.ctl->bar) >= target) { ok = true; break; }
       if ((it & 63u) == 63u) {
         if (sh->abort || ld_volatile_i32(&p.ctl->abort)) break;
-        if (it > 4096u) __nanosleep(64);
+        if (it > 8192u) __nanosleep(64);
       }
     }
     if (!ok) {
@@ -319,33 +330,83 @@ struct Ring {
   }
 };
 
+// Walks the weight tiles of this CTA in the order they are consumed: products of a job,
+// jobs of the list.  Used twice by the weight producer: once for the loads into the ring
+// and once, running ahead, for L2 prefetches.
+struct TileIter {
+  int jb, ph, q, hi, half;
+  GemmDesc g;
+  __device__ void reset() { jb = 0; ph = -1; q = 0; hi = 0; half = 0; }
+  __device__ bool next(const Params& p, int& map_idx, int& x, int& y) {
+    for (;;) {
+      if (ph >= 0 && q < hi) {
+        int tile = q / g.kc;
+        x = (q - tile * g.kc) * BK;
+        int mat = 0;
+        while (mat + 1 < g.n_mats && tile >= g.mat_tiles[mat]) { tile -= g.mat_tiles[mat]; ++mat; }
+        map_idx = g.map_base + mat + half;
+        y = tile * BM;
+        if (g.dual && half == 0) half = 1;
+        else { half = 0; ++q; }
+        return true;
+      }
+      if (jb >= p.n_jobs) return false;
+      const Job& J = p.jobs[jb];
+      ++ph;
+      if (ph >= n_gemm_phases(J)) { ++jb; ph = -1; hi = 0; q = 0; continue; }
+      g = make_desc(p.c, gemm_kind(J, ph), J.layer);
+      sk_range(p, g, blockIdx.x, q, hi);
+      half = 0;
+    }
+  }
+};
+
 __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base) {
   const Cfg& c = p.c;
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
   Ring rg{0, 0};
-  for (int jb = 0; jb < p.n_jobs; ++jb) {
-    const Job& J = p.jobs[jb];
-    const int nph = n_gemm_phases(J);
-    for (int ph = 0; ph < nph; ++ph) {
-      const GemmDesc g = make_desc(c, gemm_kind(J, ph), J.layer);
-      long long lo, hi;
-      sk_range(g, c.G, blockIdx.x, lo, hi);
-      for (long long q = lo; q < hi; ++q) {
-        int tile = (int)(q / g.kc);
-        const int kx = (int)(q % g.kc) * BK;
-        int mat = 0;
-        while (mat + 1 < g.n_mats && tile >= g.mat_tiles[mat]) { tile -= g.mat_tiles[mat]; ++mat; }
-        for (int half = 0; half <= g.dual; ++half) {
-          if (!wait_bar(&sh->empty[rg.slot], (rg.round & 1u) ^ 1u, p.ctl, sh)) return;
-          const uint32_t full = tc::smem_u32(&sh->full[rg.slot]);
-          tc::mbar_expect_tx(full, A_TILE_BYTES);
-          tc::tma_load_2d(ring_base + rg.slot * c.slot_bytes, p.wmaps + g.map_base + mat + half, full, kx,
-                          tile * BM, pol);
-          rg.advance(c.n_slots);
+  TileIter ld, pf;
+  ld.reset();
+  pf.reset();
+  int ahead = 0;        // tiles the prefetch iterator is ahead of the load iterator
+  bool pf_live = c.pf_max > 0;
+  int mi, x, y;
+  while (ld.next(p, mi, x, y)) {
+    if (ahead > 0) --ahead;
+    else if (pf_live) { int a, b2, c2; pf_live = pf.next(p, a, b2, c2); }  // keep pf >= ld
+    // wait for the slot; while the ring is full, keep HBM busy by prefetching later tiles into L2
+    const uint32_t eb = tc::smem_u32(&sh->empty[rg.slot]);
+    const uint32_t par = (rg.round & 1u) ^ 1u;
+    bool ok = false;
+    for (uint32_t it = 0; it < WAIT_SLOW; ++it) {
+      if (tc::mbar_test(eb, par)) { ok = true; break; }
+      if (pf_live && ahead < c.pf_max) {
+        int pm, px, py;
+        pf_live = pf.next(p, pm, px, py);
+        if (pf_live) {
+          asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(p.wmaps + pm),
+                       "r"(px), "r"(py)
+                       : "memory");
+          ++ahead;
         }
+        continue;
+      }
+      if (it > WAIT_FAST) {
+        if (sh->abort || ld_volatile_i32(&p.ctl->abort)) { sh->abort = 1; return; }
+        __nanosleep(100);
       }
     }
+    if (!ok) {
+      atomicExch(&p.ctl->status, 1);
+      atomicExch(&p.ctl->abort, 1);
+      sh->abort = 1;
+      return;
+    }
+    const uint32_t full = tc::smem_u32(&sh->full[rg.slot]);
+    tc::mbar_expect_tx(full, A_TILE_BYTES);
+    tc::tma_load_2d(ring_base + rg.slot * c.slot_bytes, p.wmaps + mi, full, x, y, pol);
+    rg.advance(c.n_slots);
   }
 }
 
@@ -364,20 +425,21 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
       // the operand of this product exists once the workers passed the barrier before it
       if (!wait_bar(&sh->dep, seq & 1u, p.ctl, sh)) return;
       fence_proxy_async();
-      long long lo, hi;
-      sk_range(g, c.G, blockIdx.x, lo, hi);
-      for (long long q = lo; q < hi; ++q) {
-        const int kx = (int)(q % g.kc) * BK;
+      int lo, hi;
+      sk_range(p, g, blockIdx.x, lo, hi);
+      int kcx = lo % g.kc;
+      for (int q = lo; q < hi; ++q) {
         if (!wait_bar(&sh->empty[rg.slot], (rg.round & 1u) ^ 1u, p.ctl, sh)) return;
         const uint32_t full = tc::smem_u32(&sh->full[rg.slot]);
         tc::mbar_expect_tx(full, b_bytes);
-        tc::tma_load_2d(ring_base + rg.slot * c.slot_bytes + A_TILE_BYTES, bmaps[g.bmap], full, kx, 0, pol);
+        tc::tma_load_2d(ring_base + rg.slot * c.slot_bytes + A_TILE_BYTES, bmaps[g.bmap], full, kcx * BK, 0, pol);
         rg.advance(c.n_slots);
         if (g.dual) {  // the "up" slot reuses the operand tile of the "gate" slot before it
           if (!wait_bar(&sh->empty[rg.slot], (rg.round & 1u) ^ 1u, p.ctl, sh)) return;
           mbar_arrive(tc::smem_u32(&sh->full[rg.slot]));
           rg.advance(c.n_slots);
         }
+        if (++kcx == g.kc) kcx = 0;
       }
     }
   }
@@ -393,11 +455,11 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
     const int nph = n_gemm_phases(J);
     for (int ph = 0; ph < nph; ++ph) {
       const GemmDesc g = make_desc(c, gemm_kind(J, ph), J.layer);
-      long long lo, hi;
-      sk_range(g, c.G, blockIdx.x, lo, hi);
-      long long q = lo;
+      int lo, hi;
+      sk_range(p, g, blockIdx.x, lo, hi);
+      int q = lo;
       while (q < hi) {
-        const long long seg_end = min(hi, (q / g.kc + 1) * g.kc);
+        const int seg_end = min(hi, (q / g.kc + 1) * g.kc);
         const uint32_t buf = n_acc & 1u;
         if (!wait_bar(&sh->acc_empty[buf], ((n_acc >> 1) & 1u) ^ 1u, p.ctl, sh)) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -446,7 +508,22 @@ struct Worker {
   uint32_t n_acc;
   uint32_t n_dep;
 
-  __device__ __forceinline__ bool barrier() { return grid_barrier(p, sh, epoch, wtid); }
+  int n_mark;
+  // time stamp of a step boundary (tracing aid; one thread per CTA)
+  __device__ __forceinline__ void mark() {
+    if (p.trace != nullptr && wtid == 0 && n_mark < p.trace_cap) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+      p.trace[(long long)blockIdx.x * p.trace_cap + n_mark] = t;
+    }
+    ++n_mark;
+  }
+  __device__ __forceinline__ bool barrier() {
+    mark();
+    const bool ok = grid_barrier(p, sh, epoch, wtid);
+    mark();
+    return ok;
+  }
   __device__ __forceinline__ void release_operand() {  // lets warp 1 load the next product's operand
     if (wtid == 0) mbar_arrive(tc::smem_u32(&sh->dep));
     ++n_dep;
@@ -485,54 +562,86 @@ struct Worker {
         if (lane == 0) p.b.ss_a[(long long)t * c.Rcap + r] = ssq;
       }
     }
+    fence_proxy_async();
   }
 
-  // list of the partial tiles of `tile` in CTA order (thread 0) -> sh->seg_off, sh->n_seg
+  // number of partial tiles of `tile` (host-built table)
+  __device__ __forceinline__ int count_segments(const GemmDesc& g, int tile) const {
+    const int* t = p.tabs + p.c.tab_seg0[g.kind] + tile;
+    return __ldg(t + 1) - __ldg(t);
+  }
+  // offsets of the partial tiles of `tile`, in CTA order -> sh->seg_off (threads s < n_seg)
   __device__ void list_segments(const GemmDesc& g, int tile, int R) {
     const Cfg& c = p.c;
-    const long long U = (long long)g.tiles * g.kc;
-    const long long q0 = (long long)tile * g.kc, q1 = q0 + g.kc - 1;
-    const int c_lo = (int)(((q0 + 1) * c.G - 1) / U), c_hi = (int)(((q1 + 1) * c.G - 1) / U);
-    const int segmax = sk_max_segs(g.tiles, g.kc, c.G);
+    const int s0 = __ldg(p.tabs + c.tab_seg0[g.kind] + tile);
+    const int n = min(__ldg(p.tabs + c.tab_seg0[g.kind] + tile + 1) - s0, MAX_SEGS);
     const long long stride = (long long)(g.dual + 1) * R * BM;
-    int n = 0;
-    for (int cc = c_lo; cc <= c_hi && n < MAX_SEGS; ++cc) {
-      const long long lo = U * cc / c.G, hi = U * (cc + 1) / c.G;
-      if (hi <= lo) continue;
-      const int seg = tile - (int)(lo / g.kc);
-      sh->seg_off[n++] = ((long long)cc * segmax + seg) * stride;
+    if (wtid < n) {
+      const int cc = __ldg(p.tabs + c.tab_segc[g.kind] + s0 + wtid);
+      const int lo = __ldg(p.tabs + c.tab_lo[g.kind] + cc);
+      sh->seg_off[wtid] = ((long long)cc * c.segmax[g.kind] + (tile - lo / g.kc)) * stride;
     }
-    sh->n_seg = n;
-  }
-  __device__ static int count_segments(const GemmDesc& g, int tile, int G) {
-    const long long U = (long long)g.tiles * g.kc;
-    const long long q0 = (long long)tile * g.kc, q1 = q0 + g.kc - 1;
-    const int c_lo = (int)(((q0 + 1) * G - 1) / U), c_hi = (int)(((q1 + 1) * G - 1) / U);
-    if (U >= G) return c_hi - c_lo + 1;
-    int n = 0;
-    for (int cc = c_lo; cc <= c_hi; ++cc)
-      if (U * (cc + 1) / G > U * cc / G) ++n;
-    return n;
+    if (wtid == 0) sh->n_seg = n;
+    worker_sync();
   }
 
-  __device__ __forceinline__ float4 sum4(int plane, int r, int R) const {
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+  // sum over the partial tiles (CTA order) of 4 consecutive features of two rows at once;
+  // all loads of a batch are issued before the first add
+  __device__ __forceinline__ void sum4x2(int plane, int r0, int r1, bool two, int R, float4& a0, float4& a1) const {
+    a0 = make_float4(0.f, 0.f, 0.f, 0.f);
+    a1 = a0;
     const int n = sh->n_seg;
-    for (int s = 0; s < n; ++s) {
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(p.b.part + sh->seg_off[s] +
-                                                               ((long long)plane * R + r) * BM + lane * 4));
-      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    const float* base = p.b.part + ((long long)plane * R) * BM + lane * 4;
+    for (int s0 = 0; s0 < n; s0 += 4) {
+      float4 v[4], w[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        w[k] = v[k];
+        if (s0 + k < n) {
+          const float* q = base + sh->seg_off[s0 + k];
+          v[k] = __ldcg(reinterpret_cast<const float4*>(q + (long long)r0 * BM));
+          if (two) w[k] = __ldcg(reinterpret_cast<const float4*>(q + (long long)r1 * BM));
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        a0.x += v[k].x; a0.y += v[k].y; a0.z += v[k].z; a0.w += v[k].w;
+        a1.x += w[k].x; a1.y += w[k].y; a1.z += w[k].z; a1.w += w[k].w;
+      }
     }
-    return a;
   }
-  __device__ __forceinline__ float sum1(int r, int R, int f) const {
-    float a = 0.f;
+  __device__ __forceinline__ void sum1x2(int r, int R, int f0, int f1, float& a, float& b) const {
+    a = 0.f;
+    b = 0.f;
     const int n = sh->n_seg;
-    for (int s = 0; s < n; ++s) a += __ldcg(p.b.part + sh->seg_off[s] + (long long)r * BM + f);
-    return a;
+    for (int s0 = 0; s0 < n; s0 += 4) {
+      float v[4], w[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        v[k] = 0.f;
+        w[k] = 0.f;
+        if (s0 + k < n) {
+          const float* q = p.b.part + sh->seg_off[s0 + k] + (long long)r * BM;
+          v[k] = __ldcg(q + f0);
+          w[k] = __ldcg(q + f1);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) { a += v[k]; b += w[k]; }
+    }
   }
 
-  // ---- finishing a tile of each product kind (all 256 workers; seg list already in shared)
+  // ---- finishing a tile of each product kind (all 256 workers; seg list already in shared).
+  // Rows are taken two at a time per warp so that all loads of both rows are in flight together.
+  __device__ __forceinline__ static uint2 pack4(float a, float b, float c2, float d2) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c2, d2);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t*>(&lo);
+    u.y = *reinterpret_cast<uint32_t*>(&hi);
+    return u;
+  }
+
   __device__ void finish_qkv(const Job& J, const GemmDesc& g, int tile) {
     const Cfg& c = p.c;
     int mat = 0, trow = tile;
@@ -547,20 +656,21 @@ struct Worker {
     const float qscale = rsqrtf((float)c.hd) * 1.4426950408889634f;
     for (int r = wtid >> 6; r < J.R; r += 4) {
       const float rs = sh->rs_a[r];
-      float a = rs * sum1(r, J.R, f0), b = rs * sum1(r, J.R, f1);
-      if (mat < 2) {
-        const float2 cs = p.b.rope[(long long)(r % J.T) * half + i];
-        const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
-        a = ra; b = rb;
-      }
+      float2 cs = make_float2(1.f, 0.f);
+      if (mat < 2) cs = p.b.rope[(long long)(r % J.T) * half + i];
+      float a, b;
+      sum1x2(r, J.R, f0, f1, a, b);
+      a *= rs;
+      b *= rs;
+      const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
       if (mat == 0) {
         float* qr = p.b.q + (long long)r * c.qd + head * c.hd;
-        qr[i] = a * qscale;
-        qr[i + half] = b * qscale;
+        qr[i] = ra * qscale;
+        qr[i + half] = rb * qscale;
       } else {
         bf16* dst = (mat == 1 ? J.ok : J.ov) + (J.own_base + r) * (long long)c.kvd + head * c.hd;
-        dst[i] = __float2bfloat16_rn(a);
-        dst[i + half] = __float2bfloat16_rn(b);
+        dst[i] = __float2bfloat16_rn(ra);
+        dst[i + half] = __float2bfloat16_rn(rb);
       }
     }
   }
@@ -568,41 +678,59 @@ struct Worker {
   __device__ void finish_o(const Job& J, int tile) {
     const Cfg& c = p.c;
     const int col = tile * BM + lane * 4;
-    for (int r = ww; r < J.R; r += 8) {
-      float ssq = 0.f;
-      if (col < c.d) {
-        const float4 s = sum4(0, r, J.R);
-        const float4 x = *reinterpret_cast<const float4*>(J.x_in + r * J.ldx + col);
-        const float4 w = *reinterpret_cast<const float4*>(J.norm_mlp + col);
-        const float4 y = make_float4(x.x + s.x, x.y + s.y, x.z + s.z, x.w + s.w);
-        *reinterpret_cast<float4*>(p.b.x1 + (long long)r * c.d + col) = y;
-        ssq = y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
-        __nv_bfloat162 a = __floats2bfloat162_rn(y.x * w.x, y.y * w.y);
-        __nv_bfloat162 b = __floats2bfloat162_rn(y.z * w.z, y.w * w.w);
-        uint2 u;
-        u.x = *reinterpret_cast<uint32_t*>(&a);
-        u.y = *reinterpret_cast<uint32_t*>(&b);
-        *reinterpret_cast<uint2*>(p.b.xn_m + (long long)r * c.d + col) = u;
+    const bool cv = col < c.d;
+    float4 w = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (cv) w = *reinterpret_cast<const float4*>(J.norm_mlp + col);
+    for (int r0 = ww; r0 < J.R; r0 += 16) {
+      const int r1 = r0 + 8;
+      const bool two = r1 < J.R;
+      float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), x1v = x0, s0, s1;
+      if (cv) {
+        x0 = *reinterpret_cast<const float4*>(J.x_in + r0 * J.ldx + col);
+        if (two) x1v = *reinterpret_cast<const float4*>(J.x_in + r1 * J.ldx + col);
       }
-      ssq = warp_sum(ssq);
-      if (lane == 0) p.b.ss_m[(long long)tile * c.Rcap + r] = ssq;
+      sum4x2(0, r0, r1, two, J.R, s0, s1);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (h == 1 && !two) break;
+        const int r = h ? r1 : r0;
+        const float4 x = h ? x1v : x0, sv = h ? s1 : s0;
+        const float4 y = make_float4(x.x + sv.x, x.y + sv.y, x.z + sv.z, x.w + sv.w);
+        float ssq = 0.f;
+        if (cv) {
+          *reinterpret_cast<float4*>(p.b.x1 + (long long)r * c.d + col) = y;
+          ssq = y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+          *reinterpret_cast<uint2*>(p.b.xn_m + (long long)r * c.d + col) = pack4(y.x * w.x, y.y * w.y, y.z * w.z, y.w * w.w);
+        }
+        ssq = warp_sum(ssq);
+        if (lane == 0) p.b.ss_m[(long long)tile * c.Rcap + r] = ssq;
+      }
     }
+    fence_proxy_async();
   }
 
   __device__ void finish_gu(const Job& J, int tile) {
     const Cfg& c = p.c;
     const int col = tile * BM + lane * 4;
     if (col >= c.dffn) return;
-    for (int r = ww; r < J.R; r += 8) {
-      const float rs = sh->rs_m[r];
-      const float4 gg = sum4(0, r, J.R), uu = sum4(1, r, J.R);
-      __nv_bfloat162 a = __floats2bfloat162_rn(silu_f(rs * gg.x) * (rs * uu.x), silu_f(rs * gg.y) * (rs * uu.y));
-      __nv_bfloat162 b = __floats2bfloat162_rn(silu_f(rs * gg.z) * (rs * uu.z), silu_f(rs * gg.w) * (rs * uu.w));
-      uint2 u;
-      u.x = *reinterpret_cast<uint32_t*>(&a);
-      u.y = *reinterpret_cast<uint32_t*>(&b);
-      *reinterpret_cast<uint2*>(p.b.act + (long long)r * c.dffn + col) = u;
+    for (int r0 = ww; r0 < J.R; r0 += 16) {
+      const int r1 = r0 + 8;
+      const bool two = r1 < J.R;
+      float4 g0, g1, u0, u1;
+      sum4x2(0, r0, r1, two, J.R, g0, g1);
+      sum4x2(1, r0, r1, two, J.R, u0, u1);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (h == 1 && !two) break;
+        const int r = h ? r1 : r0;
+        const float rs = sh->rs_m[r];
+        const float4 gg = h ? g1 : g0, uu = h ? u1 : u0;
+        *reinterpret_cast<uint2*>(p.b.act + (long long)r * c.dffn + col) =
+            pack4(silu_f(rs * gg.x) * (rs * uu.x), silu_f(rs * gg.y) * (rs * uu.y), silu_f(rs * gg.z) * (rs * uu.z),
+                  silu_f(rs * gg.w) * (rs * uu.w));
+      }
     }
+    fence_proxy_async();
   }
 
   // skip candidate of state j (1-based) at row t: g[i-1][j-1]
@@ -610,22 +738,19 @@ struct Worker {
     return j == 1 ? J.x_im1 + t * J.x_tok_stride : J.g_prev + ((long long)(j - 1) * J.T + t) * p.c.d;
   }
 
-  // partial dot products of Eq. 2 over the 128 columns of `tile`: rows of the candidate
-  // states (apply and skip candidates) and, when `diag`, the rows of the diagonal state
-  __device__ void cos_partials(const Job& J, int tile, bool have_apply, int r, const float4& y) {
+  // partial dot products of Eq. 2 over the 128 columns of `tile` for row r: apply candidate y
+  // (when have_apply) and skip candidate s against x_i
+  __device__ __forceinline__ void cos_partials(int tile, int r, bool cv, bool have_apply, const float4& x,
+                                               const float4& sk, const float4& y) {
     const Cfg& c = p.c;
-    const int col = tile * BM + lane * 4;
-    const int t = r % J.T, j = r / J.T + 1;
     float v[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-    if (col < c.d) {
-      const float4 x = *reinterpret_cast<const float4*>(J.x_i + t * J.x_tok_stride + col);
-      const float4 s = *reinterpret_cast<const float4*>(skip_src(J, j, t) + col);
+    if (cv) {
       if (have_apply) {
         v[0] = x.x * y.x + x.y * y.y + x.z * y.z + x.w * y.w;
         v[1] = y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
       }
-      v[2] = x.x * s.x + x.y * s.y + x.z * s.z + x.w * s.w;
-      v[3] = s.x * s.x + s.y * s.y + s.z * s.z + s.w * s.w;
+      v[2] = x.x * sk.x + x.y * sk.y + x.z * sk.z + x.w * sk.w;
+      v[3] = sk.x * sk.x + sk.y * sk.y + sk.z * sk.z + sk.w * sk.w;
       v[4] = x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
     }
 #pragma unroll
@@ -640,65 +765,92 @@ struct Worker {
   __device__ void finish_down(const Job& J, int tile) {
     const Cfg& c = p.c;
     const int col = tile * BM + lane * 4;
+    const bool cv = col < c.d;
     const int rows = J.R + ((J.dp && J.diag) ? J.T : 0);
-    for (int r = ww; r < rows; r += 8) {
-      float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
-      float ssq = 0.f;
-      if (r < J.R && col < c.d) {
-        const float4 s = sum4(0, r, J.R);
-        const float4 x = *reinterpret_cast<const float4*>(p.b.x1 + (long long)r * c.d + col);
-        y = make_float4(x.x + s.x, x.y + s.y, x.z + s.z, x.w + s.w);
+    const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 w = z4;
+    if (cv && !J.dp && J.norm_next) w = *reinterpret_cast<const float4*>(J.norm_next + col);
+    for (int r0 = ww; r0 < rows; r0 += 16) {
+      const int r1 = r0 + 8;
+      const bool two = r1 < rows;
+      float4 xa[2] = {z4, z4}, xi[2] = {z4, z4}, sk[2] = {z4, z4}, sv[2];
+      // residual, objective and skip-candidate rows first, then the partial tiles
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int r = h ? r1 : r0;
+        if ((h == 1 && !two) || !cv) continue;
+        if (r < J.R) xa[h] = *reinterpret_cast<const float4*>(p.b.x1 + (long long)r * c.d + col);
         if (J.dp) {
-          *reinterpret_cast<float4*>(p.b.Gbuf + (long long)r * c.d + col) = y;
+          const int t = r % J.T, j = r / J.T + 1;
+          xi[h] = *reinterpret_cast<const float4*>(J.x_i + t * J.x_tok_stride + col);
+          sk[h] = *reinterpret_cast<const float4*>(skip_src(J, j, t) + col);
+        }
+      }
+      sum4x2(0, r0 < J.R ? r0 : 0, r1 < J.R ? r1 : 0, two, J.R, sv[0], sv[1]);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (h == 1 && !two) break;
+        const int r = h ? r1 : r0;
+        const bool real = r < J.R;
+        const float4 y = make_float4(xa[h].x + sv[h].x, xa[h].y + sv[h].y, xa[h].z + sv[h].z, xa[h].w + sv[h].w);
+        if (J.dp) {
+          if (real && cv) *reinterpret_cast<float4*>(p.b.Gbuf + (long long)r * c.d + col) = y;
+          cos_partials(tile, r, cv, real, xi[h], sk[h], y);
         } else {
-          *reinterpret_cast<float4*>(J.x_out + r * J.ldo + col) = y;
+          float ssq = 0.f;
+          if (cv) {
+            *reinterpret_cast<float4*>(J.x_out + r * J.ldo + col) = y;
+            if (J.norm_next) {
+              ssq = y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+              *reinterpret_cast<uint2*>(p.b.xn_a + (long long)r * c.d + col) =
+                  pack4(y.x * w.x, y.y * w.y, y.z * w.z, y.w * w.w);
+            }
+          }
           if (J.norm_next) {
-            const float4 w = *reinterpret_cast<const float4*>(J.norm_next + col);
-            ssq = y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
-            __nv_bfloat162 a = __floats2bfloat162_rn(y.x * w.x, y.y * w.y);
-            __nv_bfloat162 b = __floats2bfloat162_rn(y.z * w.z, y.w * w.w);
-            uint2 u;
-            u.x = *reinterpret_cast<uint32_t*>(&a);
-            u.y = *reinterpret_cast<uint32_t*>(&b);
-            *reinterpret_cast<uint2*>(p.b.xn_a + (long long)r * c.d + col) = u;
+            ssq = warp_sum(ssq);
+            if (lane == 0) p.b.ss_a[(long long)tile * c.Rcap + r] = ssq;
           }
         }
       }
-      if (J.dp) {
-        cos_partials(J, tile, r < J.R, r, y);
-      } else if (J.norm_next) {
-        ssq = warp_sum(ssq);
-        if (lane == 0) p.b.ss_a[(long long)tile * c.Rcap + r] = ssq;
-      }
     }
+    fence_proxy_async();
   }
 
   // logits of one vocabulary tile: greedy token (lowest index on ties) and sum of exp
   __device__ void finish_head(const Job& J, int tile) {
     const Cfg& c = p.c;
     const int col = tile * BM + lane * 4;
-    for (int r = ww; r < J.R; r += 8) {
-      const float rs = sh->rs_a[r];
-      const float4 s = sum4(0, r, J.R);
-      float v[4] = {rs * s.x, rs * s.y, rs * s.z, rs * s.w};
-      float best = -INFINITY;
-      int bi = 0x7fffffff;
+    for (int r0 = ww; r0 < J.R; r0 += 16) {
+      const int r1 = r0 + 8;
+      const bool two = r1 < J.R;
+      float4 s0, s1;
+      sum4x2(0, r0, r1, two, J.R, s0, s1);
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (col + k < c.vocab && v[k] > best) { best = v[k]; bi = col + k; }
+      for (int h = 0; h < 2; ++h) {
+        if (h == 1 && !two) break;
+        const int r = h ? r1 : r0;
+        const float4 sv = h ? s1 : s0;
+        const float rs = sh->rs_a[r];
+        float v[4] = {rs * sv.x, rs * sv.y, rs * sv.z, rs * sv.w};
+        float best = -INFINITY;
+        int bi = 0x7fffffff;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, best, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+        for (int k = 0; k < 4; ++k)
+          if (col + k < c.vocab && v[k] > best) { best = v[k]; bi = col + k; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+          if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+        }
+        float se = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (col + k < c.vocab) se += __expf(v[k] - best);
+        se = warp_sum(se);
+        if (lane == 0)
+          p.b.tile_best[(long long)tile * MAX_ROWS + r] = make_float4(best, __int_as_float(bi), se, 0.f);
       }
-      float se = 0.f;
-#pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (col + k < c.vocab) se += __expf(v[k] - best);
-      se = warp_sum(se);
-      if (lane == 0)
-        p.b.tile_best[(long long)tile * MAX_ROWS + r] = make_float4(best, __int_as_float(bi), se, 0.f);
     }
   }
 
@@ -706,18 +858,18 @@ struct Worker {
   __device__ bool gemm_epilogue(const Job& J, int kind) {
     const Cfg& c = p.c;
     const GemmDesc g = make_desc(c, kind, J.layer);
-    long long lo, hi;
-    sk_range(g, c.G, blockIdx.x, lo, hi);
-    const int segmax = sk_max_segs(g.tiles, g.kc, c.G);
+    int lo, hi;
+    sk_range(p, g, blockIdx.x, lo, hi);
+    const int segmax = c.segmax[kind];
     const int planes = g.dual + 1;
     const long long stride = (long long)planes * J.R * BM;
     const int quarter = ww & 3, group = ww >> 2;
     const int ncb = (J.R + 15) >> 4;
-    long long q = lo;
+    int q = lo;
     while (q < hi) {
-      const int tile = (int)(q / g.kc);
-      const long long seg_end = min(hi, (long long)(tile + 1) * g.kc);
-      const int seg = tile - (int)(lo / g.kc);
+      const int tile = q / g.kc;
+      const int seg_end = min(hi, (tile + 1) * g.kc);
+      const int seg = tile - lo / g.kc;
       const uint32_t buf = n_acc & 1u;
       bool ok = wait_bar(&sh->acc_full[buf], (n_acc >> 1) & 1u, p.ctl, sh);
       ok = worker_and(ok);
@@ -735,21 +887,19 @@ struct Worker {
           if (cb * 16 + k < J.R) __stcg(dst + k * BM, v[k]);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __threadfence();
       worker_sync();
       if (wtid == 0) {
         mbar_arrive(tc::smem_u32(&sh->acc_empty[buf]));
-        const int nseg = count_segments(g, tile, c.G);
+        const int nseg = count_segments(g, tile);
+        __threadfence();  // the workers' partial tiles (ordered by the CTA barrier) before the count
         const int prev = atomicAdd(&p.b.counters[g.cnt_base + tile], 1);
         const int last = ((prev + 1) % nseg) == 0;
-        if (last) {
-          __threadfence();
-          list_segments(g, tile, J.R);
-        }
+        if (last) __threadfence();
         sh->flag = last;
       }
       worker_sync();
       if (sh->flag) {
+        list_segments(g, tile, J.R);
         if (kind == G_QKV) finish_qkv(J, g, tile);
         else if (kind == G_O) finish_o(J, tile);
         else if (kind == G_GU) finish_gu(J, tile);
@@ -943,29 +1093,93 @@ struct Worker {
     }
   }
 
-  // chunks of one (row, head) merged in index order; one warp per pair
-  __device__ void attention_merge(const Job& J) {
+  // chunks of one (row, head) merged; one warp per pair.  The chunk weights come from one
+  // load per lane, the accumulators are fetched eight chunks at a time.
+  template <int DPL>
+  __device__ void attention_merge_t(const Job& J) {
     const Cfg& c = p.c;
     const int k_tot = J.uniform ? J.C + J.T : J.C;
     const int n_runs = (k_tot + c.run_len - 1) / c.run_len;
     const int n_chunks = n_runs + (J.uniform ? 0 : (J.R + ATT_KEYS - 1) / ATT_KEYS);
     const int n_pairs = J.R * c.nq;
-    const int dpl = c.hd / 32;
     for (int pr = blockIdx.x * 8 + ww; pr < n_pairs; pr += c.G * 8) {
       const float2* ml = p.b.att_ml + (long long)pr * c.chunk_cap;
-      float mx = -INFINITY;
-      for (int ch = 0; ch < n_chunks; ++ch) mx = fmaxf(mx, __ldcg(ml + ch).x);
-      float num[4] = {0.f, 0.f, 0.f, 0.f}, den = 0.f;
-      for (int ch = 0; ch < n_chunks; ++ch) {
-        const float2 v = __ldcg(ml + ch);
-        if (v.x == -INFINITY) continue;
-        const float w = exp2f(v.x - mx);
-        den = fmaf(w, v.y, den);
-        const float* a = p.b.att_acc + ((long long)pr * c.chunk_cap + ch) * c.hd + lane * dpl;
-        for (int k = 0; k < dpl; ++k) num[k] = fmaf(w, __ldcg(a + k), num[k]);
+      float2 v0 = make_float2(-INFINITY, 0.f), v1 = v0;
+      if (lane < n_chunks) v0 = __ldcg(ml + lane);
+      if (lane + 32 < n_chunks) v1 = __ldcg(ml + lane + 32);
+      const float mx = warp_max(fmaxf(v0.x, v1.x));
+      const float w0 = v0.x == -INFINITY ? 0.f : exp2f(v0.x - mx);
+      const float w1 = v1.x == -INFINITY ? 0.f : exp2f(v1.x - mx);
+      const float den = warp_sum(w0 * v0.y + w1 * v1.y);
+      float num[DPL];
+#pragma unroll
+      for (int k = 0; k < DPL; ++k) num[k] = 0.f;
+      const float* acc = p.b.att_acc + (long long)pr * c.chunk_cap * c.hd + lane * DPL;
+      for (int ch0 = 0; ch0 < n_chunks; ch0 += 8) {
+        float a[8][DPL];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+#pragma unroll
+          for (int k = 0; k < DPL; ++k) a[e][k] = 0.f;
+          if (ch0 + e < n_chunks) {
+            if (DPL == 4) {
+              const float4 t = __ldcg(reinterpret_cast<const float4*>(acc + (long long)(ch0 + e) * c.hd));
+              a[e][0] = t.x; a[e][1] = t.y; a[e][2] = t.z; a[e][3] = t.w;
+            } else {
+              const float2 t = __ldcg(reinterpret_cast<const float2*>(acc + (long long)(ch0 + e) * c.hd));
+              a[e][0] = t.x; a[e][1] = t.y;
+            }
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int ch = ch0 + e;
+          const float wa = __shfl_sync(0xffffffffu, w0, ch & 31), wb = __shfl_sync(0xffffffffu, w1, ch & 31);
+          const float w = ch < 32 ? wa : wb;
+#pragma unroll
+          for (int k = 0; k < DPL; ++k) num[k] = fmaf(w, a[e][k], num[k]);
+        }
       }
-      bf16* dst = p.b.attn + (long long)pr * c.hd + lane * dpl;
-      for (int k = 0; k < dpl; ++k) dst[k] = __float2bfloat16_rn(num[k] / den);
+      bf16* dst = p.b.attn + (long long)pr * c.hd + lane * DPL;
+      const float inv = 1.0f / den;
+      if (DPL == 4) {
+        *reinterpret_cast<uint2*>(dst) = pack4(num[0] * inv, num[1] * inv, num[2] * inv, num[DPL - 1] * inv);
+      } else {
+        __nv_bfloat162 t = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
+        *reinterpret_cast<__nv_bfloat162*>(dst) = t;
+      }
+    }
+    fence_proxy_async();
+  }
+  __device__ void attention_merge(const Job& J) {
+    if (p.c.hd == 128) attention_merge_t<4>(J);
+    else attention_merge_t<2>(J);
+  }
+
+  // L2 prefetch of the cache lines this CTA's attention items will read (issued when the
+  // job starts, long before the queries exist)
+  __device__ void attention_prefetch(const Job& J) {
+    const Cfg& c = p.c;
+    const int Gq = c.nq / c.nkv;
+    const int n_pbg = (J.R * Gq + 127) / 128;
+    const int k_tot = J.uniform ? J.C : J.C;  // keys already in the cache
+    const int n_runs_all = ((J.uniform ? J.C + J.T : J.C) + c.run_len - 1) / c.run_len;
+    const int n_own = J.uniform ? 0 : (J.R + ATT_KEYS - 1) / ATT_KEYS;
+    const int n_chunks = n_runs_all + n_own;
+    const int n_items = c.nkv * n_chunks * n_pbg;
+    const int lpr = (c.hd * 2 + 127) / 128;  // 128-byte lines per key row of one head
+    for (int it = blockIdx.x; it < n_items; it += c.G) {
+      const int chunk = (it / n_pbg) % n_chunks;
+      const int kvh = it / (n_pbg * n_chunks);
+      if (chunk >= n_runs_all) continue;
+      const int key_lo = chunk * c.run_len, key_hi = min(k_tot, key_lo + c.run_len);
+      const int n_lines = (key_hi - key_lo) * lpr * 2;
+      for (int v = wtid; v < n_lines; v += WORKERS) {
+        const int which = v & 1, ln = (v >> 1) % lpr, key = key_lo + (v >> 1) / lpr;
+        const bf16* base = which ? J.cv : J.ck;
+        const bf16* addr = base + (long long)key * c.kvd + kvh * c.hd + ln * 64;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(addr));
+      }
     }
   }
 
@@ -974,11 +1188,22 @@ struct Worker {
     const Cfg& c = p.c;
     const int rows = J.ell * J.T + (J.diag ? J.T : 0);
     const long long rstride = (long long)(c.Rcap + MAX_ROWS) * 5;
-    for (int idx = wtid; idx < rows * 5; idx += WORKERS) {
-      const int r = idx / 5, k = idx % 5;
-      double s = 0.0;
-      for (int t = 0; t < c.n_dt; ++t) s += (double)__ldcg(p.b.cosp + t * rstride + (long long)r * 5 + k);
-      sh->cosv[r][k] = s;
+    // one warp per row: lanes take column tiles, then a fixed shuffle tree adds them up
+    for (int r = ww; r < rows; r += 8) {
+      double v[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
+      for (int t = lane; t < c.n_dt; t += 32) {
+        const float* src = p.b.cosp + t * rstride + (long long)r * 5;
+        float f[5];
+#pragma unroll
+        for (int k = 0; k < 5; ++k) f[k] = __ldcg(src + k);
+#pragma unroll
+        for (int k = 0; k < 5; ++k) v[k] += (double)f[k];
+      }
+#pragma unroll
+      for (int k = 0; k < 5; ++k) {
+        v[k] = warp_sum_d(v[k]);
+        if (lane == 0) sh->cosv[r][k] = v[k];
+      }
     }
     worker_sync();
     const int n_states = J.ell + (J.diag ? 1 : 0);
@@ -1009,34 +1234,30 @@ struct Worker {
       J.choice[0] = 0;
     }
     worker_sync();
-    // write-back of g[i][1..n_states] and the next step's operand, one column tile per CTA
-    for (int tile = blockIdx.x; tile < c.n_dt; tile += c.G) {
+    // write-back of g[i][1..n_states] and the next step's operand: one (column tile, row) per warp
+    const int n_units = c.n_dt * n_states * J.T;
+    for (int u = blockIdx.x * 8 + ww; u < n_units; u += c.G * 8) {
+      const int tile = u % c.n_dt, r = u / c.n_dt;
       const int col = tile * BM + lane * 4;
-      for (int r = ww; r < n_states * J.T; r += 8) {
-        const int j = r / J.T + 1, t = r % J.T;
-        float ssq = 0.f;
-        if (col < c.d) {
-          const float* src = sh->choice[j] ? p.b.Gbuf + (long long)r * c.d : skip_src(J, j, t);
-          const float4 y = *reinterpret_cast<const float4*>(src + col);
-          *reinterpret_cast<float4*>(J.g_next + ((long long)j * J.T + t) * c.d + col) = y;
-          if (J.g_final && j == J.M) *reinterpret_cast<float4*>(J.g_final + (long long)t * c.d + col) = y;
-          if (J.norm_next) {
-            const float4 w = *reinterpret_cast<const float4*>(J.norm_next + col);
-            ssq = y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
-            __nv_bfloat162 a = __floats2bfloat162_rn(y.x * w.x, y.y * w.y);
-            __nv_bfloat162 b = __floats2bfloat162_rn(y.z * w.z, y.w * w.w);
-            uint2 u;
-            u.x = *reinterpret_cast<uint32_t*>(&a);
-            u.y = *reinterpret_cast<uint32_t*>(&b);
-            *reinterpret_cast<uint2*>(p.b.xn_a + (long long)r * c.d + col) = u;
-          }
-        }
+      const int j = r / J.T + 1, t = r % J.T;
+      float ssq = 0.f;
+      if (col < c.d) {
+        const float* src = sh->choice[j] ? p.b.Gbuf + (long long)r * c.d : skip_src(J, j, t);
+        const float4 y = __ldcg(reinterpret_cast<const float4*>(src + col));
+        *reinterpret_cast<float4*>(J.g_next + ((long long)j * J.T + t) * c.d + col) = y;
+        if (J.g_final && j == J.M) *reinterpret_cast<float4*>(J.g_final + (long long)t * c.d + col) = y;
         if (J.norm_next) {
-          ssq = warp_sum(ssq);
-          if (lane == 0) p.b.ss_a[(long long)tile * c.Rcap + r] = ssq;
+          const float4 w = *reinterpret_cast<const float4*>(J.norm_next + col);
+          ssq = y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+          *reinterpret_cast<uint2*>(p.b.xn_a + (long long)r * c.d + col) = pack4(y.x * w.x, y.y * w.y, y.z * w.z, y.w * w.w);
         }
       }
+      if (J.norm_next) {
+        ssq = warp_sum(ssq);
+        if (lane == 0) p.b.ss_a[(long long)tile * c.Rcap + r] = ssq;
+      }
     }
+    fence_proxy_async();
   }
 
   // greedy token of each head row from the per-tile results (CTA 0, one warp per row)
@@ -1078,8 +1299,18 @@ struct Worker {
       const Job& J = p.jobs[jb];
       if (J.type == JOB_SELECT) {
         // step with no candidate that goes through a layer (i = 1): only the diagonal state
-        for (int tile = blockIdx.x; tile < c.n_dt; tile += c.G)
-          for (int r = ww; r < J.T; r += 8) cos_partials(J, tile, false, r, make_float4(0.f, 0.f, 0.f, 0.f));
+        for (int tile = blockIdx.x; tile < c.n_dt; tile += c.G) {
+          const int col = tile * BM + lane * 4;
+          const bool cv = col < c.d;
+          for (int r = ww; r < J.T; r += 8) {
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f), sk = x;
+            if (cv) {
+              x = *reinterpret_cast<const float4*>(J.x_i + r * J.x_tok_stride + col);
+              sk = *reinterpret_cast<const float4*>(skip_src(J, 1, r) + col);
+            }
+            cos_partials(tile, r, cv, false, x, sk, x);
+          }
+        }
         if (!barrier()) return false;
         dp_select(J);
         if (!barrier()) return false;
@@ -1094,6 +1325,7 @@ struct Worker {
         if (!barrier()) return false;
         continue;
       }
+      attention_prefetch(J);
       if (J.prep) {
         prep(J);
         if (!barrier()) return false;
@@ -1174,7 +1406,7 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
   } else if (warp == 2) {
     if (lane == 0) mma_issuer(p, &sh, ring_base, tmem_base);
   } else if (warp >= 4) {
-    Worker w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0u, 0u};
+    Worker w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0u, 0u, 0};
     w.run();
   }
 

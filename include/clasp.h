@@ -246,12 +246,14 @@ int clasp_gemm_xwT_noalloc(const void* x, const void* w, int32_t R, int32_t N, i
  * since the last call (the word is then cleared), or CLASP_ERR_CUDA. */
 int clasp_last_device_status(clasp_ctx* ctx);
 
-/* Per-launch timing of the weight-streaming GEMM (measurement aid; no counterpart in
- * the paper).  enable != 0 starts bracketing every tensor-core GEMM launch with a pair
- * of CUDA events on the context's stream.  enable == 0 synchronises the stream, stops,
- * and reports through the non-NULL HOST pointers the number of launches bracketed, the
- * sum of their durations in milliseconds and the weight bytes they streamed (N*K*2 per
- * matrix).  Returns CLASP_ERR_CUDA if an event call fails. */
+/* Per-launch timing of the weight-streaming kernels (measurement aid; no counterpart in
+ * the paper).  enable != 0 starts bracketing every launch of the persistent layer kernel
+ * (one launch = one search / verify / draft call) and of the stand-alone tensor-core GEMM
+ * with a pair of CUDA events on the context's stream.  enable == 0 synchronises the
+ * stream, stops, and reports through the non-NULL HOST pointers the number of launches
+ * bracketed, the sum of their durations in milliseconds and the bytes those launches had
+ * to move (every weight matrix once, N*K*2 bytes, plus the visible K/V of each layer
+ * pass).  Returns CLASP_ERR_CUDA if an event call fails. */
 int clasp_profile_gemm(clasp_ctx* ctx, int32_t enable, int64_t* n_launches, double* total_ms,
                        double* weight_bytes);
 

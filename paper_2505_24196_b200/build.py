@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libclasp.so")
 SOURCES = [os.path.join(CSRC, "clasp_api.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("kernels.cuh", "gemm_tc.cuh", "engine.cuh")] + [
+DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("kernels.cuh", "gemm_tc.cuh", "engine2.cuh")] + [
     os.path.join(os.path.dirname(HERE), "include", "clasp.h")]
 
 

@@ -18,7 +18,7 @@
 
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
-#include "engine.cuh"
+#include "engine2.cuh"
 
 namespace {
 
@@ -57,19 +57,17 @@ struct Workspace {
   float* partial;
   // persistent layer engine
   void* xn_m;
-  float* e_part;
   float* e_att_acc;
   float2* e_att_ml;
   float* ss_a;
   float* ss_m;
   float* cosp;
-  float4* tile_best;
-  int* e_counters;
+  float4* head_best;
+  int* flags;
   clasp::pk::Ctl* ctl;
   CUtensorMap* wmaps;
   clasp::pk::Job* jobs;
   int* tabs;
-  size_t e_part_bytes;
   int e_chunk_cap;
   int e_run_len;
   int e_rcap;
@@ -89,29 +87,8 @@ bool config_ok(const clasp_config* c) {
   return true;
 }
 
-constexpr int ENGINE_SIZING_CTAS = 148;
-constexpr int ENGINE_MAX_CTAS = 192;
-constexpr size_t ENGINE_TAB_INTS = 5 * (ENGINE_MAX_CTAS + 1) + 2 * (4096 + 5) + 5 * ENGINE_MAX_CTAS;
-
-// Bytes of split-K partial tiles the layer engine needs with a grid of G CTAs: every CTA owns
-// sk_max_segs slots of (planes x rows x 128) floats in each product.
-size_t engine_part_bytes(const clasp_config& c, int G) {
-  namespace pk = clasp::pk;
-  const long long R = c.max_rows < pk::MAX_ROWS ? c.max_rows : pk::MAX_ROWS;
-  const long long Rh = c.max_head_rows < pk::MAX_ROWS ? c.max_head_rows : pk::MAX_ROWS;
-  const long long d = c.d_model, qd = (long long)c.n_q_heads * c.head_dim, kvd = (long long)c.n_kv_heads * c.head_dim;
-  auto tiles = [](long long n) { return (n + pk::BM - 1) / pk::BM; };
-  auto chunks = [](long long k) { return (k + pk::BK - 1) / pk::BK; };
-  auto need = [&](long long t, long long kc, long long planes, long long rows) {
-    return (size_t)G * pk::sk_max_segs(t, kc, G) * planes * rows * pk::BM * 4;
-  };
-  size_t m = need(tiles(qd) + 2 * tiles(kvd), chunks(d), 1, R);
-  size_t v = need(tiles(d), chunks(qd), 1, R); if (v > m) m = v;
-  v = need(tiles(c.d_ffn), chunks(d), 2, R); if (v > m) m = v;
-  v = need(tiles(d), chunks(c.d_ffn), 1, R); if (v > m) m = v;
-  v = need(tiles(c.vocab), chunks(d), 1, Rh); if (v > m) m = v;
-  return m;
-}
+constexpr int ENGINE_MAX_CTAS = clasp::pk::MAX_CTAS;
+constexpr size_t ENGINE_TAB_INTS = 96 * 1024;
 
 // Lays the workspace out; with base == nullptr only the size is computed.
 Workspace carve(const clasp_config& c, uint8_t* base) {
@@ -148,26 +125,24 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
   w.logits = (float*)take((size_t)c.max_head_rows * c.vocab * 4);
   w.partial = (float*)take(PARTIAL_FLOATS * 4);
   if (c.dtype == CLASP_BF16) {
-    // buffers of the persistent layer engine (sized for a grid of ENGINE_SIZING_CTAS)
+    // buffers of the persistent layer engine (per-CTA tables sized for ENGINE_MAX_CTAS)
     namespace pk = clasp::pk;
     const size_t Re = R < (size_t)pk::MAX_ROWS ? R : (size_t)pk::MAX_ROWS;
     const size_t rcap = align_up(Re, 16);
-    const size_t n_dt = (d + pk::BM - 1) / pk::BM;
+    const size_t G = ENGINE_MAX_CTAS;
     w.e_rcap = (int)rcap;
-    w.xn_m = take(rcap * d * 2);
-    w.e_part_bytes = engine_part_bytes(c, ENGINE_SIZING_CTAS);
-    w.e_part = (float*)take(w.e_part_bytes);
+    w.xn_m = take(R * d * 2);
     w.e_run_len = pk::ATT_KEYS * ((c.max_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32));
     w.e_chunk_cap = (c.max_ctx + w.e_run_len - 1) / w.e_run_len + (int)((rcap + pk::ATT_KEYS - 1) / pk::ATT_KEYS);
     w.e_att_acc = (float*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * c.head_dim * 4);
     w.e_att_ml = (float2*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * sizeof(float2));
-    w.ss_a = (float*)take(n_dt * rcap * 4);
-    w.ss_m = (float*)take(n_dt * rcap * 4);
-    w.cosp = (float*)take(n_dt * (rcap + pk::MAX_ROWS) * 5 * 4);
-    w.tile_best = (float4*)take((size_t)((c.vocab + pk::BM - 1) / pk::BM) * pk::MAX_ROWS * sizeof(float4));
-    w.e_counters = (int*)take(MAX_COUNTERS * sizeof(int));
+    w.ss_a = (float*)take(G * rcap * 4);
+    w.ss_m = (float*)take(G * rcap * 4);
+    w.cosp = (float*)take(G * (rcap + pk::MAX_ROWS) * 5 * 4);
+    w.head_best = (float4*)take(G * pk::MAX_ROWS * sizeof(float4));
+    w.flags = (int*)take(pk::N_FLAGS * G * sizeof(int));
     w.ctl = (pk::Ctl*)take(256);
-    w.wmaps = (CUtensorMap*)take(((size_t)c.L * 7 + 1) * sizeof(CUtensorMap));
+    w.wmaps = (CUtensorMap*)take(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS * sizeof(CUtensorMap));
     w.jobs = (pk::Job*)take(((size_t)c.L + 4) * sizeof(pk::Job));
     w.tabs = (int*)take(ENGINE_TAB_INTS * sizeof(int));
   }
@@ -202,9 +177,8 @@ struct clasp_ctx {
   bool use_engine = false;
   int e_G = 0;              // CTAs of the cooperative grid (one per SM)
   int e_static_smem = 0;
-  int e_cnt_base[5] = {0, 0, 0, 0, 0};
-  int e_tab_lo[5], e_tab_seg0[5], e_tab_segc[5], e_segmax[5];
-  int e_pf_max = 0;
+  int e_split_lo[clasp::pk::N_SPLITS], e_split_units[clasp::pk::N_SPLITS], e_tile_idx[5], e_tiles_off = 0,
+      e_loads_off = 0, e_kpi[5];
   std::vector<CUtensorMap> e_wmaps_host;
   bool e_wmaps_dirty = true;
   std::map<int, std::array<CUtensorMap, 4>> e_bmaps;           // by BN
@@ -512,7 +486,7 @@ int embed_rows(clasp_ctx* ctx, const int32_t* tokens, int n, float* out, int64_t
 
 
 // ---------------------------------------------------------------- persistent layer engine
-// Host side of engine.cuh: builds the job list of a call and launches the cooperative
+// Host side of engine2.cuh: builds the job list of a call and launches the cooperative
 // kernel once.  Used by the bf16 tensor-core configuration; the per-kernel sequences
 // above remain for the fp32 model, for CLASP_FLAG_FORCE_SIMT and for shapes the engine
 // does not take (more than 128 rows).
@@ -528,66 +502,105 @@ int engine_setup(clasp_ctx* ctx) {
   CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
   if (!coop) return CLASP_OK;
   const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
-  auto tiles = [](int n) { return (n + pk::BM - 1) / pk::BM; };
-  const int t_qkv = tiles(qd) + 2 * tiles(kvd), t_o = tiles(d), t_gu = tiles(c.d_ffn), t_down = tiles(d);
-  const int t_head = tiles(c.vocab);
-  ctx->e_cnt_base[0] = 0;
-  ctx->e_cnt_base[1] = t_qkv;
-  ctx->e_cnt_base[2] = t_qkv + t_o;
-  ctx->e_cnt_base[3] = t_qkv + t_o + t_gu;
-  ctx->e_cnt_base[4] = t_qkv + t_o + t_gu + t_down;
-  if (ctx->e_cnt_base[4] + t_head > MAX_COUNTERS) return CLASP_OK;
+  if (d % 8 || c.d_ffn % 8 || c.vocab % 8) return CLASP_OK;
   cudaFuncAttributes fa;
   CUDA_TRY(cudaFuncGetAttributes(&fa, pk::engine_kernel));
   ctx->e_static_smem = (int)fa.sharedSizeBytes;
   const int dyn_max = optin - ctx->e_static_smem;
-  if (dyn_max < 1024 + 2 * (pk::A_TILE_BYTES + 128 * 128) + pk::SCRATCH_BYTES) return CLASP_OK;
+  if (dyn_max < 1024 + 64 * pk::PAGE + pk::SCRATCH_BYTES) return CLASP_OK;
   CUDA_TRY(cudaFuncSetAttribute(pk::engine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
   int G = ctx->num_sms;
   if (const char* e = getenv("CLASP_ENGINE_CTAS")) {
     const int v = atoi(e);
     if (v >= 1 && v < G) G = v;
   }
-  if (engine_part_bytes(c, G) > ctx->ws.e_part_bytes || G > ENGINE_MAX_CTAS) return CLASP_OK;
-  // stream-K tables: unit range of every CTA and, per output tile, the CTAs that hold a partial tile
-  {
-    const int kc_d = (d + pk::BK - 1) / pk::BK, kc_q = (qd + pk::BK - 1) / pk::BK, kc_f = (c.d_ffn + pk::BK - 1) / pk::BK;
-    const int n_tiles[5] = {t_qkv, t_o, t_gu, t_down, t_head};
-    const int n_kc[5] = {kc_d, kc_q, kc_d, kc_f, kc_d};
-    std::vector<int> tab;
-    for (int k = 0; k < 5; ++k) {
-      const long long U = (long long)n_tiles[k] * n_kc[k];
-      ctx->e_segmax[k] = pk::sk_max_segs(n_tiles[k], n_kc[k], G);
-      ctx->e_tab_lo[k] = (int)tab.size();
-      std::vector<int> lo(G + 1);
-      for (int cc = 0; cc <= G; ++cc) lo[cc] = (int)(U * cc / G);
-      tab.insert(tab.end(), lo.begin(), lo.end());
-      std::vector<int> seg0(n_tiles[k] + 1, 0), segc;
-      for (int t = 0; t < n_tiles[k]; ++t) {
-        seg0[t] = (int)segc.size();
-        const long long q0 = (long long)t * n_kc[k], q1 = q0 + n_kc[k];
-        for (int cc = 0; cc < G; ++cc)
-          if (lo[cc + 1] > lo[cc] && lo[cc] < q1 && lo[cc + 1] > q0) segc.push_back(cc);
+  if (G > ENGINE_MAX_CTAS) G = ENGINE_MAX_CTAS;
+  // ---- feature splits and per-CTA tile / load lists
+  const int split_n[pk::N_SPLITS] = {qd + 2 * kvd, d, c.d_ffn, c.vocab};
+  const int kind_split[5] = {pk::S_QKV, pk::S_D, pk::S_F, pk::S_D, pk::S_V};
+  std::vector<int> tab;
+  std::vector<std::vector<int>> lo(pk::N_SPLITS);
+  for (int s = 0; s < pk::N_SPLITS; ++s) {
+    const long long units = split_n[s] / 8;
+    if ((units + 1) * G > 0x7fffffffLL) return CLASP_OK;
+    lo[s].resize(G + 1);
+    for (int cc = 0; cc <= G; ++cc) lo[s][cc] = (int)(units * cc / G) * 8;
+    ctx->e_split_lo[s] = (int)tab.size();
+    ctx->e_split_units[s] = (int)units;
+    tab.insert(tab.end(), lo[s].begin(), lo[s].end());
+  }
+  for (int cc = 0; cc < G; ++cc)
+    if (lo[pk::S_D][cc + 1] - lo[pk::S_D][cc] > 128) return CLASP_OK;  // the Eq. 2 step takes one feature per thread
+  std::vector<pk::TileDesc> tiles;
+  std::vector<pk::LoadDesc> loads;
+  std::vector<std::vector<int>> tidx(5, std::vector<int>(G + 1, 0));
+  for (int k = 0; k < 5; ++k) {
+    const int s = kind_split[k];
+    // matrices stacked along the feature axis of this product
+    int mat_n[3] = {split_n[s], 0, 0}, n_mats = 1;
+    if (k == pk::G_QKV) { mat_n[0] = qd; mat_n[1] = kvd; mat_n[2] = kvd; n_mats = 3; }
+    int max_rows = 8;
+    for (int cc = 0; cc < G; ++cc) {
+      tidx[k][cc] = (int)tiles.size();
+      for (int f0 = lo[s][cc]; f0 < lo[s][cc + 1]; f0 += 128) {
+        const int n = std::min(128, lo[s][cc + 1] - f0);
+        pk::TileDesc td{};
+        td.f0 = f0; td.n_rows = (short)n; td.load0 = (int)loads.size();
+        if (n > max_rows) max_rows = n;
+        int f = f0, left = n;
+        while (left > 0) {
+          int m = 0, base = 0;
+          while (m + 1 < n_mats && f >= base + mat_n[m]) { base += mat_n[m]; ++m; }
+          int piece = std::min(left, base + mat_n[m] - f);
+          int y = f - base;
+          for (int hi = pk::N_HEIGHTS - 1; hi >= 0 && piece > 0; --hi) {
+            const int h = 8 << hi;
+            while (piece >= h) {
+              pk::LoadDesc ld{};
+              ld.map_local = (short)(m * pk::N_HEIGHTS + hi); ld.row_off = (short)(f - f0); ld.y0 = y; ld.rows = h;
+              loads.push_back(ld);
+              y += h; f += h; piece -= h; left -= h;
+            }
+          }
+        }
+        td.n_loads = (short)((int)loads.size() - td.load0);
+        if (td.n_loads > pk::MAX_TILE_LOADS) return CLASP_OK;
+        tiles.push_back(td);
       }
-      seg0[n_tiles[k]] = (int)segc.size();
-      ctx->e_tab_seg0[k] = (int)tab.size();
-      tab.insert(tab.end(), seg0.begin(), seg0.end());
-      ctx->e_tab_segc[k] = (int)tab.size();
-      tab.insert(tab.end(), segc.begin(), segc.end());
     }
-    if (tab.size() > ENGINE_TAB_INTS) return CLASP_OK;
-    CUDA_TRY(cudaMemcpyAsync(ctx->ws.tabs, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
-    CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+    tidx[k][G] = (int)tiles.size();
+    const int a_pages = (k == pk::G_GU ? 2 : 1) * (max_rows / 8);
+    int kpi = 16 / a_pages;
+    ctx->e_kpi[k] = kpi < 1 ? 1 : (kpi > 4 ? 4 : kpi);
   }
-  if (const char* e = getenv("CLASP_ENGINE_PF")) {
-    const int v = atoi(e);
-    if (v >= 0 && v <= 256) ctx->e_pf_max = v;
+  for (int k = 0; k < 5; ++k) {
+    ctx->e_tile_idx[k] = (int)tab.size();
+    tab.insert(tab.end(), tidx[k].begin(), tidx[k].end());
   }
+  static_assert(sizeof(pk::TileDesc) == 12 && sizeof(pk::LoadDesc) == 12, "table records are three ints");
+  ctx->e_tiles_off = (int)tab.size();
+  tab.resize(tab.size() + tiles.size() * 3);
+  memcpy(tab.data() + ctx->e_tiles_off, tiles.data(), tiles.size() * sizeof(pk::TileDesc));
+  ctx->e_loads_off = (int)tab.size();
+  tab.resize(tab.size() + loads.size() * 3);
+  memcpy(tab.data() + ctx->e_loads_off, loads.data(), loads.size() * sizeof(pk::LoadDesc));
+  if (tab.size() > ENGINE_TAB_INTS) return CLASP_OK;
+  CUDA_TRY(cudaMemcpyAsync(ctx->ws.tabs, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+  CUDA_TRY(cudaStreamSynchronize(ctx->stream));
   ctx->e_G = G;
-  ctx->e_wmaps_host.assign((size_t)c.L * 7 + 1, CUtensorMap{});
+  ctx->e_wmaps_host.assign(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS, CUtensorMap{});
   ctx->e_wmaps_dirty = true;
   ctx->use_engine = true;
   return CLASP_OK;
+}
+
+// tensor maps of one weight matrix for every box height
+int engine_maps(clasp_ctx* ctx, int slot, const void* w, int rows, int cols) {
+  int rc = 0;
+  for (int hi = 0; hi < pk::N_HEIGHTS; ++hi)
+    rc |= make_map(ctx, w, rows, cols, 8 << hi, &ctx->e_wmaps_host[(size_t)slot * pk::N_HEIGHTS + hi]);
+  ctx->e_wmaps_dirty = true;
+  return rc ? CLASP_ERR_CUDA : CLASP_OK;
 }
 
 // weight + visible K/V bytes one job must move (for the per-launch bandwidth figure)
@@ -596,8 +609,7 @@ double job_bytes(const clasp_ctx* ctx, const pk::Job& J) {
   const double d = c.d_model, qd = (double)c.n_q_heads * c.head_dim, kvd = (double)c.n_kv_heads * c.head_dim;
   if (J.type == pk::JOB_HEAD) return 2.0 * c.vocab * d;
   if (J.type != pk::JOB_LAYER) return 0.0;
-  const double keys = J.uniform ? J.C + J.T : J.C;
-  return 2.0 * (d * (qd + 2 * kvd) + qd * d + 3.0 * d * c.d_ffn) + 2.0 * keys * kvd * 2.0;
+  return 2.0 * (d * (qd + 2 * kvd) + qd * d + 3.0 * d * c.d_ffn) + 2.0 * (double)J.C * kvd * 2.0;
 }
 
 // Launch the engine over ctx->e_jobs.  Rmax: most rows of any job; head_off: first row of the
@@ -613,15 +625,21 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   int dev = 0, optin = 0;
   CUDA_TRY(cudaGetDevice(&dev));
   CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-  const int slot_bytes = pk::A_TILE_BYTES + BN * pk::BK * 2;
-  int n_slots = (optin - ctx->e_static_smem - 1024 - pk::SCRATCH_BYTES) / slot_bytes;
-  if (n_slots > pk::MAX_SLOTS) n_slots = pk::MAX_SLOTS;
-  if (const char* e = getenv("CLASP_ENGINE_SLOTS")) {
+  int ring_pages = (optin - ctx->e_static_smem - 1024 - pk::SCRATCH_BYTES) / pk::PAGE;
+  if (const char* e = getenv("CLASP_ENGINE_PAGES")) {
     const int v = atoi(e);
-    if (v >= 2 && v < n_slots) n_slots = v;
+    if (v >= 64 && v < ring_pages) ring_pages = v;
   }
-  if (n_slots < 2) return CLASP_ERR_CAPACITY;
-  const size_t dyn = 1024 + (size_t)n_slots * slot_bytes + pk::SCRATCH_BYTES;
+  // an item (gate + up rows and the operand tile of kpi chunks) must fit the ring twice over
+  const int b_pages = BN * pk::BK * 2 / pk::PAGE;
+  int kpi[5];
+  for (int k = 0; k < 5; ++k) {
+    kpi[k] = ctx->e_kpi[k];
+    const int chunk_pages = 16 * (k == pk::G_GU ? 2 : 1) + b_pages;
+    while (kpi[k] > 1 && kpi[k] * chunk_pages * 2 > ring_pages) --kpi[k];
+    if (chunk_pages > ring_pages) return CLASP_ERR_CAPACITY;
+  }
+  const size_t dyn = 1024 + (size_t)ring_pages * pk::PAGE + pk::SCRATCH_BYTES;
 
   auto bm = ctx->e_bmaps.find(BN);
   if (bm == ctx->e_bmaps.end()) {
@@ -648,26 +666,22 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   }
   CUDA_TRY(cudaMemcpyAsync(ws.jobs, ctx->e_jobs.data(), ctx->e_jobs.size() * sizeof(pk::Job),
                            cudaMemcpyHostToDevice, ctx->stream));
-  CUDA_TRY(cudaMemsetAsync(ws.ctl, 0, 8, ctx->stream));  // barrier counter and abort flag; status is sticky
-  CUDA_TRY(cudaMemsetAsync(ws.e_counters, 0, MAX_COUNTERS * sizeof(int), ctx->stream));
+  CUDA_TRY(cudaMemsetAsync(ws.ctl, 0, 4, ctx->stream));  // abort flag; the status word is sticky
+  CUDA_TRY(cudaMemsetAsync(ws.flags, 0, (size_t)pk::N_FLAGS * ctx->e_G * sizeof(int), ctx->stream));
 
   pk::Params P{};
   P.c.L = c.L; P.c.d = d; P.c.qd = qd; P.c.kvd = c.n_kv_heads * c.head_dim; P.c.hd = c.head_dim;
   P.c.nq = c.n_q_heads; P.c.nkv = c.n_kv_heads; P.c.dffn = c.d_ffn; P.c.vocab = c.vocab; P.c.eps = c.rms_eps;
-  P.c.G = ctx->e_G; P.c.Rcap = ws.e_rcap; P.c.n_dt = (d + pk::BM - 1) / pk::BM; P.c.run_len = ws.e_run_len;
-  P.c.chunk_cap = ws.e_chunk_cap;
-  for (int k = 0; k < 5; ++k) P.c.cnt_base[k] = ctx->e_cnt_base[k];
-  P.c.BN = BN; P.c.n_slots = n_slots; P.c.slot_bytes = slot_bytes; P.c.pf_max = ctx->e_pf_max;
-  for (int k = 0; k < 5; ++k) {
-    P.c.tab_lo[k] = ctx->e_tab_lo[k]; P.c.tab_seg0[k] = ctx->e_tab_seg0[k]; P.c.tab_segc[k] = ctx->e_tab_segc[k];
-    P.c.segmax[k] = ctx->e_segmax[k];
-  }
-  P.tabs = ws.tabs;
+  P.c.G = ctx->e_G; P.c.Rcap = ws.e_rcap; P.c.run_len = ws.e_run_len; P.c.chunk_cap = ws.e_chunk_cap;
+  P.c.BN = BN; P.c.ring_pages = ring_pages;
+  for (int s = 0; s < pk::N_SPLITS; ++s) { P.c.split_lo[s] = ctx->e_split_lo[s]; P.c.split_units[s] = ctx->e_split_units[s]; }
+  for (int k = 0; k < 5; ++k) { P.c.tile_idx[k] = ctx->e_tile_idx[k]; P.c.kpi[k] = kpi[k]; }
+  P.c.tiles_off = ctx->e_tiles_off; P.c.loads_off = ctx->e_loads_off;
   P.b.xn_a = (bf16*)ws.xn; P.b.xn_m = (bf16*)ws.xn_m; P.b.attn = (bf16*)ws.attn; P.b.act = (bf16*)ws.act;
-  P.b.q = ws.qkv; P.b.x1 = ws.x1; P.b.Gbuf = ws.G; P.b.part = ws.e_part; P.b.att_acc = ws.e_att_acc;
-  P.b.att_ml = ws.e_att_ml; P.b.ss_a = ws.ss_a; P.b.ss_m = ws.ss_m; P.b.cosp = ws.cosp;
-  P.b.tile_best = ws.tile_best; P.b.counters = ws.e_counters; P.b.rope = ws.rope;
-  P.jobs = ws.jobs; P.n_jobs = (int)ctx->e_jobs.size(); P.wmaps = ws.wmaps; P.ctl = ws.ctl;
+  P.b.qkv = ws.qkv; P.b.x1 = ws.x1; P.b.Gbuf = ws.G; P.b.att_acc = ws.e_att_acc; P.b.att_ml = ws.e_att_ml;
+  P.b.ss_a = ws.ss_a; P.b.ss_m = ws.ss_m; P.b.cosp = ws.cosp; P.b.head_best = ws.head_best; P.b.flags = ws.flags;
+  P.b.rope = ws.rope;
+  P.jobs = ws.jobs; P.n_jobs = (int)ctx->e_jobs.size(); P.wmaps = ws.wmaps; P.tabs = ws.tabs; P.ctl = ws.ctl;
   P.trace = ctx->e_trace; P.trace_cap = ctx->e_trace_cap;
 
   cudaEvent_t e0 = nullptr, e1 = nullptr;
@@ -689,17 +703,25 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
 }
 
 // a decoder-layer job with the fields every caller sets the same way
-pk::Job layer_job(clasp_ctx* ctx, int l, int S, int T, int C, bool uniform, const clasp_kv_layer& kv, int64_t pos0) {
-  const clasp_config& c = ctx->cfg;
+pk::Job layer_job(clasp_ctx* ctx, int l, int S, int T, int C, bool uniform, const clasp_kv_layer& kv) {
   pk::Job J{};
   J.type = pk::JOB_LAYER; J.layer = l; J.S = S; J.T = T; J.R = S * T; J.C = C; J.uniform = uniform ? 1 : 0;
   J.norm_in = ctx->layers[l].attn_norm; J.norm_mlp = ctx->layers[l].mlp_norm;
-  J.ck = (const bf16*)kv.k; J.cv = (const bf16*)kv.v;
-  J.ok = uniform ? (bf16*)kv.k : (bf16*)ctx->ws.own_k;
-  J.ov = uniform ? (bf16*)kv.v : (bf16*)ctx->ws.own_v;
-  J.own_base = uniform ? pos0 : 0;
-  (void)c;
+  J.ck = (bf16*)kv.k; J.cv = (bf16*)kv.v;
   return J;
+}
+
+// fills in where each job's first operand comes from (the step of the previous job that wrote it)
+void link_jobs(std::vector<pk::Job>& jobs) {
+  for (size_t k = 0; k < jobs.size(); ++k) {
+    pk::Job& J = jobs[k];
+    if (J.type == pk::JOB_SELECT) continue;
+    if (J.type == pk::JOB_LAYER && J.prep) { J.src_flag = pk::F_PREP; J.src_epoch = (int)k + 1; continue; }
+    const pk::Job& prev = jobs[k - 1];
+    const bool from_select = prev.type == pk::JOB_SELECT || (prev.type == pk::JOB_LAYER && prev.dp);
+    J.src_flag = from_select ? pk::F_SELECT : pk::F_DOWN;
+    J.src_epoch = (int)k;
+  }
 }
 
 }  // namespace
@@ -800,10 +822,16 @@ int clasp_load_layers(clasp_ctx* ctx, int32_t first, int32_t count, const clasp_
       rc |= make_map(ctx, lw.w_down, d, c.d_ffn, clasp::tc::BM, &m.w_down);
       if (rc) return CLASP_ERR_CUDA;
       if (ctx->use_engine) {
-        CUtensorMap* dst = &ctx->e_wmaps_host[(size_t)(first + k) * 7];
-        dst[0] = m.wq; dst[1] = m.wk; dst[2] = m.wv; dst[3] = m.wo; dst[4] = m.w_gate; dst[5] = m.w_up;
-        dst[6] = m.w_down;
-        ctx->e_wmaps_dirty = true;
+        const int b7 = (first + k) * 7;
+        int erc = 0;
+        erc |= engine_maps(ctx, b7 + 0, lw.wq, qd, d);
+        erc |= engine_maps(ctx, b7 + 1, lw.wk, kvd, d);
+        erc |= engine_maps(ctx, b7 + 2, lw.wv, kvd, d);
+        erc |= engine_maps(ctx, b7 + 3, lw.wo, d, qd);
+        erc |= engine_maps(ctx, b7 + 4, lw.w_gate, c.d_ffn, d);
+        erc |= engine_maps(ctx, b7 + 5, lw.w_up, c.d_ffn, d);
+        erc |= engine_maps(ctx, b7 + 6, lw.w_down, d, c.d_ffn);
+        if (erc) return CLASP_ERR_CUDA;
       }
     }
     ctx->loaded[first + k] = 1;
@@ -820,10 +848,8 @@ int clasp_load_head(clasp_ctx* ctx, const void* embed, const float* final_norm, 
   ctx->lm_head = lm_head;
   if (ctx->use_tc && make_map(ctx, lm_head, ctx->cfg.vocab, ctx->cfg.d_model, clasp::tc::BM, &ctx->lm_head_map))
     return CLASP_ERR_CUDA;
-  if (ctx->use_engine) {
-    ctx->e_wmaps_host[(size_t)ctx->cfg.L * 7] = ctx->lm_head_map;
-    ctx->e_wmaps_dirty = true;
-  }
+  if (ctx->use_engine && engine_maps(ctx, ctx->cfg.L * 7, lm_head, ctx->cfg.vocab, ctx->cfg.d_model))
+    return CLASP_ERR_CUDA;
   return CLASP_OK;
 }
 
@@ -840,9 +866,10 @@ int clasp_layer_forward(clasp_ctx* ctx, int32_t layer, const float* x_in, int64_
   int rc = rope_table(ctx, T, pos0);
   if (rc) return rc;
   if (ctx->use_engine && S * T <= pk::MAX_ROWS && (!write_kv || pos0 == ctx_len)) {
-    pk::Job J = layer_job(ctx, layer, S, T, ctx_len, write_kv != 0, *kv_layer, pos0);
+    pk::Job J = layer_job(ctx, layer, S, T, ctx_len, write_kv != 0, *kv_layer);
     J.prep = 1; J.x_in = x_in; J.ldx = in_stride; J.x_out = x_out; J.ldo = out_stride;
     ctx->e_jobs.assign(1, J);
+    link_jobs(ctx->e_jobs);
     return engine_launch(ctx, S * T, 0);
   }
   return run_layer_any(ctx, layer, x_in, in_stride, S, T, ctx_len, pos0, *kv_layer, write_kv != 0, x_out,
@@ -881,7 +908,7 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
       const int ell = (i - 1 < M) ? i - 1 : M;
       pk::Job J{};
       if (ell > 0) {
-        J = layer_job(ctx, i - 1, ell, T, ctx_len, false, kv[i - 1], pos0);
+        J = layer_job(ctx, i - 1, ell, T, ctx_len, false, kv[i - 1]);
         J.x_in = ws.grow[cur] + Td; J.ldx = d; J.dp = 1;
       } else {
         J.type = pk::JOB_SELECT; J.T = T;
@@ -900,6 +927,7 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
       ctx->e_jobs.push_back(J);
       cur ^= 1;
     }
+    link_jobs(ctx->e_jobs);
     if ((rc = engine_launch(ctx, M * T, 0))) return rc;
     clasp::backtrack_kernel<<<1, 32, 0, ctx->stream>>>(ws.choice, L, M, skip_mask);
     return launch_check(ctx);
@@ -969,7 +997,7 @@ int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0,
     float* a = ctx->ws.hping;
     float* b = ctx->ws.hpong;
     for (int l = 0; l < L; ++l) {
-      pk::Job J = layer_job(ctx, l, 1, n, pos0, true, kv[l], pos0);
+      pk::Job J = layer_job(ctx, l, 1, n, pos0, true, kv[l]);
       J.prep = l == 0 ? 1 : 0;
       if (hidden_out) {
         J.x_in = hidden_out + (int64_t)l * d; J.x_out = hidden_out + (int64_t)(l + 1) * d;
@@ -987,6 +1015,7 @@ int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0,
       H.argmax_out = argmax_out;
       ctx->e_jobs.push_back(H);
     }
+    link_jobs(ctx->e_jobs);
     return engine_launch(ctx, n, n_head_rows > 0 ? n - n_head_rows : 0);
   }
   const float* x;
@@ -1036,7 +1065,7 @@ int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int
     for (int l = 0; l < c.L; ++l) {
       if (skip_mask_host[l]) continue;  // skipped layer: nothing read, nothing written
       if (!kv[l].k || !kv[l].v) return CLASP_ERR_INVALID_ARG;
-      pk::Job J = layer_job(ctx, l, 1, 1, pos, true, kv[l], pos);
+      pk::Job J = layer_job(ctx, l, 1, 1, pos, true, kv[l]);
       J.prep = ctx->e_jobs.empty() ? 1 : 0;
       J.x_in = a; J.ldx = d; J.x_out = b; J.ldo = d;
       float* t = a; a = b; b = t;
@@ -1048,6 +1077,7 @@ int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int
     pk::Job H{};
     H.type = pk::JOB_HEAD; H.R = 1; H.T = 1; H.row_off = 0; H.argmax_out = token_out; H.top1_out = top1_prob_out;
     ctx->e_jobs.push_back(H);
+    link_jobs(ctx->e_jobs);
     return engine_launch(ctx, 1, 0);
   }
   for (int l = 0; l < c.L; ++l) {

@@ -1,0 +1,1392 @@
+// Persistent layer engine: one cooperative kernel runs a whole list of jobs (decoder layers,
+// Eq. 2 steps, the LM head), streaming every weight matrix from HBM exactly once and without
+// a gap between consecutive products.
+//
+// Work split of a product y = x W^T: the output features are dealt out to the CTAs in
+// contiguous ranges of 8-feature units and every CTA runs the whole reduction for its range.
+// There is no split-K, so no partial sums are exchanged: the CTA that owns a feature finishes
+// it (residual, norm operand, SwiGLU, cosine partials, arg-max) straight from its accumulator.
+// The split and all reduction orders depend on shapes and grid size only, never on the number
+// of rows or on timing.
+//
+// One CTA per SM, twelve warps:
+//   warp 0      lane 0 issues the TMA loads of weight rows (boxes of 8..128 rows x 64 columns,
+//               128B swizzle) into a ring of 1 KB shared-memory pages.  Weight addresses never
+//               depend on activations: this warp runs ahead across products, layers and jobs.
+//   warp 1      lane 0 loads the activation operand ([BN x 64] bf16 per 64-column chunk) next to
+//               the weight rows once the CTAs that produce those columns have published them.
+//   warp 2      lane 0 issues tcgen05.mma: M = 128 weight rows (rows beyond the CTA's range are
+//               whatever bytes follow in the ring; their accumulator lanes are never read),
+//               N = BN activation rows, K = 16, two accumulators in tensor memory.
+//   warp 3      allocates / frees tensor memory.
+//   warps 4-11  "workers": epilogues, attention, Eq. 2 select, arg-max.
+//
+// Synchronisation between CTAs is by epoch flags in global memory: after finishing step s of
+// job j a CTA stores j+1 to flag[s][cta] (release); a consumer polls the flags of exactly the
+// CTAs whose output it needs (acquire).  RMSNorm is applied as (x * w) W^T * rsqrt(mean(x^2) +
+// eps): the operand is x * w rounded to bf16, the per-row factor multiplies the product later.
+//
+// Every wait (mbarrier, flag) is bounded: when one runs out the CTA raises an abort flag that
+// all other waits observe, drains, frees its tensor memory and returns; the host then reports
+// CLASP_ERR_TIMEOUT.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gemm_tc.cuh"
+#include "kernels.cuh"
+
+namespace clasp {
+namespace pk {
+
+using bf16 = __nv_bfloat16;
+
+constexpr int BK = 64;
+constexpr int PAGE = 1024;            // ring granule: 8 rows x 128 B, one swizzle atom
+constexpr int THREADS = 384;
+constexpr int WORKERS = 256;
+constexpr int WORKER_T0 = 128;
+constexpr int NB = 32;                // items in flight (mbarrier pairs)
+constexpr int ATT_KEYS = 32;
+constexpr int SCRATCH_BYTES = 2 * ATT_KEYS * 136 * 2 + 2048;  // two padded K/V tiles + slack (>= 16 KB guard)
+constexpr int MAX_ROWS = 128;         // rows one launch may push through a layer
+constexpr int N_HEIGHTS = 5;          // TMA box heights 8, 16, 32, 64, 128
+constexpr int MAX_TILE_LOADS = 8;
+constexpr int MAX_CTAS = 192;
+
+enum { JOB_LAYER = 0, JOB_HEAD = 1, JOB_SELECT = 2 };
+enum { G_QKV = 0, G_O = 1, G_GU = 2, G_DOWN = 3, G_HEAD = 4 };
+// feature splits: which CTA owns which output features
+enum { S_QKV = 0, S_D = 1, S_F = 2, S_V = 3, N_SPLITS = 4 };
+// flag kinds
+enum { F_PREP = 0, F_QKV, F_ATTN, F_MERGE, F_O, F_GU, F_DOWN, F_SELECT, F_HEAD, N_FLAGS };
+
+struct TileDesc {      // one accumulator's worth of a CTA's feature range
+  int f0;              // first feature in the product's feature space
+  short n_rows;        // features (multiple of 8, <= 128)
+  short n_loads;
+  int load0;           // first LoadDesc
+};
+struct LoadDesc {
+  short map_local;     // matrix * N_HEIGHTS + height index
+  short row_off;       // destination row inside the tile (multiple of 8)
+  int y0;              // first row in the matrix
+  int rows;            // box height
+};
+
+struct Cfg {
+  int L, d, qd, kvd, hd, nq, nkv, dffn, vocab;
+  float eps;
+  int G;
+  int Rcap;            // row capacity of the per-row tables
+  int run_len, chunk_cap;
+  int BN;              // activation rows padded to a multiple of 16 (MMA N)
+  int ring_pages;
+  // tables (ints / structs in Params::tabs, offsets in ints)
+  int split_lo[N_SPLITS];    // [G + 1] first feature of each CTA: lo(c) = 8 floor(c units / G)
+  int split_units[N_SPLITS]; // 8-feature units of each split
+  int tile_idx[5];           // per product kind: [G + 1] first TileDesc of each CTA
+  int tiles_off;             // TileDesc array
+  int loads_off;             // LoadDesc array
+  int kpi[5];                // 64-column chunks per ring item
+};
+
+struct Bufs {
+  bf16* xn_a;      // [rows, d]    operand of the q/k/v product and of the LM head
+  bf16* xn_m;      // [rows, d]    operand of the gate/up product
+  bf16* attn;      // [rows, qd]   operand of the o product
+  bf16* act;       // [rows, dffn] operand of the down product
+  float* qkv;      // [rows, qd + 2 kvd] projections (norm factor applied, not rotated)
+  float* x1;       // [rows, d]    residual stream after attention
+  float* Gbuf;     // [rows, d]    layer outputs of the candidate states (Eq. 2)
+  float* att_acc;  // [rows*nq, chunk_cap, hd]
+  float2* att_ml;  // [rows*nq, chunk_cap]
+  float* ss_a;     // [G, Rcap] sums of squares per CTA feature slice (attention norm / head norm)
+  float* ss_m;     // [G, Rcap] (MLP norm)
+  float* cosp;     // [G, Rcap + MAX_ROWS, 5] partial dot products of Eq. 2
+  float4* head_best;  // [G, MAX_ROWS] (max, index bits, sum exp, -)
+  int* flags;      // [N_FLAGS, G]
+  const float2* rope;  // [T, hd/2] (cos, sin) of the rows' positions
+};
+
+struct Ctl {
+  int abort;
+  int status;
+  int pad[2];
+};
+
+struct Job {
+  int type, layer;
+  int S, T, R;
+  int C;         // cache positions visible to every row (own rows separate), or, when `uniform`,
+                 // the position of the first row
+  int uniform;   // 1: the rows' K/V go into the cache and attention is causal by position
+  int prep;      // 1: build the first operand from x_in when the job starts
+  int dp;        // 1: the layer output feeds the Eq. 2 step below
+  int row_off;   // JOB_HEAD: first row (of the previous job's rows) that goes through the head
+  int src_flag;  // flag kind that publishes this job's first operand (F_PREP / F_DOWN / F_SELECT)
+  int src_epoch;
+  const float* x_in;
+  long long ldx;
+  float* x_out;
+  long long ldo;
+  const float* norm_in;    // norm weight used by `prep`
+  const float* norm_mlp;
+  const float* norm_next;  // norm weight of the next product's operand, or null
+  bf16* ck;                // cache of this layer (written when `uniform`)
+  bf16* cv;
+  // Eq. 2 step i
+  int i, ell, diag, M;
+  const float* x_i;
+  const float* x_im1;
+  long long x_tok_stride;
+  const float* g_prev;
+  float* g_next;
+  float* D;
+  float* margin;
+  uint8_t* choice;
+  const uint8_t* forced;
+  float* g_final;  // written with g_next[M] when not null
+  // head
+  int32_t* argmax_out;
+  float* top1_out;
+};
+
+struct Params {
+  Cfg c;
+  Bufs b;
+  const Job* jobs;
+  int n_jobs;
+  const CUtensorMap* wmaps;  // [(L*7 + 1) * N_HEIGHTS]
+  const int* tabs;
+  Ctl* ctl;
+  unsigned long long* trace;  // optional [G, trace_cap] time stamps (ns)
+  int trace_cap;
+};
+
+// ------------------------------------------------------------------ small PTX helpers
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_i32(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_i32(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_volatile_i32(const int* p) {
+  int v;
+  asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ bool worker_and(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "barrier.cta.red.and.pred p, 1, 256, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)ok)
+      : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                                  uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+// x = hi + lo with hi, lo bf16: two values packed per register (first value in the low half)
+__device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t& lo) {
+  const bf16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
+  const bf16 xl = __float2bfloat16_rn(x - __bfloat162float(xh));
+  const bf16 yl = __float2bfloat16_rn(y - __bfloat162float(yh));
+  hi = (uint32_t)__bfloat16_as_ushort(xh) | ((uint32_t)__bfloat16_as_ushort(yh) << 16);
+  lo = (uint32_t)__bfloat16_as_ushort(xl) | ((uint32_t)__bfloat16_as_ushort(yl) << 16);
+}
+__device__ __forceinline__ uint2 pack4(float a, float b, float c2, float d2) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c2, d2);
+  uint2 u;
+  u.x = *reinterpret_cast<uint32_t*>(&lo);
+  u.y = *reinterpret_cast<uint32_t*>(&hi);
+  return u;
+}
+
+// ------------------------------------------------------------------ shared state
+struct Shared {
+  uint64_t full[NB], empty[NB];
+  uint64_t acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+  volatile int abort;
+  volatile int a_issued;    // ring items whose weight loads have been issued (warp 0 -> warp 1)
+  int flag;                 // broadcast of a one-thread decision to the workers
+  float rs[MAX_ROWS];       // per-row norm factors of the current product
+  int choice[MAX_ROWS + 2];
+};
+// The workers' scratch area holds either the attention K/V tiles or, during epilogues and the
+// Eq. 2 step, the cross-warp reduction tables below (the two uses never overlap in time).
+constexpr int RED_ROWS = MAX_ROWS + 16;
+struct RedTables {
+  float red[4][RED_ROWS][5];   // [lane quarter][row][value]: per-row sums of one warp
+  double cosv[RED_ROWS][5];
+};
+static_assert(sizeof(RedTables) <= SCRATCH_BYTES, "reduction tables must fit the scratch area");
+
+constexpr uint32_t WAIT_FAST = 1u << 12;
+constexpr uint32_t WAIT_SLOW = 1u << 22;  // x ~100 ns: gives up after roughly half a second
+
+__device__ __forceinline__ void raise_abort(Ctl* ctl, Shared* sh, bool timed_out) {
+  if (timed_out && !ld_volatile_i32(&ctl->abort)) atomicExch(&ctl->status, 1);
+  atomicExch(&ctl->abort, 1);
+  sh->abort = 1;
+}
+__device__ __forceinline__ bool aborted(Ctl* ctl, Shared* sh) {
+  if (sh->abort) return true;
+  if (ld_volatile_i32(&ctl->abort)) { sh->abort = 1; return true; }
+  return false;
+}
+
+// Bounded mbarrier wait that also ends when any CTA raised the abort flag.
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctl* ctl, Shared* sh) {
+  const uint32_t b = tc::smem_u32(bar);
+  for (uint32_t it = 0; it < WAIT_FAST; ++it)
+    if (tc::mbar_test(b, parity)) return true;
+  for (uint32_t it = 0; it < WAIT_SLOW; ++it) {
+    if (tc::mbar_test(b, parity)) return true;
+    if (aborted(ctl, sh)) return false;
+    __nanosleep(100);
+  }
+  raise_abort(ctl, sh, true);
+  return false;
+}
+
+// Bounded wait until flag >= epoch.
+__device__ __forceinline__ bool wait_flag(const int* flag, int epoch, Ctl* ctl, Shared* sh) {
+  for (uint32_t it = 0; it < (1u << 23); ++it) {
+    if (ld_acquire_i32(flag) >= epoch) return true;
+    if ((it & 15u) == 15u) {
+      if (aborted(ctl, sh)) return false;
+      if (it > 2048u) __nanosleep(64);
+    }
+  }
+  raise_abort(ctl, sh, true);
+  return false;
+}
+
+// ------------------------------------------------------------------ the schedule every role walks
+__device__ __forceinline__ int n_gemm_phases(const Job& J) {
+  return J.type == JOB_LAYER ? 4 : (J.type == JOB_HEAD ? 1 : 0);
+}
+__device__ __forceinline__ int gemm_kind(const Job& J, int ph) { return J.type == JOB_HEAD ? G_HEAD : ph; }
+__device__ __forceinline__ int kind_K(const Cfg& c, int kind) {
+  return kind == G_O ? c.qd : (kind == G_DOWN ? c.dffn : c.d);
+}
+__device__ __forceinline__ int kind_map_base(const Cfg& c, int kind, int layer) {
+  const int m = kind == G_QKV ? 0 : (kind == G_O ? 3 : (kind == G_GU ? 4 : (kind == G_DOWN ? 6 : 0)));
+  return ((kind == G_HEAD ? c.L * 7 : layer * 7) + m) * N_HEIGHTS;
+}
+
+struct Phase {   // one product of one job, as seen by this CTA
+  int kind, dual, kc, kpi, n_groups;  // chunks, chunks per item, items per tile
+  int tile0, n_tiles;                 // this CTA's TileDesc range
+  int map_base;
+  int g0;                             // chunk group this CTA starts its reduction at: CTAs walk the
+                                      // columns of their weight rows at staggered offsets so that the
+                                      // grid's reads spread over all HBM channels at any moment
+  __device__ __forceinline__ void init(const Params& p, const Job& J, int ph) {
+    const Cfg& c = p.c;
+    kind = gemm_kind(J, ph);
+    dual = kind == G_GU;
+    kc = (kind_K(c, kind) + BK - 1) / BK;
+    kpi = c.kpi[kind];
+    n_groups = (kc + kpi - 1) / kpi;
+    const int* ti = p.tabs + c.tile_idx[kind] + blockIdx.x;
+    tile0 = __ldg(ti);
+    n_tiles = __ldg(ti + 1) - tile0;
+    map_base = kind_map_base(c, kind, J.layer);
+    g0 = (int)(((long long)blockIdx.x * n_groups) / c.G);
+  }
+  __device__ __forceinline__ int group_at(int gi) const {
+    const int g = g0 + gi;
+    return g >= n_groups ? g - n_groups : g;
+  }
+};
+
+// ring placement of items: identical arithmetic in the three pipeline roles
+struct RingPos {
+  int pos;        // next free page
+  uint32_t item;  // items placed so far
+  // returns the page the item starts at and, through `footprint`, the pages it takes out of the ring
+  // (its own plus the unused tail when it wraps)
+  __device__ __forceinline__ int place(int pages, int ring_pages, int& footprint) {
+    footprint = pages;
+    if (pos + pages > ring_pages) { footprint += ring_pages - pos; pos = 0; }
+    const int at = pos;
+    pos += pages;
+    ++item;
+    return at;
+  }
+};
+
+__device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base) {
+  const Cfg& c = p.c;
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
+  const LoadDesc* loads = reinterpret_cast<const LoadDesc*>(p.tabs + c.loads_off);
+  RingPos rp{0, 0};
+  int used = 0;
+  uint32_t tail = 0;
+  int foot[NB];
+  const int b_pages = (c.BN * BK * 2) / PAGE;
+  for (int jb = 0; jb < p.n_jobs; ++jb) {
+    const Job& J = p.jobs[jb];
+    const int nph = n_gemm_phases(J);
+    for (int ph = 0; ph < nph; ++ph) {
+      Phase P;
+      P.init(p, J, ph);
+      for (int t = 0; t < P.n_tiles; ++t) {
+        const TileDesc td = tiles[P.tile0 + t];
+        const int a_pages = td.n_rows >> 3;
+        const int chunk_pages = (P.dual + 1) * a_pages + b_pages;
+        const int pages = P.kpi * chunk_pages;
+        // the tile's load list, fetched once: (row offset in bytes, map, first matrix row)
+        uint32_t l_off[MAX_TILE_LOADS];
+        int l_map[MAX_TILE_LOADS], l_y[MAX_TILE_LOADS];
+#pragma unroll
+        for (int l = 0; l < MAX_TILE_LOADS; ++l) {
+          l_off[l] = 0; l_map[l] = 0; l_y[l] = 0;
+          if (l < td.n_loads) {
+            const LoadDesc ld = loads[td.load0 + l];
+            l_off[l] = (uint32_t)ld.row_off * 128u; l_map[l] = P.map_base + ld.map_local; l_y[l] = ld.y0;
+          }
+        }
+        for (int gi = 0; gi < P.n_groups; ++gi) {
+          // make room: items leave the ring in the order they entered it
+          int fp;
+          RingPos probe = rp;
+          probe.place(pages, c.ring_pages, fp);
+          while (used + fp > c.ring_pages || rp.item - tail >= (uint32_t)NB) {
+            if (!wait_bar(&sh->empty[tail % NB], (tail / NB) & 1u, p.ctl, sh)) return;
+            used -= foot[tail % NB];
+            ++tail;
+          }
+          const uint32_t it = rp.item;
+          const int at = rp.place(pages, c.ring_pages, fp);
+          foot[it % NB] = fp;
+          used += fp;
+          const int k0 = P.group_at(gi) * P.kpi, k1 = min(P.kc, k0 + P.kpi);
+          const uint32_t full = tc::smem_u32(&sh->full[it % NB]);
+          tc::mbar_expect_tx(full, (uint32_t)((k1 - k0) * (P.dual + 1) * a_pages * PAGE));
+          for (int k = k0; k < k1; ++k) {
+            const uint32_t dst = ring_base + (uint32_t)(at + (k - k0) * chunk_pages) * PAGE;
+#pragma unroll
+            for (int l = 0; l < MAX_TILE_LOADS; ++l) {
+              if (l < td.n_loads) {
+                tc::tma_load_2d(dst + l_off[l], p.wmaps + l_map[l], full, k * BK, l_y[l], pol);
+                if (P.dual)  // the "up" rows of the same features follow the "gate" rows
+                  tc::tma_load_2d(dst + (uint32_t)(a_pages * PAGE) + l_off[l], p.wmaps + l_map[l] + N_HEIGHTS, full,
+                                  k * BK, l_y[l], pol);
+              }
+            }
+          }
+          sh->a_issued = (int)(it + 1);
+        }
+      }
+    }
+  }
+}
+
+// CTA that owns feature f of a split with `units` 8-feature units: the largest c with
+// floor(c units / G) <= f / 8  (CTAs with an empty range are never the largest such c)
+__device__ __forceinline__ int owner_of(int units, int G, int f) {
+  return (((f >> 3) + 1) * G - 1) / units;
+}
+
+__device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, const CUtensorMap* const* bmaps) {
+  const Cfg& c = p.c;
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
+  RingPos rp{0, 0};
+  const int b_pages = (c.BN * BK * 2) / PAGE;
+  const uint32_t b_bytes = (uint32_t)c.BN * BK * 2;
+  for (int jb = 0; jb < p.n_jobs; ++jb) {
+    const Job& J = p.jobs[jb];
+    const int nph = n_gemm_phases(J);
+    for (int ph = 0; ph < nph; ++ph) {
+      Phase P;
+      P.init(p, J, ph);
+      if (P.n_tiles == 0) continue;
+      // where this product's operand columns come from
+      int fkind, split, epoch, bmap;
+      if (P.kind == G_QKV) { fkind = J.src_flag; split = S_D; epoch = J.src_epoch; bmap = 0; }
+      else if (P.kind == G_O) { fkind = F_MERGE; split = -1; epoch = jb + 1; bmap = 1; }
+      else if (P.kind == G_GU) { fkind = F_O; split = S_D; epoch = jb + 1; bmap = 2; }
+      else if (P.kind == G_DOWN) { fkind = F_GU; split = S_F; epoch = jb + 1; bmap = 3; }
+      else { fkind = J.src_flag; split = S_D; epoch = J.src_epoch; bmap = 4; }
+      const int* flags = p.b.flags + fkind * c.G;
+      const int units = split >= 0 ? c.split_units[split] : 1;
+      const int Ktot = kind_K(c, P.kind);
+      uint32_t vmask[MAX_CTAS / 32];  // producers whose flag has been seen
+#pragma unroll
+      for (int w = 0; w < MAX_CTAS / 32; ++w) vmask[w] = 0u;
+      for (int t = 0; t < P.n_tiles; ++t) {
+        const TileDesc td = tiles[P.tile0 + t];
+        const int a_pages = td.n_rows >> 3;
+        const int chunk_pages = (P.dual + 1) * a_pages + b_pages;
+        const int pages = P.kpi * chunk_pages;
+        for (int gi = 0; gi < P.n_groups; ++gi) {
+          int fp;
+          const uint32_t it = rp.item;
+          const int at = rp.place(pages, c.ring_pages, fp);
+          // the weight producer has made room for this item
+          bool ok = false;
+          for (uint32_t w = 0; w < WAIT_SLOW; ++w) {
+            if ((uint32_t)sh->a_issued > it) { ok = true; break; }
+            if (w > WAIT_FAST) {
+              if (aborted(p.ctl, sh)) return;
+              __nanosleep(100);
+            }
+          }
+          if (!ok) { raise_abort(p.ctl, sh, true); return; }
+          const int k0 = P.group_at(gi) * P.kpi, k1 = min(P.kc, k0 + P.kpi);
+          // operand columns [k0*64, k1*64) must have been published by the CTAs that own them
+          int o_first, o_last;
+          const int col0 = k0 * BK, col1 = min(k1 * BK, Ktot) - 1;
+          if (split >= 0) { o_first = owner_of(units, c.G, col0); o_last = owner_of(units, c.G, col1); }
+          else { o_first = col0 / c.hd; o_last = col1 / c.hd; }   // head h is merged by CTA h % G
+          bool fresh = false;
+          for (int o = o_first; o <= o_last; ++o) {
+            const int cc = split >= 0 ? o : o % c.G;
+            if ((vmask[cc >> 5] >> (cc & 31)) & 1u) continue;
+            if (!wait_flag(flags + cc, epoch, p.ctl, sh)) return;
+            vmask[cc >> 5] |= 1u << (cc & 31);
+            fresh = true;
+          }
+          if (fresh) fence_proxy_async();  // the producers' ordinary stores before this thread's TMA reads
+          const uint32_t full = tc::smem_u32(&sh->full[it % NB]);
+          tc::mbar_expect_tx(full, (uint32_t)(k1 - k0) * b_bytes);
+          for (int k = k0; k < k1; ++k)
+            tc::tma_load_2d(ring_base + (uint32_t)(at + (k - k0) * chunk_pages + (P.dual + 1) * a_pages) * PAGE,
+                            bmaps[bmap], full, k * BK, 0, pol);
+        }
+      }
+    }
+  }
+}
+
+__device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint32_t tmem_base) {
+  const Cfg& c = p.c;
+  const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.BN >> 3) << 17) | (8u << 24);
+  const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
+  RingPos rp{0, 0};
+  const int b_pages = (c.BN * BK * 2) / PAGE;
+  uint32_t n_acc = 0;
+  for (int jb = 0; jb < p.n_jobs; ++jb) {
+    const Job& J = p.jobs[jb];
+    const int nph = n_gemm_phases(J);
+    for (int ph = 0; ph < nph; ++ph) {
+      Phase P;
+      P.init(p, J, ph);
+      for (int t = 0; t < P.n_tiles; ++t) {
+        const TileDesc td = tiles[P.tile0 + t];
+        const int a_pages = td.n_rows >> 3;
+        const int chunk_pages = (P.dual + 1) * a_pages + b_pages;
+        const int pages = P.kpi * chunk_pages;
+        const uint32_t buf = n_acc & 1u;
+        if (!wait_bar(&sh->acc_empty[buf], ((n_acc >> 1) & 1u) ^ 1u, p.ctl, sh)) return;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t acc = tmem_base + buf * 256u;
+        bool first = true;
+        for (int gi = 0; gi < P.n_groups; ++gi) {
+          int fp;
+          const uint32_t it = rp.item;
+          const int at = rp.place(pages, c.ring_pages, fp);
+          if (!wait_bar(&sh->full[it % NB], (it / NB) & 1u, p.ctl, sh)) return;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const int k0 = P.group_at(gi) * P.kpi, k1 = min(P.kc, k0 + P.kpi);
+          for (int k = k0; k < k1; ++k) {
+            const uint32_t sa = ring_base + (uint32_t)(at + (k - k0) * chunk_pages) * PAGE;
+            const uint32_t sb = sa + (uint32_t)((P.dual + 1) * a_pages) * PAGE;
+            const uint64_t da = tc::make_smem_desc(sa), db = tc::make_smem_desc(sb);
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk)
+              tc::mma_bf16(acc, da + 2 * kk, db + 2 * kk, idesc, (first && kk == 0) ? 0u : 1u);
+            if (P.dual) {
+              const uint64_t da2 = tc::make_smem_desc(sa + (uint32_t)a_pages * PAGE);
+#pragma unroll
+              for (int kk = 0; kk < BK / 16; ++kk)
+                tc::mma_bf16(acc + (uint32_t)c.BN, da2 + 2 * kk, db + 2 * kk, idesc, (first && kk == 0) ? 0u : 1u);
+            }
+            first = false;
+          }
+          tc::mma_commit(tc::smem_u32(&sh->empty[it % NB]));
+        }
+        tc::mma_commit(tc::smem_u32(&sh->acc_full[buf]));
+        ++n_acc;
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------ worker steps
+struct Worker {
+  const Params& p;
+  Shared* sh;
+  uint8_t* scratch;
+  uint32_t tmem_base;
+  int wtid, ww, lane;
+  uint32_t n_acc;
+  int n_mark;
+
+  __device__ __forceinline__ void mark() {
+    if (p.trace != nullptr && wtid == 0 && n_mark < p.trace_cap) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+      p.trace[(long long)blockIdx.x * p.trace_cap + n_mark] = t;
+    }
+    ++n_mark;
+  }
+
+  // all workers' stores of this step become visible, then the CTA's flag of `kind` says so
+  __device__ __forceinline__ void publish(int kind, int epoch) {
+    worker_sync();
+    if (wtid == 0) {
+      __threadfence();
+      st_release_i32(p.b.flags + kind * p.c.G + blockIdx.x, epoch);
+    }
+  }
+  // wait for flags [first, first + n) of `kind`: one flag per thread
+  __device__ bool wait_flags(int kind, int first, int n, int epoch) {
+    bool ok = true;
+    for (int k = wtid; k < n; k += WORKERS) ok = wait_flag(p.b.flags + kind * p.c.G + first + k, epoch, p.ctl, sh) && ok;
+    return worker_and(ok);
+  }
+
+  __device__ __forceinline__ const int* split_lo(int split) const { return p.tabs + p.c.split_lo[split]; }
+  __device__ __forceinline__ RedTables* tables() const { return reinterpret_cast<RedTables*>(scratch); }
+
+  // per-row factors rsqrt(mean(x^2) + eps) from the per-CTA sums of squares
+  __device__ void row_scales(const float* ss, int R, int row_off) {
+    const Cfg& c = p.c;
+    const int* dlo = split_lo(S_D);
+    for (int r = ww; r < R; r += 8) {
+      float s = 0.f;
+      for (int cc = lane; cc < c.G; cc += 32)
+        if (__ldg(dlo + cc + 1) > __ldg(dlo + cc)) s += __ldcg(ss + (long long)cc * c.Rcap + row_off + r);
+      s = warp_sum(s);
+      if (lane == 0) sh->rs[r] = rsqrtf(s / (float)c.d + c.eps);
+    }
+    worker_sync();
+  }
+
+  // operand of the first product from rows the engine did not produce itself: this CTA's
+  // slice of the d features
+  __device__ void prep(const Job& J, int epoch) {
+    const Cfg& c = p.c;
+    const int f_lo = __ldg(split_lo(S_D) + blockIdx.x), f_hi = __ldg(split_lo(S_D) + blockIdx.x + 1);
+    const int n4 = (f_hi - f_lo) >> 2;
+    for (int r = ww; r < J.R; r += 8) {
+      float ssq = 0.f;
+      for (int q = lane; q < n4; q += 32) {
+        const int col = f_lo + q * 4;
+        const float4 v = *reinterpret_cast<const float4*>(J.x_in + r * J.ldx + col);
+        const float4 w = *reinterpret_cast<const float4*>(J.norm_in + col);
+        ssq += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        *reinterpret_cast<uint2*>(p.b.xn_a + (long long)r * c.d + col) = pack4(v.x * w.x, v.y * w.y, v.z * w.z, v.w * w.w);
+      }
+      ssq = warp_sum(ssq);
+      if (lane == 0) p.b.ss_a[(long long)blockIdx.x * c.Rcap + r] = ssq;
+    }
+    fence_proxy_async();
+    publish(F_PREP, epoch);
+  }
+
+  // ---- epilogue of one accumulator: tile td of product P.kind.
+  // Thread (quarter q, lane) owns feature td.f0 + 32 q + lane; the two warps of a quarter take
+  // alternating blocks of 16 rows (accumulator columns).  Per-row sums over the CTA's features
+  // (sums of squares, cosine partials, arg-max) go through RedTables: one entry per (quarter, row).
+  __device__ bool epilogue(const Job& J, const Phase& P, const TileDesc& td, int tile_no) {
+    const Cfg& c = p.c;
+    RedTables* T = tables();
+    const int quarter = ww & 3, group = ww >> 2;
+    const int fl = quarter * 32 + lane;
+    const bool fv = fl < td.n_rows;
+    const int f = td.f0 + fl;
+    const int ncb = (J.R + 15) >> 4;
+    const bool resid = P.kind == G_O || P.kind == G_DOWN;
+    // residual rows of the first block are fetched before the accumulator is ready
+    float res[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) res[k] = 0.f;
+    if (resid && fv && group < ncb) {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int r = group * 16 + k;
+        if (r < J.R) res[k] = P.kind == G_O ? __ldcg(J.x_in + r * J.ldx + f) : __ldcg(p.b.x1 + (long long)r * c.d + f);
+      }
+    }
+    float wn = 0.f;
+    if (fv) {
+      if (P.kind == G_O) wn = __ldg(J.norm_mlp + f);
+      else if (P.kind == G_DOWN && !J.dp && J.norm_next) wn = __ldg(J.norm_next + f);
+    }
+    const uint32_t buf = n_acc & 1u;
+    bool ok = wait_bar(&sh->acc_full[buf], (n_acc >> 1) & 1u, p.ctl, sh);
+    ok = worker_and(ok);
+    if (!ok) return false;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if ((P.kind == G_QKV || P.kind == G_GU || P.kind == G_HEAD) && tile_no == 0) {
+      // the reduction consumed every operand column, so every CTA's sums of squares are published
+      row_scales(P.kind == G_GU ? p.b.ss_m : p.b.ss_a, J.R, P.kind == G_HEAD ? J.row_off : 0);
+    }
+    const uint32_t t_lane = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
+    for (int cb = group; cb < ncb; cb += 2) {
+      float v[16], u[16];
+      tc::tmem_ld16(t_lane + (uint32_t)(cb * 16), v);
+      if (P.dual) tc::tmem_ld16(t_lane + (uint32_t)(c.BN + cb * 16), u);
+      if (cb != group && resid && fv) {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          res[k] = 0.f;
+          if (r < J.R) res[k] = P.kind == G_O ? __ldcg(J.x_in + r * J.ldx + f) : __ldcg(p.b.x1 + (long long)r * c.d + f);
+        }
+      }
+      if (P.kind == G_QKV) {
+        if (fv) {
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            const int r = cb * 16 + k;
+            if (r < J.R) __stcg(p.b.qkv + (long long)r * (c.qd + 2 * c.kvd) + f, v[k] * sh->rs[r]);
+          }
+        }
+      } else if (P.kind == G_O) {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          if (r >= J.R) break;
+          const float y = fv ? res[k] + v[k] : 0.f;
+          if (fv) {
+            __stcg(p.b.x1 + (long long)r * c.d + f, y);
+            p.b.xn_m[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
+          }
+          const float s2 = warp_sum(y * y);
+          if (lane == 0) T->red[quarter][r][0] = s2;
+        }
+      } else if (P.kind == G_GU) {
+        if (fv) {
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            const int r = cb * 16 + k;
+            if (r < J.R) {
+              const float rs = sh->rs[r];
+              p.b.act[(long long)r * c.dffn + f] = __float2bfloat16_rn(silu_f(rs * v[k]) * (rs * u[k]));
+            }
+          }
+        }
+      } else if (P.kind == G_DOWN) {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          if (r >= J.R) break;
+          const float y = fv ? res[k] + v[k] : 0.f;
+          if (J.dp) {
+            // candidate state's layer output + its cosine partials  x_i . y  and  y . y
+            if (fv) __stcg(p.b.Gbuf + (long long)r * c.d + f, y);
+            const float xi = fv ? __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f) : 0.f;
+            const float a = warp_sum(xi * y), b2 = warp_sum(y * y);
+            if (lane == 0) { T->red[quarter][r][0] = a; T->red[quarter][r][1] = b2; }
+          } else {
+            if (fv) {
+              __stcg(J.x_out + r * J.ldo + f, y);
+              if (J.norm_next) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
+            }
+            if (J.norm_next) {
+              const float s2 = warp_sum(y * y);
+              if (lane == 0) T->red[quarter][r][0] = s2;
+            }
+          }
+        }
+      } else {  // G_HEAD: best logit of this tile per row (lowest index on ties) and sum of exp
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          if (r >= J.R) break;
+          const float mine = fv ? v[k] * sh->rs[r] : -INFINITY;
+          float best = mine;
+          int bi = fv ? f : 0x7fffffff;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+          }
+          const float se = warp_sum(fv ? __expf(mine - best) : 0.f);
+          if (lane == 0) {
+            T->red[quarter][r][0] = best;
+            T->red[quarter][r][1] = __int_as_float(bi);
+            T->red[quarter][r][2] = se;
+          }
+        }
+      }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    worker_sync();
+    if (wtid == 0) mbar_arrive(tc::smem_u32(&sh->acc_empty[buf]));
+    ++n_acc;
+    // cross-warp part of the per-row sums: add the four quarters in a fixed order
+    if (P.kind == G_O || (P.kind == G_DOWN && !J.dp && J.norm_next)) {
+      float* ss = (P.kind == G_O ? p.b.ss_m : p.b.ss_a) + (long long)blockIdx.x * c.Rcap;
+      for (int r = wtid; r < J.R; r += WORKERS) {
+        const float s2 = T->red[0][r][0] + T->red[1][r][0] + T->red[2][r][0] + T->red[3][r][0];
+        ss[r] = (tile_no == 0 ? 0.f : ss[r]) + s2;
+      }
+    } else if (P.kind == G_HEAD) {
+      for (int r = wtid; r < J.R; r += WORKERS) {
+        float best = -INFINITY, se = 0.f;
+        int bi = 0x7fffffff;
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const float ov = T->red[q4][r][0];
+          const int oi = __float_as_int(T->red[q4][r][1]);
+          if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+        }
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const float ov = T->red[q4][r][0];
+          if (ov != -INFINITY) se += T->red[q4][r][2] * __expf(ov - best);
+        }
+        float4* dst = p.b.head_best + (long long)blockIdx.x * MAX_ROWS + r;
+        if (tile_no > 0) {
+          const float4 o = *dst;
+          const int oi = __float_as_int(o.y);
+          const float nb = fmaxf(o.x, best);
+          se = se * __expf(best - nb) + o.z * __expf(o.x - nb);
+          if (o.x > best || (o.x == best && oi < bi)) { best = o.x; bi = oi; }
+        }
+        *dst = make_float4(best, __int_as_float(bi), se, 0.f);
+      }
+    }
+    if (P.kind == G_O || P.kind == G_GU || (P.kind == G_DOWN && !J.dp && J.norm_next)) fence_proxy_async();
+    if (P.kind == G_HEAD || P.kind == G_O || (P.kind == G_DOWN && !J.dp)) worker_sync();  // tables reused by the next tile
+    return true;
+  }
+
+  // skip candidate of state j (1-based) at row t: g[i-1][j-1]
+  __device__ __forceinline__ const float* skip_src(const Job& J, int j, int t) const {
+    return j == 1 ? J.x_im1 + t * J.x_tok_stride : J.g_prev + ((long long)(j - 1) * J.T + t) * p.c.d;
+  }
+
+  // ---- Eq. 2 step i over this CTA's slice of the d features (thread <-> feature as in the
+  // epilogue, so a thread meets again the layer outputs it stored itself):
+  //   (1) per-CTA partial dot products -> cosp, publish;
+  //   (2) wait for every CTA, add the partials in CTA order, decide (every CTA decides alike);
+  //   (3) write this CTA's slice of g[i][.] and of the next step's operand, publish.
+  // have_apply: the epilogue left the apply candidates' partials in the tables.
+  __device__ bool dp_step(const Job& J, int jb, bool have_apply) {
+    const Cfg& c = p.c;
+    RedTables* T = tables();
+    const int f_lo = __ldg(split_lo(S_D) + blockIdx.x), f_hi = __ldg(split_lo(S_D) + blockIdx.x + 1);
+    const int quarter = ww & 3, group = ww >> 2;
+    const int fl = quarter * 32 + lane;
+    const bool fv = fl < f_hi - f_lo;   // a slice has at most 128 features (checked on the host)
+    const int f = f_lo + fl;
+    const int n_states = J.ell + (J.diag ? 1 : 0);
+    const int rows = n_states * J.T;
+    const int ncb = (rows + 15) >> 4;
+    const long long cstride = (long long)(c.Rcap + MAX_ROWS) * 5;
+    // (1) skip candidates (rows of every state 1..n_states)
+    for (int cb = group; cb < ncb; cb += 2) {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int r = cb * 16 + k;
+        if (r >= rows) break;
+        const int j = r / J.T + 1, t = r % J.T;
+        const float xi = fv ? __ldg(J.x_i + t * J.x_tok_stride + f) : 0.f;
+        const float sv = fv ? __ldcg(skip_src(J, j, t) + f) : 0.f;
+        const float a = warp_sum(xi * sv), b2 = warp_sum(sv * sv), x2 = warp_sum(xi * xi);
+        if (lane == 0) {
+          T->red[quarter][r][2] = a; T->red[quarter][r][3] = b2; T->red[quarter][r][4] = x2;
+          if (!(have_apply && r < J.ell * J.T)) { T->red[quarter][r][0] = 0.f; T->red[quarter][r][1] = 0.f; }
+        }
+      }
+    }
+    worker_sync();
+    for (int idx = wtid; idx < rows * 5; idx += WORKERS) {
+      const int r = idx / 5, k = idx % 5;
+      __stcg(p.b.cosp + blockIdx.x * cstride + idx, T->red[0][r][k] + T->red[1][r][k] + T->red[2][r][k] + T->red[3][r][k]);
+    }
+    publish(F_DOWN, jb + 1);
+    // (2) every CTA's partials, added in CTA order by a fixed shuffle tree
+    if (!wait_flags(F_DOWN, 0, c.G, jb + 1)) return false;
+    for (int r = ww; r < rows; r += 8) {
+      double v[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
+      for (int cc = lane; cc < c.G; cc += 32) {
+        const float* src = p.b.cosp + cc * cstride + (long long)r * 5;
+        float f5[5];
+#pragma unroll
+        for (int k = 0; k < 5; ++k) f5[k] = __ldcg(src + k);
+#pragma unroll
+        for (int k = 0; k < 5; ++k) v[k] += (double)f5[k];
+      }
+#pragma unroll
+      for (int k = 0; k < 5; ++k) {
+        v[k] = warp_sum_d(v[k]);
+        if (lane == 0) T->cosv[r][k] = v[k];
+      }
+    }
+    worker_sync();
+    if (wtid < n_states) {
+      const int j = wtid + 1;
+      double app = 0.0, skp = 0.0;
+      for (int t = 0; t < J.T; ++t) {
+        const double* v = T->cosv[(j - 1) * J.T + t];
+        const double nx = fmax(sqrt(v[4]), 1e-12);
+        app += v[0] / (nx * fmax(sqrt(v[1]), 1e-12));
+        skp += v[2] / (nx * fmax(sqrt(v[3]), 1e-12));
+      }
+      const float s_app = (float)(app / J.T), s_skip = (float)(skp / J.T);
+      int take = 0;
+      if (j <= J.ell) {
+        take = s_app > s_skip;
+        if (J.forced && J.forced[j] != 255) take = (J.forced[j] == 0);
+      }
+      sh->choice[j] = take;
+      if (blockIdx.x == 0) {
+        J.D[j] = take ? s_app : s_skip;
+        J.choice[j] = take ? 0 : 1;
+        if (J.margin && j <= J.ell) J.margin[j] = s_app - s_skip;
+      }
+    }
+    if (blockIdx.x == 0 && wtid == 0) {
+      J.D[0] = 1.0f;
+      J.choice[0] = 0;
+    }
+    worker_sync();
+    // (3) write-back
+    const float wn = (fv && J.norm_next) ? __ldg(J.norm_next + f) : 0.f;
+    for (int cb = group; cb < ncb; cb += 2) {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int r = cb * 16 + k;
+        if (r >= rows) break;
+        const int j = r / J.T + 1, t = r % J.T;
+        float y = 0.f;
+        if (fv) {
+          y = sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f);
+          __stcg(J.g_next + ((long long)j * J.T + t) * c.d + f, y);
+          if (J.g_final && j == J.M) J.g_final[(long long)t * c.d + f] = y;
+          if (J.norm_next) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
+        }
+        if (J.norm_next) {
+          const float s2 = warp_sum(y * y);
+          if (lane == 0) T->red[quarter][r][0] = s2;
+        }
+      }
+    }
+    worker_sync();
+    if (J.norm_next)
+      for (int r = wtid; r < rows; r += WORKERS)
+        p.b.ss_a[(long long)blockIdx.x * c.Rcap + r] = T->red[0][r][0] + T->red[1][r][0] + T->red[2][r][0] + T->red[3][r][0];
+    fence_proxy_async();
+    publish(F_SELECT, jb + 1);
+    return true;
+  }
+
+  // ---- attention: partial softmax over one run of cache keys or one chunk of own rows.
+  // q, k, v of the rows come from the projection buffer (norm factor applied, not rotated): they
+  // are rotated here; new keys / values are rounded to the cache type before use.
+  template <int HD>
+  __device__ bool attention_partials(const Job& J, int jb) {
+    const Cfg& c = p.c;
+    constexpr int KS = HD / 16;
+    constexpr int NBLK = HD / 8;
+    constexpr int LD = HD + 8;
+    constexpr int HALF = HD / 2;
+    bf16* k_s = reinterpret_cast<bf16*>(scratch);
+    bf16* v_s = k_s + ATT_KEYS * LD;
+    const int Gq = c.nq / c.nkv;
+    const int Pn = J.R * Gq;
+    const int n_pbg = (Pn + 127) / 128;
+    const int k_tot = J.uniform ? J.C + J.T : J.C;
+    const int n_runs = (k_tot + c.run_len - 1) / c.run_len;
+    const int n_own = J.uniform ? 0 : (J.R + ATT_KEYS - 1) / ATT_KEYS;
+    const int n_chunks = n_runs + n_own;
+    const int n_items = c.nkv * n_chunks * n_pbg;
+    const int g8 = lane >> 2, c4 = lane & 3;
+    const long long kvld = c.kvd;
+    const int qkvd = c.qd + 2 * c.kvd;
+    const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;
+    const int qunits = c.split_units[S_QKV];
+    for (int it = blockIdx.x; it < n_items; it += c.G) {
+      const int pbg = it % n_pbg;
+      const int chunk = (it / n_pbg) % n_chunks;
+      const int kvh = it / (n_pbg * n_chunks);
+      const bool own = chunk >= n_runs;
+      // producers of this kv head's q heads, k head and v head
+      {
+        const int q0 = kvh * Gq * HD, q1 = q0 + Gq * HD - 1;
+        const int k0 = c.qd + kvh * HD, v0 = c.qd + c.kvd + kvh * HD;
+        const int a0 = owner_of(qunits, c.G, q0), a1 = owner_of(qunits, c.G, q1);
+        const int b0 = owner_of(qunits, c.G, k0), b1 = owner_of(qunits, c.G, k0 + HD - 1);
+        const int d0 = owner_of(qunits, c.G, v0), d1 = owner_of(qunits, c.G, v0 + HD - 1);
+        bool ok = true;
+        const int na = a1 - a0 + 1, nb2 = b1 - b0 + 1, nd = d1 - d0 + 1;
+        for (int k = wtid; k < na + nb2 + nd; k += WORKERS) {
+          const int cc = k < na ? a0 + k : (k < na + nb2 ? b0 + (k - na) : d0 + (k - na - nb2));
+          ok = wait_flag(p.b.flags + F_QKV * c.G + cc, jb + 1, p.ctl, sh) && ok;
+        }
+        if (!worker_and(ok)) return false;
+      }
+      const int p0 = (pbg * 8 + ww) * 16;
+      const bool active = p0 < Pn;
+      int rr[2], hq[2];
+      bool pv[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int pp = p0 + g8 + h * 8;
+        pv[h] = pp < Pn;
+        rr[h] = pv[h] ? pp / Gq : 0;
+        hq[h] = kvh * Gq + (pv[h] ? pp % Gq : 0);
+      }
+      // q fragments, rotated: element d pairs with d +- HD/2
+      uint32_t qh[KS][4], ql[KS][4];
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+#pragma unroll
+          for (int kh = 0; kh < 2; ++kh) {
+            float2 v = make_float2(0.f, 0.f);
+            if (active && pv[h]) {
+              const int dd = ks * 16 + kh * 8 + c4 * 2;          // dims dd, dd+1 (same half)
+              const int i = dd % HALF;
+              const float* qr = p.b.qkv + (long long)rr[h] * qkvd + hq[h] * HD;
+              const float2 lo2 = __ldcg(reinterpret_cast<const float2*>(qr + i));
+              const float2 hi2 = __ldcg(reinterpret_cast<const float2*>(qr + i + HALF));
+              const float2 cs0 = p.b.rope[(long long)(rr[h] % J.T) * HALF + i];
+              const float2 cs1 = p.b.rope[(long long)(rr[h] % J.T) * HALF + i + 1];
+              if (dd < HALF) v = make_float2(lo2.x * cs0.x - hi2.x * cs0.y, lo2.y * cs1.x - hi2.y * cs1.y);
+              else v = make_float2(hi2.x * cs0.x + lo2.x * cs0.y, hi2.y * cs1.x + lo2.y * cs1.y);
+              v.x *= qscale;
+              v.y *= qscale;
+            }
+            split2(v.x, v.y, qh[ks][h + kh * 2], ql[ks][h + kh * 2]);
+          }
+        }
+      }
+      float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+      float o[NBLK][4];
+#pragma unroll
+      for (int nb = 0; nb < NBLK; ++nb) { o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f; }
+
+      int key_lo, key_hi;
+      if (!own) { key_lo = chunk * c.run_len; key_hi = min(k_tot, key_lo + c.run_len); }
+      else { key_lo = (chunk - n_runs) * ATT_KEYS; key_hi = min(J.R, key_lo + ATT_KEYS); }
+      for (int key0 = key_lo; key0 < key_hi; key0 += ATT_KEYS) {
+        const int nkeys = min(ATT_KEYS, key_hi - key0);
+        worker_sync();  // previous tile consumed
+        // K/V tile: cache rows as they are; rows of this call rotated / rounded from the projections
+        for (int vv = wtid; vv < ATT_KEYS * (HD / 8); vv += WORKERS) {
+          const int row = vv / (HD / 8), cv8 = vv % (HD / 8);
+          uint4 kk = make_uint4(0, 0, 0, 0), vq = make_uint4(0, 0, 0, 0);
+          if (row < nkeys) {
+            const int key = key0 + row;
+            const int new_row = own ? key : (J.uniform ? key - J.C : -1);
+            if (new_row < 0) {
+              kk = __ldcg(reinterpret_cast<const uint4*>(J.ck + (long long)key * kvld + kvh * HD + cv8 * 8));
+              vq = __ldcg(reinterpret_cast<const uint4*>(J.cv + (long long)key * kvld + kvh * HD + cv8 * 8));
+            } else {
+              const float* kr = p.b.qkv + (long long)new_row * qkvd + c.qd + kvh * HD;
+              const float* vr = kr + c.kvd;
+              const int d0 = cv8 * 8, i0 = d0 % HALF;
+              float ka[8], kb[8], vf[8];
+#pragma unroll
+              for (int e = 0; e < 8; e += 4) {
+                const float4 a4 = __ldcg(reinterpret_cast<const float4*>(kr + i0 + e));
+                const float4 b4 = __ldcg(reinterpret_cast<const float4*>(kr + i0 + HALF + e));
+                const float4 v4 = __ldcg(reinterpret_cast<const float4*>(vr + d0 + e));
+                ka[e] = a4.x; ka[e + 1] = a4.y; ka[e + 2] = a4.z; ka[e + 3] = a4.w;
+                kb[e] = b4.x; kb[e + 1] = b4.y; kb[e + 2] = b4.z; kb[e + 3] = b4.w;
+                vf[e] = v4.x; vf[e + 1] = v4.y; vf[e + 2] = v4.z; vf[e + 3] = v4.w;
+              }
+              float kro[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float2 cs = p.b.rope[(long long)(new_row % J.T) * HALF + i0 + e];
+                kro[e] = d0 < HALF ? ka[e] * cs.x - kb[e] * cs.y : kb[e] * cs.x + ka[e] * cs.y;
+              }
+              const uint2 k01 = pack4(kro[0], kro[1], kro[2], kro[3]), k23 = pack4(kro[4], kro[5], kro[6], kro[7]);
+              const uint2 v01 = pack4(vf[0], vf[1], vf[2], vf[3]), v23 = pack4(vf[4], vf[5], vf[6], vf[7]);
+              kk = make_uint4(k01.x, k01.y, k23.x, k23.y);
+              vq = make_uint4(v01.x, v01.y, v23.x, v23.y);
+              if (J.uniform && pbg == 0) {  // this item owns the cache rows of its keys
+                *reinterpret_cast<uint4*>(J.ck + (long long)key * kvld + kvh * HD + cv8 * 8) = kk;
+                *reinterpret_cast<uint4*>(J.cv + (long long)key * kvld + kvh * HD + cv8 * 8) = vq;
+              }
+            }
+          }
+          *reinterpret_cast<uint4*>(k_s + row * LD + cv8 * 8) = kk;
+          *reinterpret_cast<uint4*>(v_s + row * LD + cv8 * 8) = vq;
+        }
+        worker_sync();
+        if (!active) continue;
+        float s[4][4];
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb) {
+          s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
+          const bf16* kr = k_s + (nb * 8 + g8) * LD + c4 * 2;
+#pragma unroll
+          for (int ks = 0; ks < KS; ++ks) {
+            const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kr + ks * 16);
+            const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kr + ks * 16 + 8);
+            mma_16816(s[nb], qh[ks], b0, b1);
+            mma_16816(s[nb], ql[ks], b0, b1);
+          }
+        }
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int h = e >> 1;
+            const int key = key0 + nb * 8 + c4 * 2 + (e & 1);
+            bool vis = pv[h] && key < key_hi;
+            if (own) vis = vis && (key / J.T == rr[h] / J.T) && key <= rr[h];
+            else if (J.uniform) vis = vis && key <= J.C + rr[h];
+            if (!vis) s[nb][e] = -INFINITY;
+            mx[h] = fmaxf(mx[h], s[nb][e]);
+          }
+        }
+        float corr[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+          mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+          const float m_new = fmaxf(m[h], mx[h]);
+          corr[h] = (m_new == -INFINITY) ? 1.f : exp2f(m[h] - m_new);
+          m[h] = m_new;
+        }
+        float rsum[2] = {0.f, 0.f};
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int h = e >> 1;
+            const float pe = (s[nb][e] == -INFINITY) ? 0.f : exp2f(s[nb][e] - m[h]);
+            s[nb][e] = pe;
+            rsum[h] += pe;
+          }
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 1);
+          rsum[h] += __shfl_xor_sync(0xffffffffu, rsum[h], 2);
+          l[h] = l[h] * corr[h] + rsum[h];
+        }
+#pragma unroll
+        for (int nb = 0; nb < NBLK; ++nb) {
+          o[nb][0] *= corr[0]; o[nb][1] *= corr[0];
+          o[nb][2] *= corr[1]; o[nb][3] *= corr[1];
+        }
+#pragma unroll
+        for (int k2 = 0; k2 < 2; ++k2) {
+          uint32_t ph[4], pl[4];
+          split2(s[2 * k2][0], s[2 * k2][1], ph[0], pl[0]);
+          split2(s[2 * k2][2], s[2 * k2][3], ph[1], pl[1]);
+          split2(s[2 * k2 + 1][0], s[2 * k2 + 1][1], ph[2], pl[2]);
+          split2(s[2 * k2 + 1][2], s[2 * k2 + 1][3], ph[3], pl[3]);
+          const int mrow = k2 * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          const int mcol = (lane >> 4) * 8;
+#pragma unroll
+          for (int nb = 0; nb < NBLK; nb += 2) {
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4_trans(tc::smem_u32(v_s + mrow * LD + nb * 8 + mcol), b0, b1, b2, b3);
+            mma_16816(o[nb], ph, b0, b1);
+            mma_16816(o[nb], pl, b0, b1);
+            mma_16816(o[nb + 1], ph, b2, b3);
+            mma_16816(o[nb + 1], pl, b2, b3);
+          }
+        }
+      }
+      if (active) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (!pv[h]) continue;
+          const long long idx = ((long long)rr[h] * c.nq + hq[h]) * c.chunk_cap + chunk;
+          float* pa = p.b.att_acc + idx * HD + c4 * 2;
+#pragma unroll
+          for (int nb = 0; nb < NBLK; ++nb)
+            __stcg(reinterpret_cast<float2*>(pa + nb * 8), make_float2(o[nb][2 * h], o[nb][2 * h + 1]));
+          if (c4 == 0) __stcg(p.b.att_ml + idx, make_float2(m[h], l[h]));
+        }
+      }
+    }
+    publish(F_ATTN, jb + 1);
+    return true;
+  }
+
+  // all chunks of query head h merged, one warp per row; head h is merged by CTA h % G
+  template <int DPL>
+  __device__ bool attention_merge(const Job& J, int jb) {
+    const Cfg& c = p.c;
+    const int Gq = c.nq / c.nkv;
+    const int n_pbg = (J.R * Gq + 127) / 128;
+    const int k_tot = J.uniform ? J.C + J.T : J.C;
+    const int n_runs = (k_tot + c.run_len - 1) / c.run_len;
+    const int n_chunks = n_runs + (J.uniform ? 0 : (J.R + ATT_KEYS - 1) / ATT_KEYS);
+    for (int hq = blockIdx.x; hq < c.nq; hq += c.G) {
+      // the items of this head's kv head ran on CTAs (item index) % G
+      const int kvh = hq / Gq;
+      const int it0 = kvh * n_chunks * n_pbg, n_it = n_chunks * n_pbg;
+      bool ok = true;
+      for (int k = wtid; k < min(n_it, c.G); k += WORKERS)
+        ok = wait_flag(p.b.flags + F_ATTN * c.G + (it0 + k) % c.G, jb + 1, p.ctl, sh) && ok;
+      if (!worker_and(ok)) return false;
+      for (int r = ww; r < J.R; r += 8) {
+        const long long pr = (long long)r * c.nq + hq;
+        const float2* ml = p.b.att_ml + pr * c.chunk_cap;
+        float2 v0 = make_float2(-INFINITY, 0.f), v1 = v0;
+        if (lane < n_chunks) v0 = __ldcg(ml + lane);
+        if (lane + 32 < n_chunks) v1 = __ldcg(ml + lane + 32);
+        const float mx = warp_max(fmaxf(v0.x, v1.x));
+        const float w0 = v0.x == -INFINITY ? 0.f : exp2f(v0.x - mx);
+        const float w1 = v1.x == -INFINITY ? 0.f : exp2f(v1.x - mx);
+        const float den = warp_sum(w0 * v0.y + w1 * v1.y);
+        float num[DPL];
+#pragma unroll
+        for (int k = 0; k < DPL; ++k) num[k] = 0.f;
+        const float* acc = p.b.att_acc + pr * c.chunk_cap * c.hd + lane * DPL;
+        for (int ch0 = 0; ch0 < n_chunks; ch0 += 8) {
+          float a[8][DPL];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+#pragma unroll
+            for (int k = 0; k < DPL; ++k) a[e][k] = 0.f;
+            if (ch0 + e < n_chunks) {
+              if (DPL == 4) {
+                const float4 t = __ldcg(reinterpret_cast<const float4*>(acc + (long long)(ch0 + e) * c.hd));
+                a[e][0] = t.x; a[e][1] = t.y; a[e][2] = t.z; a[e][3] = t.w;
+              } else {
+                const float2 t = __ldcg(reinterpret_cast<const float2*>(acc + (long long)(ch0 + e) * c.hd));
+                a[e][0] = t.x; a[e][1] = t.y;
+              }
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int ch = ch0 + e;
+            const float wa = __shfl_sync(0xffffffffu, w0, ch & 31), wb = __shfl_sync(0xffffffffu, w1, ch & 31);
+            const float w = ch < 32 ? wa : wb;
+#pragma unroll
+            for (int k = 0; k < DPL; ++k) num[k] = fmaf(w, a[e][k], num[k]);
+          }
+        }
+        bf16* dst = p.b.attn + pr * c.hd + lane * DPL;
+        const float inv = 1.0f / den;
+        if (DPL == 4) {
+          *reinterpret_cast<uint2*>(dst) = pack4(num[0] * inv, num[1] * inv, num[2] * inv, num[DPL - 1] * inv);
+        } else {
+          __nv_bfloat162 t = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
+          *reinterpret_cast<__nv_bfloat162*>(dst) = t;
+        }
+      }
+    }
+    fence_proxy_async();
+    publish(F_MERGE, jb + 1);
+    return true;
+  }
+
+  // L2 prefetch of the cache lines this CTA's attention items will read
+  __device__ void attention_prefetch(const Job& J) {
+    const Cfg& c = p.c;
+    const int Gq = c.nq / c.nkv;
+    const int n_pbg = (J.R * Gq + 127) / 128;
+    const int k_tot = J.uniform ? J.C + J.T : J.C;
+    const int n_runs = (k_tot + c.run_len - 1) / c.run_len;
+    const int n_own = J.uniform ? 0 : (J.R + ATT_KEYS - 1) / ATT_KEYS;
+    const int n_chunks = n_runs + n_own;
+    const int n_items = c.nkv * n_chunks * n_pbg;
+    const int lpr = (c.hd * 2 + 127) / 128;
+    for (int it = blockIdx.x; it < n_items; it += c.G) {
+      const int chunk = (it / n_pbg) % n_chunks;
+      const int kvh = it / (n_pbg * n_chunks);
+      if (chunk >= n_runs) continue;
+      const int key_lo = chunk * c.run_len, key_hi = min(J.C, key_lo + c.run_len);
+      const int n_lines = (key_hi - key_lo) * lpr * 2;
+      for (int v = wtid; v < n_lines; v += WORKERS) {
+        const int which = v & 1, ln = (v >> 1) % lpr, key = key_lo + (v >> 1) / lpr;
+        const bf16* addr = (which ? J.cv : J.ck) + (long long)key * c.kvd + kvh * c.hd + ln * 64;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(addr));
+      }
+    }
+  }
+
+  // greedy token of each head row from every CTA's best (CTA 0, one warp per row)
+  __device__ bool head_merge(const Job& J, int jb) {
+    const Cfg& c = p.c;
+    publish(F_HEAD, jb + 1);
+    if (blockIdx.x != 0) return true;
+    if (!wait_flags(F_HEAD, 0, c.G, jb + 1)) return false;
+    const int* vlo = split_lo(S_V);
+    for (int r = ww; r < J.R; r += 8) {
+      float best = -INFINITY;
+      int bi = 0x7fffffff;
+      for (int cc = lane; cc < c.G; cc += 32) {
+        if (__ldg(vlo + cc + 1) <= __ldg(vlo + cc)) continue;
+        const float4 v = __ldcg(p.b.head_best + (long long)cc * MAX_ROWS + r);
+        const int vi = __float_as_int(v.y);
+        if (v.x > best || (v.x == best && vi < bi)) { best = v.x; bi = vi; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+      }
+      float se = 0.f;
+      for (int cc = lane; cc < c.G; cc += 32) {
+        if (__ldg(vlo + cc + 1) <= __ldg(vlo + cc)) continue;
+        const float4 v = __ldcg(p.b.head_best + (long long)cc * MAX_ROWS + r);
+        se += v.z * __expf(v.x - best);
+      }
+      se = warp_sum(se);
+      if (lane == 0) {
+        J.argmax_out[r] = bi;
+        if (J.top1_out) J.top1_out[r] = 1.0f / se;
+      }
+    }
+    return true;
+  }
+
+  // ---- the job list
+  __device__ bool run() {
+    const Cfg& c = p.c;
+    const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
+    for (int jb = 0; jb < p.n_jobs; ++jb) {
+      const Job& J = p.jobs[jb];
+      mark();
+      if (J.type == JOB_SELECT) {
+        if (!dp_step(J, jb, false)) return false;
+        continue;
+      }
+      if (J.type == JOB_HEAD) {
+        Phase P;
+        P.init(p, J, 0);
+        for (int t = 0; t < P.n_tiles; ++t)
+          if (!epilogue(J, P, tiles[P.tile0 + t], t)) return false;
+        if (!head_merge(J, jb)) return false;
+        continue;
+      }
+      attention_prefetch(J);
+      if (J.prep) prep(J, jb + 1);
+      for (int ph = 0; ph < 4; ++ph) {
+        Phase P;
+        P.init(p, J, ph);
+        for (int t = 0; t < P.n_tiles; ++t)
+          if (!epilogue(J, P, tiles[P.tile0 + t], t)) return false;
+        mark();
+        if (ph == G_QKV) {
+          publish(F_QKV, jb + 1);
+          if (!(c.hd == 128 ? attention_partials<128>(J, jb) : attention_partials<64>(J, jb))) return false;
+          mark();
+          if (!(c.hd == 128 ? attention_merge<4>(J, jb) : attention_merge<2>(J, jb))) return false;
+          mark();
+        } else if (ph == G_O) {
+          publish(F_O, jb + 1);
+        } else if (ph == G_GU) {
+          publish(F_GU, jb + 1);
+        } else {
+          if (J.dp) {
+            if (!dp_step(J, jb, P.n_tiles > 0)) return false;
+          } else {
+            publish(F_DOWN, jb + 1);
+          }
+          mark();
+        }
+      }
+    }
+    return true;
+  }
+};
+
+// ------------------------------------------------------------------ the kernel
+__global__ void __launch_bounds__(THREADS, 1)
+engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constant__ CUtensorMap map_attn,
+              const __grid_constant__ CUtensorMap map_xn_m, const __grid_constant__ CUtensorMap map_act,
+              const __grid_constant__ CUtensorMap map_head, const __grid_constant__ Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ Shared sh;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t* ring = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t ring_base = tc::smem_u32(ring);
+  uint8_t* scratch = ring + (size_t)p.c.ring_pages * PAGE;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NB; ++s) {
+      tc::mbar_init(tc::smem_u32(&sh.full[s]), 2);   // weight rows + operand tile
+      tc::mbar_init(tc::smem_u32(&sh.empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      tc::mbar_init(tc::smem_u32(&sh.acc_full[b]), 1);
+      tc::mbar_init(tc::smem_u32(&sh.acc_empty[b]), 1);
+    }
+    sh.abort = 0;
+    sh.a_issued = 0;
+    sh.flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 3) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(&sh.tmem_base)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = sh.tmem_base;
+
+  if (warp == 0) {
+    if (lane == 0) producer_a(p, &sh, ring_base);
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const CUtensorMap* bmaps[5] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head};
+      producer_b(p, &sh, ring_base, bmaps);
+    }
+  } else if (warp == 2) {
+    if (lane == 0) mma_issuer(p, &sh, ring_base, tmem_base);
+  } else if (warp >= 4) {
+    Worker w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0};
+    w.run();
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (sh.abort) {
+    // a wait gave up somewhere: let copies and MMAs still in flight land before the CTA's
+    // shared and tensor memory are released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  if (warp == 3) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace pk
+}  // namespace clasp

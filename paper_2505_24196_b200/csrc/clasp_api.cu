@@ -140,7 +140,7 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
     w.ss_m = (float*)take(G * rcap * 4);
     w.cosp = (float*)take(G * (rcap + pk::MAX_ROWS) * 5 * 4);
     w.head_best = (float4*)take(G * pk::MAX_ROWS * sizeof(float4));
-    w.flags = (int*)take(pk::N_FLAGS * G * sizeof(int));
+    w.flags = (int*)take(pk::N_FLAGS * (G + 32) * sizeof(int));
     w.ctl = (pk::Ctl*)take(256);
     w.wmaps = (CUtensorMap*)take(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS * sizeof(CUtensorMap));
     w.jobs = (pk::Job*)take(((size_t)c.L + 4) * sizeof(pk::Job));
@@ -667,7 +667,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   CUDA_TRY(cudaMemcpyAsync(ws.jobs, ctx->e_jobs.data(), ctx->e_jobs.size() * sizeof(pk::Job),
                            cudaMemcpyHostToDevice, ctx->stream));
   CUDA_TRY(cudaMemsetAsync(ws.ctl, 0, 4, ctx->stream));  // abort flag; the status word is sticky
-  CUDA_TRY(cudaMemsetAsync(ws.flags, 0, (size_t)pk::N_FLAGS * ctx->e_G * sizeof(int), ctx->stream));
+  CUDA_TRY(cudaMemsetAsync(ws.flags, 0, (size_t)pk::N_FLAGS * (ctx->e_G + 32) * sizeof(int), ctx->stream));
 
   pk::Params P{};
   P.c.L = c.L; P.c.d = d; P.c.qd = qd; P.c.kvd = c.n_kv_heads * c.head_dim; P.c.hd = c.head_dim;
@@ -711,16 +711,32 @@ pk::Job layer_job(clasp_ctx* ctx, int l, int S, int T, int C, bool uniform, cons
   return J;
 }
 
-// fills in where each job's first operand comes from (the step of the previous job that wrote it)
+// fills in, per job, how often each step kind has been published once the job's own step of
+// that kind is done, and which step of the previous job publishes the job's first operand
 void link_jobs(std::vector<pk::Job>& jobs) {
+  int n_pub[pk::N_FLAGS] = {0};
   for (size_t k = 0; k < jobs.size(); ++k) {
     pk::Job& J = jobs[k];
-    if (J.type == pk::JOB_SELECT) continue;
-    if (J.type == pk::JOB_LAYER && J.prep) { J.src_flag = pk::F_PREP; J.src_epoch = (int)k + 1; continue; }
-    const pk::Job& prev = jobs[k - 1];
-    const bool from_select = prev.type == pk::JOB_SELECT || (prev.type == pk::JOB_LAYER && prev.dp);
-    J.src_flag = from_select ? pk::F_SELECT : pk::F_DOWN;
-    J.src_epoch = (int)k;
+    int src_tgt = 0, src_flag = pk::F_PREP;
+    if (k > 0) {
+      const pk::Job& prev = jobs[k - 1];
+      const bool from_select = prev.type == pk::JOB_SELECT || (prev.type == pk::JOB_LAYER && prev.dp);
+      src_flag = from_select ? pk::F_SELECT : pk::F_DOWN;
+      src_tgt = n_pub[src_flag];
+    }
+    if (J.type == pk::JOB_LAYER) {
+      if (J.prep) ++n_pub[pk::F_PREP];
+      ++n_pub[pk::F_QKV]; ++n_pub[pk::F_ATTN]; ++n_pub[pk::F_MERGE]; ++n_pub[pk::F_O]; ++n_pub[pk::F_GU];
+      ++n_pub[pk::F_DOWN];
+      if (J.dp) ++n_pub[pk::F_SELECT];
+      if (J.prep) { src_flag = pk::F_PREP; src_tgt = n_pub[pk::F_PREP]; }
+    } else if (J.type == pk::JOB_SELECT) {
+      ++n_pub[pk::F_DOWN]; ++n_pub[pk::F_SELECT];
+    } else {
+      ++n_pub[pk::F_HEAD];
+    }
+    J.src_flag = src_flag; J.src_tgt = src_tgt;
+    for (int f = 0; f < pk::N_FLAGS; ++f) J.tgt[f] = n_pub[f];
   }
 }
 

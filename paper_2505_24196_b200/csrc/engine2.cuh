@@ -21,9 +21,10 @@
 //   warp 3      allocates / frees tensor memory.
 //   warps 4-11  "workers": epilogues, attention, Eq. 2 select, arg-max.
 //
-// Synchronisation between CTAs is by epoch flags in global memory: after finishing step s of
-// job j a CTA stores j+1 to flag[s][cta] (release); a consumer polls the flags of exactly the
-// CTAs whose output it needs (acquire).  RMSNorm is applied as (x * w) W^T * rsqrt(mean(x^2) +
+// Synchronisation between CTAs is through global memory: after finishing step s of job j a
+// CTA stores j+1 to flag[s][cta] (release) and adds one to the arrival counter of step s.  A
+// consumer that needs a few specific producers (attention) polls their flags; one that needs
+// all of them (the operand of a product, the Eq. 2 decision) polls the counter once.  RMSNorm is applied as (x * w) W^T * rsqrt(mean(x^2) +
 // eps): the operand is x * w rounded to bf16, the per-row factor multiplies the product later.
 //
 // Every wait (mbarrier, flag) is bounded: when one runs out the CTA raises an abort flag that
@@ -107,7 +108,7 @@ struct Bufs {
   float* ss_m;     // [G, Rcap] (MLP norm)
   float* cosp;     // [G, Rcap + MAX_ROWS, 5] partial dot products of Eq. 2
   float4* head_best;  // [G, MAX_ROWS] (max, index bits, sum exp, -)
-  int* flags;      // [N_FLAGS, G]
+  int* flags;      // [N_FLAGS, G] epoch flags, followed by N_FLAGS arrival counters 32 ints apart
   const float2* rope;  // [T, hd/2] (cos, sin) of the rows' positions
 };
 
@@ -126,8 +127,9 @@ struct Job {
   int prep;      // 1: build the first operand from x_in when the job starts
   int dp;        // 1: the layer output feeds the Eq. 2 step below
   int row_off;   // JOB_HEAD: first row (of the previous job's rows) that goes through the head
-  int src_flag;  // flag kind that publishes this job's first operand (F_PREP / F_DOWN / F_SELECT)
-  int src_epoch;
+  int src_flag;  // step kind that publishes this job's first operand (F_PREP / F_DOWN / F_SELECT)
+  int src_tgt;   // how often every CTA has published that step once the operand is complete
+  int tgt[N_FLAGS];  // how often every CTA has published each step kind when this job's step is done
   const float* x_in;
   long long ldx;
   float* x_out;
@@ -235,6 +237,7 @@ struct Shared {
   int flag;                 // broadcast of a one-thread decision to the workers
   float rs[MAX_ROWS];       // per-row norm factors of the current product
   int choice[MAX_ROWS + 2];
+  int foot[NB];             // warp 0: ring pages each item in flight gives back when it retires
 };
 // The workers' scratch area holds either the attention K/V tiles or, during epilogues and the
 // Eq. 2 step, the cross-warp reduction tables below (the two uses never overlap in time).
@@ -284,6 +287,12 @@ __device__ __forceinline__ bool wait_flag(const int* flag, int epoch, Ctl* ctl, 
   }
   raise_abort(ctl, sh, true);
   return false;
+}
+
+// Bounded wait until all G CTAs have published step `kind` `tgt` times.
+__device__ __forceinline__ bool wait_count(const Params& p, int kind, int tgt, Shared* sh) {
+  const int* cnt = p.b.flags + N_FLAGS * p.c.G + kind * 32;
+  return wait_flag(cnt, tgt * p.c.G, p.ctl, sh);
 }
 
 // ------------------------------------------------------------------ the schedule every role walks
@@ -350,7 +359,7 @@ __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base) {
   RingPos rp{0, 0};
   int used = 0;
   uint32_t tail = 0;
-  int foot[NB];
+  int* foot = sh->foot;
   const int b_pages = (c.BN * BK * 2) / PAGE;
   for (int jb = 0; jb < p.n_jobs; ++jb) {
     const Job& J = p.jobs[jb];
@@ -431,19 +440,15 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
       Phase P;
       P.init(p, J, ph);
       if (P.n_tiles == 0) continue;
-      // where this product's operand columns come from
-      int fkind, split, epoch, bmap;
-      if (P.kind == G_QKV) { fkind = J.src_flag; split = S_D; epoch = J.src_epoch; bmap = 0; }
-      else if (P.kind == G_O) { fkind = F_MERGE; split = -1; epoch = jb + 1; bmap = 1; }
-      else if (P.kind == G_GU) { fkind = F_O; split = S_D; epoch = jb + 1; bmap = 2; }
-      else if (P.kind == G_DOWN) { fkind = F_GU; split = S_F; epoch = jb + 1; bmap = 3; }
-      else { fkind = J.src_flag; split = S_D; epoch = J.src_epoch; bmap = 4; }
-      const int* flags = p.b.flags + fkind * c.G;
-      const int units = split >= 0 ? c.split_units[split] : 1;
-      const int Ktot = kind_K(c, P.kind);
-      uint32_t vmask[MAX_CTAS / 32];  // producers whose flag has been seen
-#pragma unroll
-      for (int w = 0; w < MAX_CTAS / 32; ++w) vmask[w] = 0u;
+      // the operand exists once every CTA has published the step that writes it
+      int fkind, tgt, bmap;
+      if (P.kind == G_QKV) { fkind = J.src_flag; tgt = J.src_tgt; bmap = 0; }
+      else if (P.kind == G_O) { fkind = F_MERGE; tgt = J.tgt[F_MERGE]; bmap = 1; }
+      else if (P.kind == G_GU) { fkind = F_O; tgt = J.tgt[F_O]; bmap = 2; }
+      else if (P.kind == G_DOWN) { fkind = F_GU; tgt = J.tgt[F_GU]; bmap = 3; }
+      else { fkind = J.src_flag; tgt = J.src_tgt; bmap = 4; }
+      if (!wait_count(p, fkind, tgt, sh)) return;
+      fence_proxy_async();  // the producers' ordinary stores before this thread's TMA reads
       for (int t = 0; t < P.n_tiles; ++t) {
         const TileDesc td = tiles[P.tile0 + t];
         const int a_pages = td.n_rows >> 3;
@@ -464,20 +469,6 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
           }
           if (!ok) { raise_abort(p.ctl, sh, true); return; }
           const int k0 = P.group_at(gi) * P.kpi, k1 = min(P.kc, k0 + P.kpi);
-          // operand columns [k0*64, k1*64) must have been published by the CTAs that own them
-          int o_first, o_last;
-          const int col0 = k0 * BK, col1 = min(k1 * BK, Ktot) - 1;
-          if (split >= 0) { o_first = owner_of(units, c.G, col0); o_last = owner_of(units, c.G, col1); }
-          else { o_first = col0 / c.hd; o_last = col1 / c.hd; }   // head h is merged by CTA h % G
-          bool fresh = false;
-          for (int o = o_first; o <= o_last; ++o) {
-            const int cc = split >= 0 ? o : o % c.G;
-            if ((vmask[cc >> 5] >> (cc & 31)) & 1u) continue;
-            if (!wait_flag(flags + cc, epoch, p.ctl, sh)) return;
-            vmask[cc >> 5] |= 1u << (cc & 31);
-            fresh = true;
-          }
-          if (fresh) fence_proxy_async();  // the producers' ordinary stores before this thread's TMA reads
           const uint32_t full = tc::smem_u32(&sh->full[it % NB]);
           tc::mbar_expect_tx(full, (uint32_t)(k1 - k0) * b_bytes);
           for (int k = k0; k < k1; ++k)
@@ -568,7 +559,14 @@ struct Worker {
     if (wtid == 0) {
       __threadfence();
       st_release_i32(p.b.flags + kind * p.c.G + blockIdx.x, epoch);
+      atomicAdd(p.b.flags + N_FLAGS * p.c.G + kind * 32, 1);
     }
+  }
+  // every CTA has published step `kind` tgt times: one thread polls, the others wait for it
+  __device__ bool wait_all(int kind, int tgt) {
+    bool ok = true;
+    if (wtid == 0) ok = wait_count(p, kind, tgt, sh);
+    return worker_and(ok);
   }
   // wait for flags [first, first + n) of `kind`: one flag per thread
   __device__ bool wait_flags(int kind, int first, int n, int epoch) {
@@ -831,7 +829,7 @@ struct Worker {
     }
     publish(F_DOWN, jb + 1);
     // (2) every CTA's partials, added in CTA order by a fixed shuffle tree
-    if (!wait_flags(F_DOWN, 0, c.G, jb + 1)) return false;
+    if (!wait_all(F_DOWN, J.tgt[F_DOWN])) return false;
     for (int r = ww; r < rows; r += 8) {
       double v[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
       for (int cc = lane; cc < c.G; cc += 32) {
@@ -1240,7 +1238,7 @@ struct Worker {
     const Cfg& c = p.c;
     publish(F_HEAD, jb + 1);
     if (blockIdx.x != 0) return true;
-    if (!wait_flags(F_HEAD, 0, c.G, jb + 1)) return false;
+    if (!wait_all(F_HEAD, J.tgt[F_HEAD])) return false;
     const int* vlo = split_lo(S_V);
     for (int r = ww; r < J.R; r += 8) {
       float best = -INFINITY;

@@ -63,6 +63,9 @@ enum { G_QKV = 0, G_O = 1, G_GU = 2, G_DOWN = 3, G_HEAD = 4 };
 enum { S_QKV = 0, S_D = 1, S_F = 2, S_V = 3, N_SPLITS = 4 };
 // flag kinds
 enum { F_PREP = 0, F_QKV, F_ATTN, F_MERGE, F_O, F_GU, F_DOWN, F_SELECT, F_HEAD, N_FLAGS };
+// trace slots of a job (time stamps of the workers' step boundaries)
+enum { T_START = 0, T_QKV, T_ATT_READY, T_ATT_Q, T_ATT_TILES, T_ATT_PUB, T_MERGE, T_O, T_GU, T_DOWN, T_DP_PUB,
+       T_DP_ALL, T_DP_DECIDED, T_DP_DONE, T_HEAD };
 
 struct TileDesc {      // one accumulator's worth of a CTA's feature range
   int f0;              // first feature in the product's feature space
@@ -238,6 +241,7 @@ struct Shared {
   float rs[MAX_ROWS];       // per-row norm factors of the current product
   int choice[MAX_ROWS + 2];
   int foot[NB];             // warp 0: ring pages each item in flight gives back when it retires
+  int job_words[(sizeof(Job) + 3) / 4];  // the workers' copy of the current job descriptor
 };
 // The workers' scratch area holds either the attention K/V tiles or, during epilogues and the
 // Eq. 2 step, the cross-warp reduction tables below (the two uses never overlap in time).
@@ -544,13 +548,14 @@ struct Worker {
   uint32_t n_acc;
   int n_mark;
 
-  __device__ __forceinline__ void mark() {
-    if (p.trace != nullptr && wtid == 0 && n_mark < p.trace_cap) {
+  // time stamp of step `slot` (one of the T_* below) of the current job: 16 slots per job
+  __device__ __forceinline__ void mark(int slot) {
+    const int idx = n_mark * 16 + slot;
+    if (p.trace != nullptr && wtid == 0 && idx < p.trace_cap) {
       unsigned long long t;
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-      p.trace[(long long)blockIdx.x * p.trace_cap + n_mark] = t;
+      p.trace[(long long)blockIdx.x * p.trace_cap + idx] = t;
     }
-    ++n_mark;
   }
 
   // all workers' stores of this step become visible, then the CTA's flag of `kind` says so
@@ -618,15 +623,35 @@ struct Worker {
   // Thread (quarter q, lane) owns feature td.f0 + 32 q + lane; the two warps of a quarter take
   // alternating blocks of 16 rows (accumulator columns).  Per-row sums over the CTA's features
   // (sums of squares, cosine partials, arg-max) go through RedTables: one entry per (quarter, row).
-  __device__ bool epilogue(const Job& J, const Phase& P, const TileDesc& td, int tile_no) {
+  // For the down product of an Eq. 2 job the thread's layer outputs (keep_y) and skip candidates
+  // (keep_s) of its first block of 16 rows stay in registers for dp_step.
+  __device__ bool epilogue(const Job& J, const Phase& P, const TileDesc& td, int tile_no, float (&keep_y)[16],
+                           float (&keep_s)[16]) {
     const Cfg& c = p.c;
     RedTables* T = tables();
     const int quarter = ww & 3, group = ww >> 2;
     const int fl = quarter * 32 + lane;
     const bool fv = fl < td.n_rows;
     const int f = td.f0 + fl;
-    const int ncb = (J.R + 15) >> 4;
+    const bool dpd = P.kind == G_DOWN && J.dp;
+    const int rows_all = J.R + ((dpd && J.diag) ? J.T : 0);   // Eq. 2: plus the rows of the diagonal state
+    const int ncb = (rows_all + 15) >> 4;
     const bool resid = P.kind == G_O || P.kind == G_DOWN;
+    // Eq. 2: objective row and skip candidate of every row of the first block, fetched early
+    float xi[16];
+    if (dpd) {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int r = group * 16 + k;
+        xi[k] = 0.f;
+        keep_s[k] = 0.f;
+        keep_y[k] = 0.f;
+        if (fv && r < rows_all) {
+          xi[k] = __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f);
+          keep_s[k] = __ldcg(skip_src(J, r / J.T + 1, r % J.T) + f);
+        }
+      }
+    }
     // residual rows of the first block are fetched before the accumulator is ready
     float res[16];
 #pragma unroll
@@ -697,27 +722,52 @@ struct Worker {
             }
           }
         }
+      } else if (dpd) {
+        // candidate states: layer output y, skip candidate sv; five partial dot products per row
+        float sv[16];
+        if (cb != group) {
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            const int r = cb * 16 + k;
+            xi[k] = 0.f;
+            sv[k] = 0.f;
+            if (fv && r < rows_all) {
+              xi[k] = __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f);
+              sv[k] = __ldcg(skip_src(J, r / J.T + 1, r % J.T) + f);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 16; ++k) sv[k] = keep_s[k];
+        }
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          if (r < rows_all) {
+            const float y = (fv && r < J.R) ? res[k] + v[k] : 0.f;
+            if (fv && r < J.R) __stcg(p.b.Gbuf + (long long)r * c.d + f, y);
+            if (cb == group) keep_y[k] = y;
+            const float s0 = warp_sum(xi[k] * y), s1 = warp_sum(y * y), s2 = warp_sum(xi[k] * sv[k]);
+            const float s3 = warp_sum(sv[k] * sv[k]), s4 = warp_sum(xi[k] * xi[k]);
+            if (lane == 0) {
+              float* dst = T->red[quarter][r];
+              dst[0] = s0; dst[1] = s1; dst[2] = s2; dst[3] = s3; dst[4] = s4;
+            }
+          }
+        }
       } else if (P.kind == G_DOWN) {
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
           const int r = cb * 16 + k;
           if (r >= J.R) break;
           const float y = fv ? res[k] + v[k] : 0.f;
-          if (J.dp) {
-            // candidate state's layer output + its cosine partials  x_i . y  and  y . y
-            if (fv) __stcg(p.b.Gbuf + (long long)r * c.d + f, y);
-            const float xi = fv ? __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f) : 0.f;
-            const float a = warp_sum(xi * y), b2 = warp_sum(y * y);
-            if (lane == 0) { T->red[quarter][r][0] = a; T->red[quarter][r][1] = b2; }
-          } else {
-            if (fv) {
-              __stcg(J.x_out + r * J.ldo + f, y);
-              if (J.norm_next) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
-            }
-            if (J.norm_next) {
-              const float s2 = warp_sum(y * y);
-              if (lane == 0) T->red[quarter][r][0] = s2;
-            }
+          if (fv) {
+            __stcg(J.x_out + r * J.ldo + f, y);
+            if (J.norm_next) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
+          }
+          if (J.norm_next) {
+            const float s2 = warp_sum(y * y);
+            if (lane == 0) T->red[quarter][r][0] = s2;
           }
         }
       } else {  // G_HEAD: best logit of this tile per row (lowest index on ties) and sum of exp
@@ -789,12 +839,13 @@ struct Worker {
   }
 
   // ---- Eq. 2 step i over this CTA's slice of the d features (thread <-> feature as in the
-  // epilogue, so a thread meets again the layer outputs it stored itself):
+  // epilogue):
   //   (1) per-CTA partial dot products -> cosp, publish;
   //   (2) wait for every CTA, add the partials in CTA order, decide (every CTA decides alike);
   //   (3) write this CTA's slice of g[i][.] and of the next step's operand, publish.
-  // have_apply: the epilogue left the apply candidates' partials in the tables.
-  __device__ bool dp_step(const Job& J, int jb, bool have_apply) {
+  // from_epilogue: the down product's epilogue left the partials of this CTA in the tables and
+  // the thread's layer outputs / skip candidates of its first row block in keep_y / keep_s.
+  __device__ bool dp_step(const Job& J, int jb, bool from_epilogue, float (&keep_y)[16], float (&keep_s)[16]) {
     const Cfg& c = p.c;
     RedTables* T = tables();
     const int f_lo = __ldg(split_lo(S_D) + blockIdx.x), f_hi = __ldg(split_lo(S_D) + blockIdx.x + 1);
@@ -806,19 +857,31 @@ struct Worker {
     const int rows = n_states * J.T;
     const int ncb = (rows + 15) >> 4;
     const long long cstride = (long long)(c.Rcap + MAX_ROWS) * 5;
-    // (1) skip candidates (rows of every state 1..n_states)
-    for (int cb = group; cb < ncb; cb += 2) {
+    if (!from_epilogue) {
+      // (1) no layer ran for this CTA's features: only skip candidates exist
+      for (int cb = group; cb < ncb; cb += 2) {
+        float xi[16], sv[16];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        const int r = cb * 16 + k;
-        if (r >= rows) break;
-        const int j = r / J.T + 1, t = r % J.T;
-        const float xi = fv ? __ldg(J.x_i + t * J.x_tok_stride + f) : 0.f;
-        const float sv = fv ? __ldcg(skip_src(J, j, t) + f) : 0.f;
-        const float a = warp_sum(xi * sv), b2 = warp_sum(sv * sv), x2 = warp_sum(xi * xi);
-        if (lane == 0) {
-          T->red[quarter][r][2] = a; T->red[quarter][r][3] = b2; T->red[quarter][r][4] = x2;
-          if (!(have_apply && r < J.ell * J.T)) { T->red[quarter][r][0] = 0.f; T->red[quarter][r][1] = 0.f; }
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          xi[k] = 0.f;
+          sv[k] = 0.f;
+          if (fv && r < rows) {
+            xi[k] = __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f);
+            sv[k] = __ldcg(skip_src(J, r / J.T + 1, r % J.T) + f);
+          }
+          if (cb == group) { keep_s[k] = sv[k]; keep_y[k] = 0.f; }
+        }
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          if (r < rows) {
+            const float s2 = warp_sum(xi[k] * sv[k]), s3 = warp_sum(sv[k] * sv[k]), s4 = warp_sum(xi[k] * xi[k]);
+            if (lane == 0) {
+              float* dst = T->red[quarter][r];
+              dst[0] = 0.f; dst[1] = 0.f; dst[2] = s2; dst[3] = s3; dst[4] = s4;
+            }
+          }
         }
       }
     }
@@ -828,8 +891,10 @@ struct Worker {
       __stcg(p.b.cosp + blockIdx.x * cstride + idx, T->red[0][r][k] + T->red[1][r][k] + T->red[2][r][k] + T->red[3][r][k]);
     }
     publish(F_DOWN, jb + 1);
+    mark(T_DP_PUB);
     // (2) every CTA's partials, added in CTA order by a fixed shuffle tree
     if (!wait_all(F_DOWN, J.tgt[F_DOWN])) return false;
+    mark(T_DP_ALL);
     for (int r = ww; r < rows; r += 8) {
       double v[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
       for (int cc = lane; cc < c.G; cc += 32) {
@@ -874,24 +939,36 @@ struct Worker {
       J.choice[0] = 0;
     }
     worker_sync();
-    // (3) write-back
+    mark(T_DP_DECIDED);
+    // (3) write-back: the first block of rows comes from registers
     const float wn = (fv && J.norm_next) ? __ldg(J.norm_next + f) : 0.f;
     for (int cb = group; cb < ncb; cb += 2) {
+      float y16[16];
 #pragma unroll
       for (int k = 0; k < 16; ++k) {
         const int r = cb * 16 + k;
-        if (r >= rows) break;
-        const int j = r / J.T + 1, t = r % J.T;
-        float y = 0.f;
-        if (fv) {
-          y = sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f);
-          __stcg(J.g_next + ((long long)j * J.T + t) * c.d + f, y);
-          if (J.g_final && j == J.M) J.g_final[(long long)t * c.d + f] = y;
-          if (J.norm_next) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
+        y16[k] = 0.f;
+        if (fv && r < rows) {
+          const int j = r / J.T + 1, t = r % J.T;
+          if (cb == group) y16[k] = sh->choice[j] ? keep_y[k] : keep_s[k];
+          else y16[k] = sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f);
         }
-        if (J.norm_next) {
-          const float s2 = warp_sum(y * y);
-          if (lane == 0) T->red[quarter][r][0] = s2;
+      }
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int r = cb * 16 + k;
+        if (r < rows) {
+          const int j = r / J.T + 1, t = r % J.T;
+          const float y = y16[k];
+          if (fv) {
+            __stcg(J.g_next + ((long long)j * J.T + t) * c.d + f, y);
+            if (J.g_final && j == J.M) J.g_final[(long long)t * c.d + f] = y;
+            if (J.norm_next) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
+          }
+          if (J.norm_next) {
+            const float s2 = warp_sum(y * y);
+            if (lane == 0) T->red[quarter][r][0] = s2;
+          }
         }
       }
     }
@@ -949,6 +1026,7 @@ struct Worker {
         }
         if (!worker_and(ok)) return false;
       }
+      mark(T_ATT_READY);
       const int p0 = (pbg * 8 + ww) * 16;
       const bool active = p0 < Pn;
       int rr[2], hq[2];
@@ -986,6 +1064,7 @@ struct Worker {
           }
         }
       }
+      mark(T_ATT_Q);
       float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
       float o[NBLK][4];
 #pragma unroll
@@ -1120,6 +1199,7 @@ struct Worker {
           }
         }
       }
+      mark(T_ATT_TILES);
       if (active) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -1274,19 +1354,32 @@ struct Worker {
   __device__ bool run() {
     const Cfg& c = p.c;
     const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
+    float keep_y[16], keep_s[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) { keep_y[k] = 0.f; keep_s[k] = 0.f; }
     for (int jb = 0; jb < p.n_jobs; ++jb) {
-      const Job& J = p.jobs[jb];
-      mark();
+      // the job descriptor goes to shared memory and from there into a local copy: its fields
+      // must not look as if a store to global memory could change them
+      worker_sync();
+      {
+        const int* src = reinterpret_cast<const int*>(p.jobs + jb);
+        for (int k = wtid; k < (int)(sizeof(Job) / 4); k += WORKERS) sh->job_words[k] = __ldg(src + k);
+      }
+      worker_sync();
+      const Job J = *reinterpret_cast<const Job*>(sh->job_words);
+      n_mark = jb;
+      mark(T_START);
       if (J.type == JOB_SELECT) {
-        if (!dp_step(J, jb, false)) return false;
+        if (!dp_step(J, jb, false, keep_y, keep_s)) return false;
         continue;
       }
       if (J.type == JOB_HEAD) {
         Phase P;
         P.init(p, J, 0);
         for (int t = 0; t < P.n_tiles; ++t)
-          if (!epilogue(J, P, tiles[P.tile0 + t], t)) return false;
+          if (!epilogue(J, P, tiles[P.tile0 + t], t, keep_y, keep_s)) return false;
         if (!head_merge(J, jb)) return false;
+        mark(T_HEAD);
         continue;
       }
       attention_prefetch(J);
@@ -1295,25 +1388,25 @@ struct Worker {
         Phase P;
         P.init(p, J, ph);
         for (int t = 0; t < P.n_tiles; ++t)
-          if (!epilogue(J, P, tiles[P.tile0 + t], t)) return false;
-        mark();
+          if (!epilogue(J, P, tiles[P.tile0 + t], t, keep_y, keep_s)) return false;
+        mark(ph == G_QKV ? T_QKV : (ph == G_O ? T_O : (ph == G_GU ? T_GU : T_DOWN)));
         if (ph == G_QKV) {
           publish(F_QKV, jb + 1);
           if (!(c.hd == 128 ? attention_partials<128>(J, jb) : attention_partials<64>(J, jb))) return false;
-          mark();
+          mark(T_ATT_PUB);
           if (!(c.hd == 128 ? attention_merge<4>(J, jb) : attention_merge<2>(J, jb))) return false;
-          mark();
+          mark(T_MERGE);
         } else if (ph == G_O) {
           publish(F_O, jb + 1);
         } else if (ph == G_GU) {
           publish(F_GU, jb + 1);
         } else {
           if (J.dp) {
-            if (!dp_step(J, jb, P.n_tiles > 0)) return false;
+            if (!dp_step(J, jb, P.n_tiles > 0, keep_y, keep_s)) return false;
           } else {
             publish(F_DOWN, jb + 1);
           }
-          mark();
+          mark(T_DP_DONE);
         }
       }
     }

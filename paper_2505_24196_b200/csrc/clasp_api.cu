@@ -673,7 +673,8 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   P.c.L = c.L; P.c.d = d; P.c.qd = qd; P.c.kvd = c.n_kv_heads * c.head_dim; P.c.hd = c.head_dim;
   P.c.nq = c.n_q_heads; P.c.nkv = c.n_kv_heads; P.c.dffn = c.d_ffn; P.c.vocab = c.vocab; P.c.eps = c.rms_eps;
   P.c.G = ctx->e_G; P.c.Rcap = ws.e_rcap; P.c.run_len = ws.e_run_len; P.c.chunk_cap = ws.e_chunk_cap;
-  P.c.BN = BN; P.c.ring_pages = ring_pages;
+  P.c.BN = BN; P.c.ring_pages = ring_pages; P.c.n_iss = BN <= 64 ? 2 : 1;
+  if (getenv("CLASP_ENGINE_ONE_ISSUER")) P.c.n_iss = 1;
   for (int s = 0; s < pk::N_SPLITS; ++s) { P.c.split_lo[s] = ctx->e_split_lo[s]; P.c.split_units[s] = ctx->e_split_units[s]; }
   for (int k = 0; k < 5; ++k) { P.c.tile_idx[k] = ctx->e_tile_idx[k]; P.c.kpi[k] = kpi[k]; }
   P.c.tiles_off = ctx->e_tiles_off; P.c.loads_off = ctx->e_loads_off;

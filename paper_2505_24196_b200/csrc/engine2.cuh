@@ -15,10 +15,12 @@
 //               depend on activations: this warp runs ahead across products, layers and jobs.
 //   warp 1      lane 0 loads the activation operand ([BN x 64] bf16 per 64-column chunk) next to
 //               the weight rows once the CTAs that produce those columns have published them.
-//   warp 2      lane 0 issues tcgen05.mma: M = 128 weight rows (rows beyond the CTA's range are
-//               whatever bytes follow in the ring; their accumulator lanes are never read),
-//               N = BN activation rows, K = 16, two accumulators in tensor memory.
-//   warp 3      allocates / frees tensor memory.
+//   warps 2, 3  lane 0 of each issues tcgen05.mma: M = 128 weight rows (rows beyond the CTA's
+//               range are whatever bytes follow in the ring; their accumulator lanes are never
+//               read), N = BN activation rows, K = 16.  One thread can issue an MMA only every
+//               ~55 cycles while the tensor pipe takes ~39 for this shape, so the two warps take
+//               alternate ring items and accumulate into separate accumulators, which the
+//               epilogue adds in a fixed order.  Warp 3 also allocates / frees tensor memory.
 //   warps 4-11  "workers": epilogues, attention, Eq. 2 select, arg-max.
 //
 // Synchronisation between CTAs is through global memory: after finishing step s of job j a
@@ -88,6 +90,8 @@ struct Cfg {
   int run_len, chunk_cap;
   int BN;              // activation rows padded to a multiple of 16 (MMA N)
   int ring_pages;
+  int n_iss;           // MMA issuers in use: 2 while two accumulators of (gate, up) x BN columns fit one
+                       // 256-column buffer (BN <= 64), else 1
   // tables (ints / structs in Params::tabs, offsets in ints)
   int split_lo[N_SPLITS];    // [G + 1] first feature of each CTA: lo(c) = 8 floor(c units / G)
   int split_units[N_SPLITS]; // 8-feature units of each split
@@ -230,6 +234,40 @@ __device__ __forceinline__ uint2 pack4(float a, float b, float c2, float d2) {
   return u;
 }
 
+// tcgen05.mma with the operand descriptors given by their low words (start address and leading
+// byte offset; the high word -- 1024-byte group stride, version, 128B swizzle -- is the same for
+// every tile).  A thread issues thousands of these per layer, so nothing else is in the asm.
+constexpr uint32_t DESC_HI = 64u | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+template <bool ACC>
+__device__ __forceinline__ void mma_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+  if (ACC) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.eq.u32 p, 1, 1;\n\t"
+        "mov.b64 da, {%1, %4};\n\t"
+        "mov.b64 db, {%2, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI));
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.eq.u32 p, 1, 0;\n\t"
+        "mov.b64 da, {%1, %4};\n\t"
+        "mov.b64 db, {%2, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI));
+  }
+}
+// the four K = 16 steps of one 64-column chunk
+template <bool FIRST>
+__device__ __forceinline__ void mma_chunk(uint32_t acc, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+  mma_lo<!FIRST>(acc, a_lo, b_lo, idesc);
+  mma_lo<true>(acc, a_lo + 2, b_lo + 2, idesc);
+  mma_lo<true>(acc, a_lo + 4, b_lo + 4, idesc);
+  mma_lo<true>(acc, a_lo + 6, b_lo + 6, idesc);
+}
+
 // ------------------------------------------------------------------ shared state
 struct Shared {
   uint64_t full[NB], empty[NB];
@@ -354,7 +392,10 @@ struct RingPos {
   }
 };
 
-__device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base) {
+// Warp 0, all lanes: every lane walks the schedule; lane 0 does the ring bookkeeping and each
+// lane issues at most one of an item's TMA boxes, so that all boxes of an item leave in one
+// instruction (a single thread can only issue a TMA every few hundred cycles).
+__device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base, int lane) {
   const Cfg& c = p.c;
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
@@ -376,47 +417,42 @@ __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base) {
         const int a_pages = td.n_rows >> 3;
         const int chunk_pages = (P.dual + 1) * a_pages + b_pages;
         const int pages = P.kpi * chunk_pages;
-        // the tile's load list, fetched once: (row offset in bytes, map, first matrix row)
-        uint32_t l_off[MAX_TILE_LOADS];
-        int l_map[MAX_TILE_LOADS], l_y[MAX_TILE_LOADS];
-#pragma unroll
-        for (int l = 0; l < MAX_TILE_LOADS; ++l) {
-          l_off[l] = 0; l_map[l] = 0; l_y[l] = 0;
-          if (l < td.n_loads) {
-            const LoadDesc ld = loads[td.load0 + l];
-            l_off[l] = (uint32_t)ld.row_off * 128u; l_map[l] = P.map_base + ld.map_local; l_y[l] = ld.y0;
-          }
-        }
+        // boxes of one chunk: n_loads (x2 with the "up" matrix); lane l issues box l % per_chunk of
+        // chunk l / per_chunk.  Its load descriptor is fixed for the whole tile.
+        const int per_chunk = td.n_loads * (P.dual + 1);
+        const int my_box = lane % per_chunk, my_chunk = lane / per_chunk;
+        const int my_half = my_box / td.n_loads;
+        const LoadDesc ld = loads[td.load0 + my_box % td.n_loads];
+        const uint32_t my_off = (uint32_t)(my_half * a_pages * PAGE) + (uint32_t)ld.row_off * 128u;
+        const CUtensorMap* my_map = p.wmaps + P.map_base + my_half * N_HEIGHTS + ld.map_local;
         for (int gi = 0; gi < P.n_groups; ++gi) {
           // make room: items leave the ring in the order they entered it
           int fp;
           RingPos probe = rp;
           probe.place(pages, c.ring_pages, fp);
           while (used + fp > c.ring_pages || rp.item - tail >= (uint32_t)NB) {
-            if (!wait_bar(&sh->empty[tail % NB], (tail / NB) & 1u, p.ctl, sh)) return;
+            const bool ok = wait_bar(&sh->empty[tail % NB], (tail / NB) & 1u, p.ctl, sh);
+            if (!__all_sync(0xffffffffu, ok)) return;
             used -= foot[tail % NB];
             ++tail;
           }
           const uint32_t it = rp.item;
           const int at = rp.place(pages, c.ring_pages, fp);
-          foot[it % NB] = fp;
+          __syncwarp();
+          if (lane == 0) foot[it % NB] = fp;
           used += fp;
-          const int k0 = P.group_at(gi) * P.kpi, k1 = min(P.kc, k0 + P.kpi);
+          const int k0 = P.group_at(gi) * P.kpi, nk = min(P.kc, k0 + P.kpi) - k0;
           const uint32_t full = tc::smem_u32(&sh->full[it % NB]);
-          tc::mbar_expect_tx(full, (uint32_t)((k1 - k0) * (P.dual + 1) * a_pages * PAGE));
-          for (int k = k0; k < k1; ++k) {
-            const uint32_t dst = ring_base + (uint32_t)(at + (k - k0) * chunk_pages) * PAGE;
-#pragma unroll
-            for (int l = 0; l < MAX_TILE_LOADS; ++l) {
-              if (l < td.n_loads) {
-                tc::tma_load_2d(dst + l_off[l], p.wmaps + l_map[l], full, k * BK, l_y[l], pol);
-                if (P.dual)  // the "up" rows of the same features follow the "gate" rows
-                  tc::tma_load_2d(dst + (uint32_t)(a_pages * PAGE) + l_off[l], p.wmaps + l_map[l] + N_HEIGHTS, full,
-                                  k * BK, l_y[l], pol);
-              }
-            }
+          if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)(nk * (P.dual + 1) * a_pages * PAGE));
+          __syncwarp();
+          for (int base = 0; base < nk; base += 32 / per_chunk) {   // one pass unless an item has > 32 boxes
+            const int kk = base + my_chunk;
+            if (my_chunk < 32 / per_chunk && kk < nk)
+              tc::tma_load_2d(ring_base + (uint32_t)(at + kk * chunk_pages) * PAGE + my_off, my_map, full, (k0 + kk) * BK,
+                              ld.y0, pol);
           }
-          sh->a_issued = (int)(it + 1);
+          __syncwarp();
+          if (lane == 0) sh->a_issued = (int)(it + 1);
         }
       }
     }
@@ -429,7 +465,8 @@ __device__ __forceinline__ int owner_of(int units, int G, int f) {
   return (((f >> 3) + 1) * G - 1) / units;
 }
 
-__device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, const CUtensorMap* const* bmaps) {
+// Warp 1, all lanes: lane k issues the operand tile of an item's chunk k.
+__device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, const CUtensorMap* const* bmaps, int lane) {
   const Cfg& c = p.c;
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
@@ -451,8 +488,12 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
       else if (P.kind == G_GU) { fkind = F_O; tgt = J.tgt[F_O]; bmap = 2; }
       else if (P.kind == G_DOWN) { fkind = F_GU; tgt = J.tgt[F_GU]; bmap = 3; }
       else { fkind = J.src_flag; tgt = J.src_tgt; bmap = 4; }
-      if (!wait_count(p, fkind, tgt, sh)) return;
-      fence_proxy_async();  // the producers' ordinary stores before this thread's TMA reads
+      {
+        bool ok = true;
+        if (lane == 0) ok = wait_count(p, fkind, tgt, sh);
+        if (!__all_sync(0xffffffffu, ok)) return;
+      }
+      fence_proxy_async();  // the producers' ordinary stores before this warp's TMA reads
       for (int t = 0; t < P.n_tiles; ++t) {
         const TileDesc td = tiles[P.tile0 + t];
         const int a_pages = td.n_rows >> 3;
@@ -467,24 +508,30 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
           for (uint32_t w = 0; w < WAIT_SLOW; ++w) {
             if ((uint32_t)sh->a_issued > it) { ok = true; break; }
             if (w > WAIT_FAST) {
-              if (aborted(p.ctl, sh)) return;
+              if (aborted(p.ctl, sh)) break;
               __nanosleep(100);
             }
           }
-          if (!ok) { raise_abort(p.ctl, sh, true); return; }
-          const int k0 = P.group_at(gi) * P.kpi, k1 = min(P.kc, k0 + P.kpi);
+          if (!ok && !aborted(p.ctl, sh)) raise_abort(p.ctl, sh, true);
+          if (!__all_sync(0xffffffffu, ok)) return;
+          const int k0 = P.group_at(gi) * P.kpi, nk = min(P.kc, k0 + P.kpi) - k0;
           const uint32_t full = tc::smem_u32(&sh->full[it % NB]);
-          tc::mbar_expect_tx(full, (uint32_t)(k1 - k0) * b_bytes);
-          for (int k = k0; k < k1; ++k)
-            tc::tma_load_2d(ring_base + (uint32_t)(at + (k - k0) * chunk_pages + (P.dual + 1) * a_pages) * PAGE,
-                            bmaps[bmap], full, k * BK, 0, pol);
+          if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)nk * b_bytes);
+          __syncwarp();
+          if (lane < nk)
+            tc::tma_load_2d(ring_base + (uint32_t)(at + lane * chunk_pages + (P.dual + 1) * a_pages) * PAGE, bmaps[bmap],
+                            full, (k0 + lane) * BK, 0, pol);
+          __syncwarp();
         }
       }
     }
   }
 }
 
-__device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint32_t tmem_base) {
+// MMA issuer `which` (0 or 1) takes the ring items of each tile with that parity and adds them up
+// in accumulator `which` of the tile's buffer: buffer b holds accumulator a at column
+// b * 256 + a * (dual + 1) * BN  (gate at +0, up at +BN).
+__device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint32_t tmem_base, int which) {
   const Cfg& c = p.c;
   const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.BN >> 3) << 17) | (8u << 24);
   const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
@@ -505,33 +552,43 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
         const uint32_t buf = n_acc & 1u;
         if (!wait_bar(&sh->acc_empty[buf], ((n_acc >> 1) & 1u) ^ 1u, p.ctl, sh)) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t acc = tmem_base + buf * 256u;
-        bool first = true;
+        const uint32_t acc = tmem_base + buf * 256u + (uint32_t)(which * (P.dual + 1) * c.BN);
+        const uint32_t acc2 = acc + (uint32_t)c.BN;
+        const uint32_t up_lo = (uint32_t)a_pages * (PAGE / 16);                  // gate rows -> up rows
+        const uint32_t b_off = (uint32_t)((P.dual + 1) * a_pages) * (PAGE / 16);  // weight rows -> operand tile
+        const uint32_t chunk_lo = (uint32_t)chunk_pages * (PAGE / 16);
         for (int gi = 0; gi < P.n_groups; ++gi) {
           int fp;
           const uint32_t it = rp.item;
           const int at = rp.place(pages, c.ring_pages, fp);
+          if ((gi & (c.n_iss - 1)) != which) continue;
           if (!wait_bar(&sh->full[it % NB], (it / NB) & 1u, p.ctl, sh)) return;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const int k0 = P.group_at(gi) * P.kpi, k1 = min(P.kc, k0 + P.kpi);
-          for (int k = k0; k < k1; ++k) {
-            const uint32_t sa = ring_base + (uint32_t)(at + (k - k0) * chunk_pages) * PAGE;
-            const uint32_t sb = sa + (uint32_t)((P.dual + 1) * a_pages) * PAGE;
-            const uint64_t da = tc::make_smem_desc(sa), db = tc::make_smem_desc(sb);
-#pragma unroll
-            for (int kk = 0; kk < BK / 16; ++kk)
-              tc::mma_bf16(acc, da + 2 * kk, db + 2 * kk, idesc, (first && kk == 0) ? 0u : 1u);
-            if (P.dual) {
-              const uint64_t da2 = tc::make_smem_desc(sa + (uint32_t)a_pages * PAGE);
-#pragma unroll
-              for (int kk = 0; kk < BK / 16; ++kk)
-                tc::mma_bf16(acc + (uint32_t)c.BN, da2 + 2 * kk, db + 2 * kk, idesc, (first && kk == 0) ? 0u : 1u);
+          const int k0 = P.group_at(gi) * P.kpi;
+          const int nk = min(P.kc, k0 + P.kpi) - k0;
+          uint32_t a_lo = desc_lo(ring_base + (uint32_t)at * PAGE);
+          int k = 0;
+          if (gi < c.n_iss) {  // this issuer's first item of the tile overwrites its accumulator
+            mma_chunk<true>(acc, a_lo, a_lo + b_off, idesc);
+            if (P.dual) mma_chunk<true>(acc2, a_lo + up_lo, a_lo + b_off, idesc);
+            a_lo += chunk_lo;
+            k = 1;
+          }
+          if (P.dual) {
+            for (; k < nk; ++k) {
+              mma_chunk<false>(acc, a_lo, a_lo + b_off, idesc);
+              mma_chunk<false>(acc2, a_lo + up_lo, a_lo + b_off, idesc);
+              a_lo += chunk_lo;
             }
-            first = false;
+          } else {
+            for (; k < nk; ++k) {
+              mma_chunk<false>(acc, a_lo, a_lo + b_off, idesc);
+              a_lo += chunk_lo;
+            }
           }
           tc::mma_commit(tc::smem_u32(&sh->empty[it % NB]));
         }
-        tc::mma_commit(tc::smem_u32(&sh->acc_full[buf]));
+        tc::mma_commit(tc::smem_u32(&sh->acc_full[buf]));  // both issuers arrive, with or without items
         ++n_acc;
       }
     }
@@ -682,6 +739,18 @@ struct Worker {
       float v[16], u[16];
       tc::tmem_ld16(t_lane + (uint32_t)(cb * 16), v);
       if (P.dual) tc::tmem_ld16(t_lane + (uint32_t)(c.BN + cb * 16), u);
+      if (c.n_iss == 2 && P.n_groups >= 2) {  // the second MMA issuer's share of the reduction
+        const uint32_t off = (uint32_t)((P.dual + 1) * c.BN + cb * 16);
+        float w[16];
+        tc::tmem_ld16(t_lane + off, w);
+#pragma unroll
+        for (int k = 0; k < 16; ++k) v[k] += w[k];
+        if (P.dual) {
+          tc::tmem_ld16(t_lane + off + (uint32_t)c.BN, w);
+#pragma unroll
+          for (int k = 0; k < 16; ++k) u[k] += w[k];
+        }
+      }
       if (cb != group && resid && fv) {
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
@@ -1432,7 +1501,7 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
       tc::mbar_init(tc::smem_u32(&sh.empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
-      tc::mbar_init(tc::smem_u32(&sh.acc_full[b]), 1);
+      tc::mbar_init(tc::smem_u32(&sh.acc_full[b]), 2);   // one arrival per MMA issuer
       tc::mbar_init(tc::smem_u32(&sh.acc_empty[b]), 1);
     }
     sh.abort = 0;
@@ -1453,14 +1522,12 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
   const uint32_t tmem_base = sh.tmem_base;
 
   if (warp == 0) {
-    if (lane == 0) producer_a(p, &sh, ring_base);
+    producer_a(p, &sh, ring_base, lane);
   } else if (warp == 1) {
-    if (lane == 0) {
-      const CUtensorMap* bmaps[5] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head};
-      producer_b(p, &sh, ring_base, bmaps);
-    }
-  } else if (warp == 2) {
-    if (lane == 0) mma_issuer(p, &sh, ring_base, tmem_base);
+    const CUtensorMap* bmaps[5] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head};
+    producer_b(p, &sh, ring_base, bmaps, lane);
+  } else if (warp == 2 || warp == 3) {
+    if (lane == 0) mma_issuer(p, &sh, ring_base, tmem_base, warp - 2);
   } else if (warp >= 4) {
     Worker w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0};
     w.run();

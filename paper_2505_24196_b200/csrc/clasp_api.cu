@@ -61,7 +61,8 @@ struct Workspace {
   float2* e_att_ml;
   float* ss_a;
   float* ss_m;
-  float* cosp;
+  long long* cosacc;
+  size_t cosacc_bytes;
   float4* head_best;
   int* flags;
   clasp::pk::Ctl* ctl;
@@ -138,7 +139,8 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
     w.e_att_ml = (float2*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * sizeof(float2));
     w.ss_a = (float*)take(G * rcap * 4);
     w.ss_m = (float*)take(G * rcap * 4);
-    w.cosp = (float*)take(G * (rcap + pk::MAX_ROWS) * 5 * 4);
+    w.cosacc_bytes = ((size_t)c.L + 4) * (rcap + pk::MAX_ROWS) * 5 * sizeof(long long);
+    w.cosacc = (long long*)take(w.cosacc_bytes);
     w.head_best = (float4*)take(G * pk::MAX_ROWS * sizeof(float4));
     w.flags = (int*)take(pk::N_FLAGS * (G + 32) * sizeof(int));
     w.ctl = (pk::Ctl*)take(256);
@@ -667,6 +669,9 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   CUDA_TRY(cudaMemcpyAsync(ws.jobs, ctx->e_jobs.data(), ctx->e_jobs.size() * sizeof(pk::Job),
                            cudaMemcpyHostToDevice, ctx->stream));
   CUDA_TRY(cudaMemsetAsync(ws.ctl, 0, 4, ctx->stream));  // abort flag; the status word is sticky
+  bool any_dp = false;
+  for (const pk::Job& J : ctx->e_jobs) any_dp = any_dp || J.type == pk::JOB_SELECT || J.dp;
+  if (any_dp) CUDA_TRY(cudaMemsetAsync(ws.cosacc, 0, ws.cosacc_bytes, ctx->stream));
   CUDA_TRY(cudaMemsetAsync(ws.flags, 0, (size_t)pk::N_FLAGS * (ctx->e_G + 32) * sizeof(int), ctx->stream));
 
   pk::Params P{};
@@ -680,7 +685,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   P.c.tiles_off = ctx->e_tiles_off; P.c.loads_off = ctx->e_loads_off;
   P.b.xn_a = (bf16*)ws.xn; P.b.xn_m = (bf16*)ws.xn_m; P.b.attn = (bf16*)ws.attn; P.b.act = (bf16*)ws.act;
   P.b.qkv = ws.qkv; P.b.x1 = ws.x1; P.b.Gbuf = ws.G; P.b.att_acc = ws.e_att_acc; P.b.att_ml = ws.e_att_ml;
-  P.b.ss_a = ws.ss_a; P.b.ss_m = ws.ss_m; P.b.cosp = ws.cosp; P.b.head_best = ws.head_best; P.b.flags = ws.flags;
+  P.b.ss_a = ws.ss_a; P.b.ss_m = ws.ss_m; P.b.cosacc = ws.cosacc; P.b.head_best = ws.head_best; P.b.flags = ws.flags;
   P.b.rope = ws.rope;
   P.jobs = ws.jobs; P.n_jobs = (int)ctx->e_jobs.size(); P.wmaps = ws.wmaps; P.tabs = ws.tabs; P.ctl = ws.ctl;
   P.trace = ctx->e_trace; P.trace_cap = ctx->e_trace_cap;

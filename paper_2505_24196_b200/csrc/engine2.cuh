@@ -113,7 +113,8 @@ struct Bufs {
   float2* att_ml;  // [rows*nq, chunk_cap]
   float* ss_a;     // [G, Rcap] sums of squares per CTA feature slice (attention norm / head norm)
   float* ss_m;     // [G, Rcap] (MLP norm)
-  float* cosp;     // [G, Rcap + MAX_ROWS, 5] partial dot products of Eq. 2
+  long long* cosacc;  // [jobs, Rcap + MAX_ROWS, 5] dot products of Eq. 2 summed over the CTAs in fixed point
+                   // (integer atomics: the sum does not depend on arrival order); zero at launch
   float4* head_best;  // [G, MAX_ROWS] (max, index bits, sum exp, -)
   int* flags;      // [N_FLAGS, G] epoch flags, followed by N_FLAGS arrival counters 32 ints apart
   const float2* rope;  // [T, hd/2] (cos, sin) of the rows' positions
@@ -909,8 +910,8 @@ struct Worker {
 
   // ---- Eq. 2 step i over this CTA's slice of the d features (thread <-> feature as in the
   // epilogue):
-  //   (1) per-CTA partial dot products -> cosp, publish;
-  //   (2) wait for every CTA, add the partials in CTA order, decide (every CTA decides alike);
+  //   (1) per-CTA partial dot products, added to the job's fixed-point accumulators, publish;
+  //   (2) wait for every CTA, read the totals, decide (every CTA decides alike);
   //   (3) write this CTA's slice of g[i][.] and of the next step's operand, publish.
   // from_epilogue: the down product's epilogue left the partials of this CTA in the tables and
   // the thread's layer outputs / skip candidates of its first row block in keep_y / keep_s.
@@ -926,6 +927,7 @@ struct Worker {
     const int rows = n_states * J.T;
     const int ncb = (rows + 15) >> 4;
     const long long cstride = (long long)(c.Rcap + MAX_ROWS) * 5;
+    constexpr double COS_FIX = 268435456.0;  // 2^28: sums up to 3e10 with 4e-9 resolution
     if (!from_epilogue) {
       // (1) no layer ran for this CTA's features: only skip candidates exist
       for (int cb = group; cb < ncb; cb += 2) {
@@ -955,31 +957,20 @@ struct Worker {
       }
     }
     worker_sync();
+    // this CTA's share of every dot product goes into the job's accumulators
+    unsigned long long* acc = reinterpret_cast<unsigned long long*>(p.b.cosacc) + (long long)jb * cstride;
     for (int idx = wtid; idx < rows * 5; idx += WORKERS) {
       const int r = idx / 5, k = idx % 5;
-      __stcg(p.b.cosp + blockIdx.x * cstride + idx, T->red[0][r][k] + T->red[1][r][k] + T->red[2][r][k] + T->red[3][r][k]);
+      const float part = T->red[0][r][k] + T->red[1][r][k] + T->red[2][r][k] + T->red[3][r][k];
+      atomicAdd(acc + idx, (unsigned long long)__double2ll_rn((double)part * COS_FIX));
     }
     publish(F_DOWN, jb + 1);
     mark(T_DP_PUB);
-    // (2) every CTA's partials, added in CTA order by a fixed shuffle tree
+    // (2) once every CTA has added its share: read the totals, decide
     if (!wait_all(F_DOWN, J.tgt[F_DOWN])) return false;
     mark(T_DP_ALL);
-    for (int r = ww; r < rows; r += 8) {
-      double v[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
-      for (int cc = lane; cc < c.G; cc += 32) {
-        const float* src = p.b.cosp + cc * cstride + (long long)r * 5;
-        float f5[5];
-#pragma unroll
-        for (int k = 0; k < 5; ++k) f5[k] = __ldcg(src + k);
-#pragma unroll
-        for (int k = 0; k < 5; ++k) v[k] += (double)f5[k];
-      }
-#pragma unroll
-      for (int k = 0; k < 5; ++k) {
-        v[k] = warp_sum_d(v[k]);
-        if (lane == 0) T->cosv[r][k] = v[k];
-      }
-    }
+    for (int idx = wtid; idx < rows * 5; idx += WORKERS)
+      T->cosv[idx / 5][idx % 5] = (double)(long long)__ldcg(acc + idx) * (1.0 / COS_FIX);
     worker_sync();
     if (wtid < n_states) {
       const int j = wtid + 1;
@@ -1107,29 +1098,27 @@ struct Worker {
         rr[h] = pv[h] ? pp / Gq : 0;
         hq[h] = kvh * Gq + (pv[h] ? pp % Gq : 0);
       }
-      // q fragments, rotated: element d pairs with d +- HD/2
+      // q fragments, rotated.  Element i of the first half pairs with element i + HD/2: one load
+      // of each gives the rotated values of both, i.e. the fragments of k-steps ks and ks + KS/2.
       uint32_t qh[KS][4], ql[KS][4];
 #pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
+      for (int ks = 0; ks < KS / 2; ++ks) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
 #pragma unroll
           for (int kh = 0; kh < 2; ++kh) {
-            float2 v = make_float2(0.f, 0.f);
+            float2 v0 = make_float2(0.f, 0.f), v1 = v0;
             if (active && pv[h]) {
-              const int dd = ks * 16 + kh * 8 + c4 * 2;          // dims dd, dd+1 (same half)
-              const int i = dd % HALF;
+              const int i = ks * 16 + kh * 8 + c4 * 2;           // dims i, i + 1 of the first half
               const float* qr = p.b.qkv + (long long)rr[h] * qkvd + hq[h] * HD;
               const float2 lo2 = __ldcg(reinterpret_cast<const float2*>(qr + i));
               const float2 hi2 = __ldcg(reinterpret_cast<const float2*>(qr + i + HALF));
-              const float2 cs0 = p.b.rope[(long long)(rr[h] % J.T) * HALF + i];
-              const float2 cs1 = p.b.rope[(long long)(rr[h] % J.T) * HALF + i + 1];
-              if (dd < HALF) v = make_float2(lo2.x * cs0.x - hi2.x * cs0.y, lo2.y * cs1.x - hi2.y * cs1.y);
-              else v = make_float2(hi2.x * cs0.x + lo2.x * cs0.y, hi2.y * cs1.x + lo2.y * cs1.y);
-              v.x *= qscale;
-              v.y *= qscale;
+              const float4 cs = *reinterpret_cast<const float4*>(p.b.rope + (long long)(rr[h] % J.T) * HALF + i);
+              v0 = make_float2((lo2.x * cs.x - hi2.x * cs.y) * qscale, (lo2.y * cs.z - hi2.y * cs.w) * qscale);
+              v1 = make_float2((hi2.x * cs.x + lo2.x * cs.y) * qscale, (hi2.y * cs.z + lo2.y * cs.w) * qscale);
             }
-            split2(v.x, v.y, qh[ks][h + kh * 2], ql[ks][h + kh * 2]);
+            split2(v0.x, v0.y, qh[ks][h + kh * 2], ql[ks][h + kh * 2]);
+            split2(v1.x, v1.y, qh[ks + KS / 2][h + kh * 2], ql[ks + KS / 2][h + kh * 2]);
           }
         }
       }

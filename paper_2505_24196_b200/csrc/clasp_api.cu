@@ -59,8 +59,9 @@ struct Workspace {
   void* xn_m;
   float* e_att_acc;
   float2* e_att_ml;
-  float* ss_a;
-  float* ss_m;
+  long long* ss_a;
+  long long* ss_m;
+  size_t acc_bytes;
   long long* cosacc;
   size_t cosacc_bytes;
   float4* head_best;
@@ -137,10 +138,13 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
     w.e_chunk_cap = (c.max_ctx + w.e_run_len - 1) / w.e_run_len + (int)((rcap + pk::ATT_KEYS - 1) / pk::ATT_KEYS);
     w.e_att_acc = (float*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * c.head_dim * 4);
     w.e_att_ml = (float2*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * sizeof(float2));
-    w.ss_a = (float*)take(G * rcap * 4);
-    w.ss_m = (float*)take(G * rcap * 4);
+    // fixed-point accumulators, zeroed before every launch: ss_a, ss_m, cosacc are contiguous
+    const size_t ss_bytes = align_up(((size_t)c.L + 5) * rcap * sizeof(long long), 256);
+    w.ss_a = (long long*)take(ss_bytes);
+    w.ss_m = (long long*)take(ss_bytes);
     w.cosacc_bytes = ((size_t)c.L + 4) * (rcap + pk::MAX_ROWS) * 5 * sizeof(long long);
     w.cosacc = (long long*)take(w.cosacc_bytes);
+    w.acc_bytes = (size_t)((uint8_t*)w.cosacc - (uint8_t*)w.ss_a) + align_up(w.cosacc_bytes, 256);
     w.head_best = (float4*)take(G * pk::MAX_ROWS * sizeof(float4));
     w.flags = (int*)take(pk::N_FLAGS * (G + 32) * sizeof(int));
     w.ctl = (pk::Ctl*)take(256);
@@ -669,9 +673,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   CUDA_TRY(cudaMemcpyAsync(ws.jobs, ctx->e_jobs.data(), ctx->e_jobs.size() * sizeof(pk::Job),
                            cudaMemcpyHostToDevice, ctx->stream));
   CUDA_TRY(cudaMemsetAsync(ws.ctl, 0, 4, ctx->stream));  // abort flag; the status word is sticky
-  bool any_dp = false;
-  for (const pk::Job& J : ctx->e_jobs) any_dp = any_dp || J.type == pk::JOB_SELECT || J.dp;
-  if (any_dp) CUDA_TRY(cudaMemsetAsync(ws.cosacc, 0, ws.cosacc_bytes, ctx->stream));
+  CUDA_TRY(cudaMemsetAsync(ws.ss_a, 0, ws.acc_bytes, ctx->stream));  // all fixed-point accumulators
   CUDA_TRY(cudaMemsetAsync(ws.flags, 0, (size_t)pk::N_FLAGS * (ctx->e_G + 32) * sizeof(int), ctx->stream));
 
   pk::Params P{};

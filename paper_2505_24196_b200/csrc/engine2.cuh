@@ -111,8 +111,9 @@ struct Bufs {
   float* Gbuf;     // [rows, d]    layer outputs of the candidate states (Eq. 2)
   float* att_acc;  // [rows*nq, chunk_cap, hd]
   float2* att_ml;  // [rows*nq, chunk_cap]
-  float* ss_a;     // [G, Rcap] sums of squares per CTA feature slice (attention norm / head norm)
-  float* ss_m;     // [G, Rcap] (MLP norm)
+  long long* ss_a; // [jobs, Rcap] row sums of squares of the operand of job j's first product (attention
+                   // norm / head norm), summed over the CTAs in fixed point; zero at launch
+  long long* ss_m; // [jobs, Rcap] same for the operand of job j's gate/up product (MLP norm)
   long long* cosacc;  // [jobs, Rcap + MAX_ROWS, 5] dot products of Eq. 2 summed over the CTAs in fixed point
                    // (integer atomics: the sum does not depend on arrival order); zero at launch
   float4* head_best;  // [G, MAX_ROWS] (max, index bits, sum exp, -)
@@ -641,16 +642,17 @@ struct Worker {
   __device__ __forceinline__ const int* split_lo(int split) const { return p.tabs + p.c.split_lo[split]; }
   __device__ __forceinline__ RedTables* tables() const { return reinterpret_cast<RedTables*>(scratch); }
 
-  // per-row factors rsqrt(mean(x^2) + eps) from the per-CTA sums of squares
-  __device__ void row_scales(const float* ss, int R, int row_off) {
+  // fixed-point scale of the sums of squares (2^24: sums up to 5e11, resolution 6e-8)
+  static constexpr double SS_FIX = 16777216.0;
+  __device__ __forceinline__ static void ss_add(long long* dst, float v) {
+    atomicAdd(reinterpret_cast<unsigned long long*>(dst), (unsigned long long)__double2ll_rn((double)v * SS_FIX));
+  }
+  // per-row factors rsqrt(mean(x^2) + eps) from the accumulated sums of squares
+  __device__ void row_scales(const long long* ss, int R, int row_off) {
     const Cfg& c = p.c;
-    const int* dlo = split_lo(S_D);
-    for (int r = ww; r < R; r += 8) {
-      float s = 0.f;
-      for (int cc = lane; cc < c.G; cc += 32)
-        if (__ldg(dlo + cc + 1) > __ldg(dlo + cc)) s += __ldcg(ss + (long long)cc * c.Rcap + row_off + r);
-      s = warp_sum(s);
-      if (lane == 0) sh->rs[r] = rsqrtf(s / (float)c.d + c.eps);
+    for (int r = wtid; r < R; r += WORKERS) {
+      const double s = (double)__ldcg(ss + row_off + r) * (1.0 / SS_FIX);
+      sh->rs[r] = rsqrtf((float)s / (float)c.d + c.eps);
     }
     worker_sync();
   }
@@ -671,7 +673,7 @@ struct Worker {
         *reinterpret_cast<uint2*>(p.b.xn_a + (long long)r * c.d + col) = pack4(v.x * w.x, v.y * w.y, v.z * w.z, v.w * w.w);
       }
       ssq = warp_sum(ssq);
-      if (lane == 0) p.b.ss_a[(long long)blockIdx.x * c.Rcap + r] = ssq;
+      if (lane == 0 && n4 > 0) ss_add(p.b.ss_a + (long long)(epoch - 1) * c.Rcap + r, ssq);
     }
     fence_proxy_async();
     publish(F_PREP, epoch);
@@ -683,7 +685,7 @@ struct Worker {
   // (sums of squares, cosine partials, arg-max) go through RedTables: one entry per (quarter, row).
   // For the down product of an Eq. 2 job the thread's layer outputs (keep_y) and skip candidates
   // (keep_s) of its first block of 16 rows stay in registers for dp_step.
-  __device__ bool epilogue(const Job& J, const Phase& P, const TileDesc& td, int tile_no, float (&keep_y)[16],
+  __device__ bool epilogue(const Job& J, int jb, const Phase& P, const TileDesc& td, int tile_no, float (&keep_y)[16],
                            float (&keep_s)[16]) {
     const Cfg& c = p.c;
     RedTables* T = tables();
@@ -733,7 +735,7 @@ struct Worker {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if ((P.kind == G_QKV || P.kind == G_GU || P.kind == G_HEAD) && tile_no == 0) {
       // the reduction consumed every operand column, so every CTA's sums of squares are published
-      row_scales(P.kind == G_GU ? p.b.ss_m : p.b.ss_a, J.R, P.kind == G_HEAD ? J.row_off : 0);
+      row_scales((P.kind == G_GU ? p.b.ss_m : p.b.ss_a) + (long long)jb * c.Rcap, J.R, P.kind == G_HEAD ? J.row_off : 0);
     }
     const uint32_t t_lane = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
     for (int cb = group; cb < ncb; cb += 2) {
@@ -869,11 +871,10 @@ struct Worker {
     ++n_acc;
     // cross-warp part of the per-row sums: add the four quarters in a fixed order
     if (P.kind == G_O || (P.kind == G_DOWN && !J.dp && J.norm_next)) {
-      float* ss = (P.kind == G_O ? p.b.ss_m : p.b.ss_a) + (long long)blockIdx.x * c.Rcap;
-      for (int r = wtid; r < J.R; r += WORKERS) {
-        const float s2 = T->red[0][r][0] + T->red[1][r][0] + T->red[2][r][0] + T->red[3][r][0];
-        ss[r] = (tile_no == 0 ? 0.f : ss[r]) + s2;
-      }
+      // o product: MLP norm of this job; down product: the next job's first operand
+      long long* ss = P.kind == G_O ? p.b.ss_m + (long long)jb * c.Rcap : p.b.ss_a + (long long)(jb + 1) * c.Rcap;
+      for (int r = wtid; r < J.R; r += WORKERS)
+        ss_add(ss + r, T->red[0][r][0] + T->red[1][r][0] + T->red[2][r][0] + T->red[3][r][0]);
     } else if (P.kind == G_HEAD) {
       for (int r = wtid; r < J.R; r += WORKERS) {
         float best = -INFINITY, se = 0.f;
@@ -1035,7 +1036,8 @@ struct Worker {
     worker_sync();
     if (J.norm_next)
       for (int r = wtid; r < rows; r += WORKERS)
-        p.b.ss_a[(long long)blockIdx.x * c.Rcap + r] = T->red[0][r][0] + T->red[1][r][0] + T->red[2][r][0] + T->red[3][r][0];
+        ss_add(p.b.ss_a + (long long)(jb + 1) * c.Rcap + r,
+               T->red[0][r][0] + T->red[1][r][0] + T->red[2][r][0] + T->red[3][r][0]);
     fence_proxy_async();
     publish(F_SELECT, jb + 1);
     return true;
@@ -1435,7 +1437,7 @@ struct Worker {
         Phase P;
         P.init(p, J, 0);
         for (int t = 0; t < P.n_tiles; ++t)
-          if (!epilogue(J, P, tiles[P.tile0 + t], t, keep_y, keep_s)) return false;
+          if (!epilogue(J, jb, P, tiles[P.tile0 + t], t, keep_y, keep_s)) return false;
         if (!head_merge(J, jb)) return false;
         mark(T_HEAD);
         continue;
@@ -1446,7 +1448,7 @@ struct Worker {
         Phase P;
         P.init(p, J, ph);
         for (int t = 0; t < P.n_tiles; ++t)
-          if (!epilogue(J, P, tiles[P.tile0 + t], t, keep_y, keep_s)) return false;
+          if (!epilogue(J, jb, P, tiles[P.tile0 + t], t, keep_y, keep_s)) return false;
         mark(ph == G_QKV ? T_QKV : (ph == G_O ? T_O : (ph == G_GU ? T_GU : T_DOWN)));
         if (ph == G_QKV) {
           publish(F_QKV, jb + 1);

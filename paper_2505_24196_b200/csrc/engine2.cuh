@@ -621,9 +621,11 @@ struct Worker {
   __device__ __forceinline__ void publish(int kind, int epoch) {
     worker_sync();
     if (wtid == 0) {
-      __threadfence();
-      st_release_i32(p.b.flags + kind * p.c.G + blockIdx.x, epoch);
-      atomicAdd(p.b.flags + N_FLAGS * p.c.G + kind * 32, 1);
+      __threadfence();  // the workers' stores (ordered before this thread by the CTA barrier) first
+      int* flag = p.b.flags + kind * p.c.G + blockIdx.x;
+      int* cnt = p.b.flags + N_FLAGS * p.c.G + kind * 32;
+      asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(epoch) : "memory");
+      asm volatile("red.relaxed.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
     }
   }
   // every CTA has published step `kind` tgt times: one thread polls, the others wait for it
@@ -645,7 +647,8 @@ struct Worker {
   // fixed-point scale of the sums of squares (2^24: sums up to 5e11, resolution 6e-8)
   static constexpr double SS_FIX = 16777216.0;
   __device__ __forceinline__ static void ss_add(long long* dst, float v) {
-    atomicAdd(reinterpret_cast<unsigned long long*>(dst), (unsigned long long)__double2ll_rn((double)v * SS_FIX));
+    const long long q = __double2ll_rn((double)v * SS_FIX);
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(dst), "l"(q) : "memory");
   }
   // per-row factors rsqrt(mean(x^2) + eps) from the accumulated sums of squares
   __device__ void row_scales(const long long* ss, int R, int row_off) {
@@ -675,7 +678,6 @@ struct Worker {
       ssq = warp_sum(ssq);
       if (lane == 0 && n4 > 0) ss_add(p.b.ss_a + (long long)(epoch - 1) * c.Rcap + r, ssq);
     }
-    fence_proxy_async();
     publish(F_PREP, epoch);
   }
 
@@ -899,7 +901,6 @@ struct Worker {
         *dst = make_float4(best, __int_as_float(bi), se, 0.f);
       }
     }
-    if (P.kind == G_O || P.kind == G_GU || (P.kind == G_DOWN && !J.dp && J.norm_next)) fence_proxy_async();
     if (P.kind == G_HEAD || P.kind == G_O || (P.kind == G_DOWN && !J.dp)) worker_sync();  // tables reused by the next tile
     return true;
   }
@@ -963,7 +964,8 @@ struct Worker {
     for (int idx = wtid; idx < rows * 5; idx += WORKERS) {
       const int r = idx / 5, k = idx % 5;
       const float part = T->red[0][r][k] + T->red[1][r][k] + T->red[2][r][k] + T->red[3][r][k];
-      atomicAdd(acc + idx, (unsigned long long)__double2ll_rn((double)part * COS_FIX));
+      const long long q = __double2ll_rn((double)part * COS_FIX);
+      asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(acc + idx), "l"(q) : "memory");
     }
     publish(F_DOWN, jb + 1);
     mark(T_DP_PUB);
@@ -1038,7 +1040,6 @@ struct Worker {
       for (int r = wtid; r < rows; r += WORKERS)
         ss_add(p.b.ss_a + (long long)(jb + 1) * c.Rcap + r,
                T->red[0][r][0] + T->red[1][r][0] + T->red[2][r][0] + T->red[3][r][0]);
-    fence_proxy_async();
     publish(F_SELECT, jb + 1);
     return true;
   }
@@ -1343,7 +1344,6 @@ struct Worker {
         }
       }
     }
-    fence_proxy_async();
     publish(F_MERGE, jb + 1);
     return true;
   }

@@ -148,7 +148,7 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
     w.head_best = (float4*)take(G * pk::MAX_ROWS * sizeof(float4));
     w.flags = (int*)take(pk::N_FLAGS * (G + 32) * sizeof(int));
     w.ctl = (pk::Ctl*)take(256);
-    w.wmaps = (CUtensorMap*)take(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS * sizeof(CUtensorMap));
+    w.wmaps = (CUtensorMap*)take(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS * 2 * sizeof(CUtensorMap));
     w.jobs = (pk::Job*)take(((size_t)c.L + 4) * sizeof(pk::Job));
     w.tabs = (int*)take(ENGINE_TAB_INTS * sizeof(int));
   }
@@ -184,11 +184,12 @@ struct clasp_ctx {
   int e_G = 0;              // CTAs of the cooperative grid (one per SM)
   int e_static_smem = 0;
   int e_split_lo[clasp::pk::N_SPLITS], e_split_units[clasp::pk::N_SPLITS], e_tile_idx[5], e_tiles_off = 0,
-      e_loads_off = 0, e_kpi[5];
+      e_kpi[5], e_use3d[5], e_wpages[5];
+  int e_heights[8][clasp::pk::N_HEIGHTS];   // tile heights per matrix slot (wq wk wv wo gate up down head)
   std::vector<CUtensorMap> e_wmaps_host;
   bool e_wmaps_dirty = true;
-  std::map<int, std::array<CUtensorMap, 4>> e_bmaps;           // by BN
-  std::map<std::pair<int, int>, CUtensorMap> e_headmaps;       // by (row offset, BN)
+  std::map<int, std::array<CUtensorMap, 8>> e_bmaps;           // by BN: 2-D maps of the four operands, then 3-D
+  std::map<std::pair<int, int>, std::array<CUtensorMap, 2>> e_headmaps;  // by (row offset, BN): 2-D, 3-D
   std::vector<clasp::pk::Job> e_jobs;
   unsigned long long* e_trace = nullptr;
   int e_trace_cap = 0;
@@ -216,6 +217,20 @@ int make_map(clasp_ctx* ctx, const void* ptr, int rows, int cols, int box_rows, 
   cuuint32_t estr[2] = {1, 1};
   CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides,
                            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? CLASP_OK : CLASP_ERR_CUDA;
+}
+
+// 3-D bf16 tensor map over the same matrix seen as {64 columns, rows, K/64 chunks} (strides
+// {cols*2, 128} bytes): a box {64, box_rows, box_chunks} lands in shared memory as box_chunks
+// consecutive [box_rows x 128 B] swizzled tiles.  Needs cols % 64 == 0.
+int make_map3(clasp_ctx* ctx, const void* ptr, int rows, int cols, int box_rows, int box_chunks, CUtensorMap* out) {
+  cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+  cuuint64_t strides[2] = {(cuuint64_t)cols * 2, 128};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_chunks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? CLASP_OK : CLASP_ERR_CUDA;
 }
@@ -521,28 +536,47 @@ int engine_setup(clasp_ctx* ctx) {
     if (v >= 1 && v < G) G = v;
   }
   if (G > ENGINE_MAX_CTAS) G = ENGINE_MAX_CTAS;
-  // ---- feature splits and per-CTA tile / load lists
+  // ---- feature splits and per-CTA tiles.  A CTA's range never straddles two weight matrices:
+  // the CTAs of the q/k/v product are dealt to the three matrices in proportion to their rows.
   const int split_n[pk::N_SPLITS] = {qd + 2 * kvd, d, c.d_ffn, c.vocab};
   const int kind_split[5] = {pk::S_QKV, pk::S_D, pk::S_F, pk::S_D, pk::S_V};
+  const int kind_K[5] = {d, qd, d, c.d_ffn, d};
+  const int kind_slot0[5] = {0, 3, 4, 6, 7};   // first matrix slot of the kind
   std::vector<int> tab;
   std::vector<std::vector<int>> lo(pk::N_SPLITS);
   for (int s = 0; s < pk::N_SPLITS; ++s) {
-    const long long units = split_n[s] / 8;
-    if ((units + 1) * G > 0x7fffffffLL) return CLASP_OK;
-    lo[s].resize(G + 1);
-    for (int cc = 0; cc <= G; ++cc) lo[s][cc] = (int)(units * cc / G) * 8;
+    lo[s].assign(G + 1, 0);
+    if (s == pk::S_QKV) {
+      const int mat_n[3] = {qd, kvd, kvd};
+      int share[3], given = 0;
+      for (int m = 0; m < 3; ++m) { share[m] = (int)((long long)G * mat_n[m] / split_n[s]); if (share[m] < 1) share[m] = 1; given += share[m]; }
+      for (int m = 0; given < G; m = (m + 1) % 3) { ++share[m]; ++given; }
+      while (given > G) { int m = share[0] >= share[1] && share[0] >= share[2] ? 0 : (share[1] >= share[2] ? 1 : 2); --share[m]; --given; }
+      if (G < 3) return CLASP_OK;
+      int cc = 0, base = 0;
+      for (int m = 0; m < 3; ++m) {
+        const long long units = mat_n[m] / 8;
+        for (int k = 0; k < share[m]; ++k) lo[s][cc + k] = base + (int)(units * k / share[m]) * 8;
+        cc += share[m];
+        base += mat_n[m];
+      }
+      lo[s][G] = base;
+    } else {
+      const long long units = split_n[s] / 8;
+      for (int cc = 0; cc <= G; ++cc) lo[s][cc] = (int)(units * cc / G) * 8;
+    }
     ctx->e_split_lo[s] = (int)tab.size();
-    ctx->e_split_units[s] = (int)units;
+    ctx->e_split_units[s] = split_n[s] / 8;
     tab.insert(tab.end(), lo[s].begin(), lo[s].end());
   }
   for (int cc = 0; cc < G; ++cc)
     if (lo[pk::S_D][cc + 1] - lo[pk::S_D][cc] > 128) return CLASP_OK;  // the Eq. 2 step takes one feature per thread
   std::vector<pk::TileDesc> tiles;
-  std::vector<pk::LoadDesc> loads;
   std::vector<std::vector<int>> tidx(5, std::vector<int>(G + 1, 0));
+  for (int sl = 0; sl < 8; ++sl)
+    for (int h = 0; h < pk::N_HEIGHTS; ++h) ctx->e_heights[sl][h] = 0;
   for (int k = 0; k < 5; ++k) {
     const int s = kind_split[k];
-    // matrices stacked along the feature axis of this product
     int mat_n[3] = {split_n[s], 0, 0}, n_mats = 1;
     if (k == pk::G_QKV) { mat_n[0] = qd; mat_n[1] = kvd; mat_n[2] = kvd; n_mats = 3; }
     int max_rows = 8;
@@ -550,63 +584,62 @@ int engine_setup(clasp_ctx* ctx) {
       tidx[k][cc] = (int)tiles.size();
       for (int f0 = lo[s][cc]; f0 < lo[s][cc + 1]; f0 += 128) {
         const int n = std::min(128, lo[s][cc + 1] - f0);
+        int m = 0, base = 0;
+        while (m + 1 < n_mats && f0 >= base + mat_n[m]) { base += mat_n[m]; ++m; }
+        if (f0 + n > base + mat_n[m]) return CLASP_OK;  // cannot happen: ranges are aligned to the matrices
+        int* hts = ctx->e_heights[kind_slot0[k] + m];
+        int hi = 0;
+        while (hi < pk::N_HEIGHTS && hts[hi] != n && hts[hi] != 0) ++hi;
+        if (hi == pk::N_HEIGHTS) return CLASP_OK;       // more distinct tile heights than maps per matrix
+        hts[hi] = n;
         pk::TileDesc td{};
-        td.f0 = f0; td.n_rows = (short)n; td.load0 = (int)loads.size();
+        td.f0 = f0; td.n_rows = (short)n; td.map_local = (short)(m * pk::N_HEIGHTS + hi); td.y0 = f0 - base;
         if (n > max_rows) max_rows = n;
-        int f = f0, left = n;
-        while (left > 0) {
-          int m = 0, base = 0;
-          while (m + 1 < n_mats && f >= base + mat_n[m]) { base += mat_n[m]; ++m; }
-          int piece = std::min(left, base + mat_n[m] - f);
-          int y = f - base;
-          for (int hi = pk::N_HEIGHTS - 1; hi >= 0 && piece > 0; --hi) {
-            const int h = 8 << hi;
-            while (piece >= h) {
-              pk::LoadDesc ld{};
-              ld.map_local = (short)(m * pk::N_HEIGHTS + hi); ld.row_off = (short)(f - f0); ld.y0 = y; ld.rows = h;
-              loads.push_back(ld);
-              y += h; f += h; piece -= h; left -= h;
-            }
-          }
-        }
-        td.n_loads = (short)((int)loads.size() - td.load0);
-        if (td.n_loads > pk::MAX_TILE_LOADS) return CLASP_OK;
         tiles.push_back(td);
       }
     }
     tidx[k][G] = (int)tiles.size();
+    if (k == pk::G_GU)  // the up matrix is loaded with the gate matrix's heights
+      for (int h = 0; h < pk::N_HEIGHTS; ++h) ctx->e_heights[5][h] = ctx->e_heights[4][h];
     const int a_pages = (k == pk::G_GU ? 2 : 1) * (max_rows / 8);
+    ctx->e_wpages[k] = a_pages;   // weight pages of one chunk of the kind's tallest tile
     int kpi = 16 / a_pages;
     ctx->e_kpi[k] = kpi < 1 ? 1 : (kpi > 4 ? 4 : kpi);
+    // (the gate/up product interleaves two matrices per chunk, which one box cannot deliver)
+    ctx->e_use3d[k] = (k != pk::G_GU && kind_K[k] % 64 == 0 && ctx->e_kpi[k] > 1 && !getenv("CLASP_ENGINE_NO3D")) ? 1 : 0;
   }
   for (int k = 0; k < 5; ++k) {
     ctx->e_tile_idx[k] = (int)tab.size();
     tab.insert(tab.end(), tidx[k].begin(), tidx[k].end());
   }
-  static_assert(sizeof(pk::TileDesc) == 12 && sizeof(pk::LoadDesc) == 12, "table records are three ints");
+  static_assert(sizeof(pk::TileDesc) == 12, "table records are three ints");
   ctx->e_tiles_off = (int)tab.size();
   tab.resize(tab.size() + tiles.size() * 3);
   memcpy(tab.data() + ctx->e_tiles_off, tiles.data(), tiles.size() * sizeof(pk::TileDesc));
-  ctx->e_loads_off = (int)tab.size();
-  tab.resize(tab.size() + loads.size() * 3);
-  memcpy(tab.data() + ctx->e_loads_off, loads.data(), loads.size() * sizeof(pk::LoadDesc));
   if (tab.size() > ENGINE_TAB_INTS) return CLASP_OK;
   CUDA_TRY(cudaMemcpyAsync(ctx->ws.tabs, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
   CUDA_TRY(cudaStreamSynchronize(ctx->stream));
   ctx->e_G = G;
-  ctx->e_wmaps_host.assign(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS, CUtensorMap{});
+  ctx->e_wmaps_host.assign(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS * 2, CUtensorMap{});
   ctx->e_wmaps_dirty = true;
   ctx->use_engine = true;
   return CLASP_OK;
 }
 
-// tensor maps of one weight matrix for every box height
-int engine_maps(clasp_ctx* ctx, int slot, const void* w, int rows, int cols) {
-  int rc = 0;
-  for (int hi = 0; hi < pk::N_HEIGHTS; ++hi)
-    rc |= make_map(ctx, w, rows, cols, 8 << hi, &ctx->e_wmaps_host[(size_t)slot * pk::N_HEIGHTS + hi]);
+// tensor maps of one weight matrix for every tile height its product uses: 2-D (one chunk per box)
+// and, where the product takes them, 3-D (all chunks of a ring item in one box)
+int engine_maps(clasp_ctx* ctx, int slot, int kind_slot, int kind, const void* w, int rows, int cols) {
+  const size_t n2 = ((size_t)ctx->cfg.L * 7 + 1) * pk::N_HEIGHTS;
+  for (int hi = 0; hi < pk::N_HEIGHTS; ++hi) {
+    const int h = ctx->e_heights[kind_slot][hi];
+    if (h == 0) continue;
+    if (make_map(ctx, w, rows, cols, h, &ctx->e_wmaps_host[(size_t)slot * pk::N_HEIGHTS + hi])) return CLASP_ERR_CUDA;
+    if (ctx->e_use3d[kind] &&
+        make_map3(ctx, w, rows, cols, h, ctx->e_kpi[kind], &ctx->e_wmaps_host[n2 + (size_t)slot * pk::N_HEIGHTS + hi]))
+      return CLASP_ERR_CUDA;
+  }
   ctx->e_wmaps_dirty = true;
-  return rc ? CLASP_ERR_CUDA : CLASP_OK;
+  return CLASP_OK;
 }
 
 // weight + visible K/V bytes one job must move (for the per-launch bandwidth figure)
@@ -636,33 +669,36 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
     const int v = atoi(e);
     if (v >= 64 && v < ring_pages) ring_pages = v;
   }
-  // an item (gate + up rows and the operand tile of kpi chunks) must fit the ring twice over
+  // an item (gate + up rows and the operand tiles of kpi chunks) must fit the ring twice over
   const int b_pages = BN * pk::BK * 2 / pk::PAGE;
-  int kpi[5];
-  for (int k = 0; k < 5; ++k) {
-    kpi[k] = ctx->e_kpi[k];
-    const int chunk_pages = 16 * (k == pk::G_GU ? 2 : 1) + b_pages;
-    while (kpi[k] > 1 && kpi[k] * chunk_pages * 2 > ring_pages) --kpi[k];
-    if (chunk_pages > ring_pages) return CLASP_ERR_CAPACITY;
-  }
+  for (int k = 0; k < 5; ++k)
+    if (ctx->e_kpi[k] * (ctx->e_wpages[k] + b_pages) * 2 > ring_pages) return CLASP_ERR_CAPACITY;
   const size_t dyn = 1024 + (size_t)ring_pages * pk::PAGE + pk::SCRATCH_BYTES;
 
+  const int qdim = qd;
   auto bm = ctx->e_bmaps.find(BN);
   if (bm == ctx->e_bmaps.end()) {
-    std::array<CUtensorMap, 4> m;
+    std::array<CUtensorMap, 8> m{};
     int rc = 0;
     rc |= make_map(ctx, ws.xn, rows_cap, d, BN, &m[0]);
-    rc |= make_map(ctx, ws.attn, rows_cap, qd, BN, &m[1]);
+    rc |= make_map(ctx, ws.attn, rows_cap, qdim, BN, &m[1]);
     rc |= make_map(ctx, ws.xn_m, rows_cap, d, BN, &m[2]);
     rc |= make_map(ctx, ws.act, rows_cap, c.d_ffn, BN, &m[3]);
+    if (ctx->e_use3d[pk::G_QKV]) rc |= make_map3(ctx, ws.xn, rows_cap, d, BN, ctx->e_kpi[pk::G_QKV], &m[4]);
+    if (ctx->e_use3d[pk::G_O]) rc |= make_map3(ctx, ws.attn, rows_cap, qdim, BN, ctx->e_kpi[pk::G_O], &m[5]);
+    if (ctx->e_use3d[pk::G_GU]) rc |= make_map3(ctx, ws.xn_m, rows_cap, d, BN, ctx->e_kpi[pk::G_GU], &m[6]);
+    if (ctx->e_use3d[pk::G_DOWN]) rc |= make_map3(ctx, ws.act, rows_cap, c.d_ffn, BN, ctx->e_kpi[pk::G_DOWN], &m[7]);
     if (rc) return CLASP_ERR_CUDA;
     bm = ctx->e_bmaps.emplace(BN, m).first;
   }
   auto hk = std::make_pair(head_off, BN);
   auto hm = ctx->e_headmaps.find(hk);
   if (hm == ctx->e_headmaps.end()) {
-    CUtensorMap m;
-    if (make_map(ctx, (const bf16*)ws.xn + (size_t)head_off * d, rows_cap - head_off, d, BN, &m)) return CLASP_ERR_CUDA;
+    std::array<CUtensorMap, 2> m{};
+    const bf16* base = (const bf16*)ws.xn + (size_t)head_off * d;
+    int rc = make_map(ctx, base, rows_cap - head_off, d, BN, &m[0]);
+    if (ctx->e_use3d[pk::G_HEAD]) rc |= make_map3(ctx, base, rows_cap - head_off, d, BN, ctx->e_kpi[pk::G_HEAD], &m[1]);
+    if (rc) return CLASP_ERR_CUDA;
     hm = ctx->e_headmaps.emplace(hk, m).first;
   }
   if (ctx->e_wmaps_dirty) {
@@ -683,8 +719,8 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   P.c.BN = BN; P.c.ring_pages = ring_pages; P.c.n_iss = BN <= 64 ? 2 : 1;
   if (getenv("CLASP_ENGINE_ONE_ISSUER")) P.c.n_iss = 1;
   for (int s = 0; s < pk::N_SPLITS; ++s) { P.c.split_lo[s] = ctx->e_split_lo[s]; P.c.split_units[s] = ctx->e_split_units[s]; }
-  for (int k = 0; k < 5; ++k) { P.c.tile_idx[k] = ctx->e_tile_idx[k]; P.c.kpi[k] = kpi[k]; }
-  P.c.tiles_off = ctx->e_tiles_off; P.c.loads_off = ctx->e_loads_off;
+  for (int k = 0; k < 5; ++k) { P.c.tile_idx[k] = ctx->e_tile_idx[k]; P.c.kpi[k] = ctx->e_kpi[k]; P.c.use3d[k] = ctx->e_use3d[k]; }
+  P.c.tiles_off = ctx->e_tiles_off; P.c.map3d_off = (int)(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS);
   P.b.xn_a = (bf16*)ws.xn; P.b.xn_m = (bf16*)ws.xn_m; P.b.attn = (bf16*)ws.attn; P.b.act = (bf16*)ws.act;
   P.b.qkv = ws.qkv; P.b.x1 = ws.x1; P.b.Gbuf = ws.G; P.b.att_acc = ws.e_att_acc; P.b.att_ml = ws.e_att_ml;
   P.b.ss_a = ws.ss_a; P.b.ss_m = ws.ss_m; P.b.cosacc = ws.cosacc; P.b.head_best = ws.head_best; P.b.flags = ws.flags;
@@ -698,7 +734,8 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
     cudaEventRecord(e0, ctx->stream);
   }
   void* args[] = {(void*)&bm->second[0], (void*)&bm->second[1], (void*)&bm->second[2], (void*)&bm->second[3],
-                  (void*)&hm->second, (void*)&P};
+                  (void*)&hm->second[0], (void*)&bm->second[4], (void*)&bm->second[5], (void*)&bm->second[6],
+                  (void*)&bm->second[7], (void*)&hm->second[1], (void*)&P};
   cudaError_t err = cudaLaunchCooperativeKernel((const void*)pk::engine_kernel, dim3(ctx->e_G), dim3(pk::THREADS),
                                                 args, dyn, ctx->stream);
   if (ctx->profiling) {
@@ -848,13 +885,13 @@ int clasp_load_layers(clasp_ctx* ctx, int32_t first, int32_t count, const clasp_
       if (ctx->use_engine) {
         const int b7 = (first + k) * 7;
         int erc = 0;
-        erc |= engine_maps(ctx, b7 + 0, lw.wq, qd, d);
-        erc |= engine_maps(ctx, b7 + 1, lw.wk, kvd, d);
-        erc |= engine_maps(ctx, b7 + 2, lw.wv, kvd, d);
-        erc |= engine_maps(ctx, b7 + 3, lw.wo, d, qd);
-        erc |= engine_maps(ctx, b7 + 4, lw.w_gate, c.d_ffn, d);
-        erc |= engine_maps(ctx, b7 + 5, lw.w_up, c.d_ffn, d);
-        erc |= engine_maps(ctx, b7 + 6, lw.w_down, d, c.d_ffn);
+        erc |= engine_maps(ctx, b7 + 0, 0, pk::G_QKV, lw.wq, qd, d);
+        erc |= engine_maps(ctx, b7 + 1, 1, pk::G_QKV, lw.wk, kvd, d);
+        erc |= engine_maps(ctx, b7 + 2, 2, pk::G_QKV, lw.wv, kvd, d);
+        erc |= engine_maps(ctx, b7 + 3, 3, pk::G_O, lw.wo, d, qd);
+        erc |= engine_maps(ctx, b7 + 4, 4, pk::G_GU, lw.w_gate, c.d_ffn, d);
+        erc |= engine_maps(ctx, b7 + 5, 5, pk::G_GU, lw.w_up, c.d_ffn, d);
+        erc |= engine_maps(ctx, b7 + 6, 6, pk::G_DOWN, lw.w_down, d, c.d_ffn);
         if (erc) return CLASP_ERR_CUDA;
       }
     }
@@ -872,7 +909,7 @@ int clasp_load_head(clasp_ctx* ctx, const void* embed, const float* final_norm, 
   ctx->lm_head = lm_head;
   if (ctx->use_tc && make_map(ctx, lm_head, ctx->cfg.vocab, ctx->cfg.d_model, clasp::tc::BM, &ctx->lm_head_map))
     return CLASP_ERR_CUDA;
-  if (ctx->use_engine && engine_maps(ctx, ctx->cfg.L * 7, lm_head, ctx->cfg.vocab, ctx->cfg.d_model))
+  if (ctx->use_engine && engine_maps(ctx, ctx->cfg.L * 7, 7, pk::G_HEAD, lm_head, ctx->cfg.vocab, ctx->cfg.d_model))
     return CLASP_ERR_CUDA;
   return CLASP_OK;
 }

@@ -55,8 +55,7 @@ constexpr int NB = 32;                // items in flight (mbarrier pairs)
 constexpr int ATT_KEYS = 32;
 constexpr int SCRATCH_BYTES = 2 * ATT_KEYS * 136 * 2 + 2048;  // two padded K/V tiles + slack (>= 16 KB guard)
 constexpr int MAX_ROWS = 128;         // rows one launch may push through a layer
-constexpr int N_HEIGHTS = 5;          // TMA box heights 8, 16, 32, 64, 128
-constexpr int MAX_TILE_LOADS = 8;
+constexpr int N_HEIGHTS = 4;          // distinct tile heights (TMA box heights) per weight matrix
 constexpr int MAX_CTAS = 192;
 
 enum { JOB_LAYER = 0, JOB_HEAD = 1, JOB_SELECT = 2 };
@@ -69,17 +68,11 @@ enum { F_PREP = 0, F_QKV, F_ATTN, F_MERGE, F_O, F_GU, F_DOWN, F_SELECT, F_HEAD, 
 enum { T_START = 0, T_QKV, T_ATT_READY, T_ATT_Q, T_ATT_TILES, T_ATT_PUB, T_MERGE, T_O, T_GU, T_DOWN, T_DP_PUB,
        T_DP_ALL, T_DP_DECIDED, T_DP_DONE, T_HEAD };
 
-struct TileDesc {      // one accumulator's worth of a CTA's feature range
+struct TileDesc {      // one accumulator's worth of a CTA's feature range: rows y0.. of one weight matrix
   int f0;              // first feature in the product's feature space
-  short n_rows;        // features (multiple of 8, <= 128)
-  short n_loads;
-  int load0;           // first LoadDesc
-};
-struct LoadDesc {
+  short n_rows;        // features (multiple of 8, <= 128) = height of the TMA box
   short map_local;     // matrix * N_HEIGHTS + height index
-  short row_off;       // destination row inside the tile (multiple of 8)
   int y0;              // first row in the matrix
-  int rows;            // box height
 };
 
 struct Cfg {
@@ -97,8 +90,10 @@ struct Cfg {
   int split_units[N_SPLITS]; // 8-feature units of each split
   int tile_idx[5];           // per product kind: [G + 1] first TileDesc of each CTA
   int tiles_off;             // TileDesc array
-  int loads_off;             // LoadDesc array
   int kpi[5];                // 64-column chunks per ring item
+  int use3d[5];              // 1: one 3-D box {64 columns, rows, kpi chunks} per item and matrix (needs K % 64 == 0),
+                             // 0: one 2-D box per chunk
+  int map3d_off;             // index of the first 3-D weight map in Params::wmaps
 };
 
 struct Bufs {
@@ -170,7 +165,7 @@ struct Params {
   Bufs b;
   const Job* jobs;
   int n_jobs;
-  const CUtensorMap* wmaps;  // [(L*7 + 1) * N_HEIGHTS]
+  const CUtensorMap* wmaps;  // [(L*7 + 1) * N_HEIGHTS] 2-D maps, then as many 3-D maps
   const int* tabs;
   Ctl* ctl;
   unsigned long long* trace;  // optional [G, trace_cap] time stamps (ns)
@@ -268,6 +263,16 @@ __device__ __forceinline__ void mma_chunk(uint32_t acc, uint32_t a_lo, uint32_t 
   mma_lo<true>(acc, a_lo + 2, b_lo + 2, idesc);
   mma_lo<true>(acc, a_lo + 4, b_lo + 4, idesc);
   mma_lo<true>(acc, a_lo + 6, b_lo + 6, idesc);
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      :
+      : "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "l"(policy)
+      : "memory");
 }
 
 // ------------------------------------------------------------------ shared state
@@ -394,15 +399,17 @@ struct RingPos {
   }
 };
 
-// Warp 0, all lanes: every lane walks the schedule; lane 0 does the ring bookkeeping and each
-// lane issues at most one of an item's TMA boxes, so that all boxes of an item leave in one
-// instruction (a single thread can only issue a TMA every few hundred cycles).
+// Ring item of tile (rows n) of a product: kpi chunks of weight rows, then kpi operand tiles:
+//   [W chunk 0 | W chunk 1 | ...]  each (dual + 1) * n / 8 pages (gate rows, then up rows)
+//   [X chunk 0 | X chunk 1 | ...]  each BN / 8 pages
+// Warp 0, all lanes: every lane walks the schedule; lane 0 does the ring bookkeeping.  With 3-D
+// maps one box brings all chunks of an item (a thread can issue a TMA only every ~150 cycles, so
+// the number of boxes, not their size, bounds the rate); otherwise lane k issues chunk k.
 __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base, int lane) {
   const Cfg& c = p.c;
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
   const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
-  const LoadDesc* loads = reinterpret_cast<const LoadDesc*>(p.tabs + c.loads_off);
   RingPos rp{0, 0};
   int used = 0;
   uint32_t tail = 0;
@@ -414,19 +421,14 @@ __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base, int 
     for (int ph = 0; ph < nph; ++ph) {
       Phase P;
       P.init(p, J, ph);
+      const bool d3 = c.use3d[P.kind] != 0;
       for (int t = 0; t < P.n_tiles; ++t) {
         const TileDesc td = tiles[P.tile0 + t];
         const int a_pages = td.n_rows >> 3;
-        const int chunk_pages = (P.dual + 1) * a_pages + b_pages;
-        const int pages = P.kpi * chunk_pages;
-        // boxes of one chunk: n_loads (x2 with the "up" matrix); lane l issues box l % per_chunk of
-        // chunk l / per_chunk.  Its load descriptor is fixed for the whole tile.
-        const int per_chunk = td.n_loads * (P.dual + 1);
-        const int my_box = lane % per_chunk, my_chunk = lane / per_chunk;
-        const int my_half = my_box / td.n_loads;
-        const LoadDesc ld = loads[td.load0 + my_box % td.n_loads];
-        const uint32_t my_off = (uint32_t)(my_half * a_pages * PAGE) + (uint32_t)ld.row_off * 128u;
-        const CUtensorMap* my_map = p.wmaps + P.map_base + my_half * N_HEIGHTS + ld.map_local;
+        const int w_pages = (P.dual + 1) * a_pages;       // weight pages of one chunk
+        const int pages = P.kpi * (w_pages + b_pages);
+        const CUtensorMap* map2 = p.wmaps + P.map_base + td.map_local;
+        const CUtensorMap* map3 = map2 + c.map3d_off;
         for (int gi = 0; gi < P.n_groups; ++gi) {
           // make room: items leave the ring in the order they entered it
           int fp;
@@ -445,13 +447,19 @@ __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base, int 
           used += fp;
           const int k0 = P.group_at(gi) * P.kpi, nk = min(P.kc, k0 + P.kpi) - k0;
           const uint32_t full = tc::smem_u32(&sh->full[it % NB]);
-          if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)(nk * (P.dual + 1) * a_pages * PAGE));
-          __syncwarp();
-          for (int base = 0; base < nk; base += 32 / per_chunk) {   // one pass unless an item has > 32 boxes
-            const int kk = base + my_chunk;
-            if (my_chunk < 32 / per_chunk && kk < nk)
-              tc::tma_load_2d(ring_base + (uint32_t)(at + kk * chunk_pages) * PAGE + my_off, my_map, full, (k0 + kk) * BK,
-                              ld.y0, pol);
+          const uint32_t dst = ring_base + (uint32_t)at * PAGE;
+          if (d3) {  // boxes always span kpi chunks; chunks beyond K arrive as zeros
+            if (lane == 0) {
+              tc::mbar_expect_tx(full, (uint32_t)(P.kpi * w_pages * PAGE));
+              tma_load_3d(dst, map3, full, 0, td.y0, k0, pol);
+            }
+          } else {
+            if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)(nk * w_pages * PAGE));
+            __syncwarp();
+            const int kk = lane >> 1, half = lane & 1;     // lane -> (chunk, gate / up)
+            if (kk < nk && half <= P.dual)
+              tc::tma_load_2d(dst + (uint32_t)((kk * w_pages + half * a_pages) * PAGE), map2 + half * N_HEIGHTS, full,
+                              (k0 + kk) * BK, td.y0, pol);
           }
           __syncwarp();
           if (lane == 0) sh->a_issued = (int)(it + 1);
@@ -461,14 +469,9 @@ __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base, int 
   }
 }
 
-// CTA that owns feature f of a split with `units` 8-feature units: the largest c with
-// floor(c units / G) <= f / 8  (CTAs with an empty range are never the largest such c)
-__device__ __forceinline__ int owner_of(int units, int G, int f) {
-  return (((f >> 3) + 1) * G - 1) / units;
-}
-
 // Warp 1, all lanes: lane k issues the operand tile of an item's chunk k.
-__device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, const CUtensorMap* const* bmaps, int lane) {
+__device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, const CUtensorMap* const* bmaps,
+                           const CUtensorMap* const* bmaps3, int lane) {
   const Cfg& c = p.c;
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
@@ -496,11 +499,11 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
         if (!__all_sync(0xffffffffu, ok)) return;
       }
       fence_proxy_async();  // the producers' ordinary stores before this warp's TMA reads
+      const bool d3 = c.use3d[P.kind] != 0;
       for (int t = 0; t < P.n_tiles; ++t) {
         const TileDesc td = tiles[P.tile0 + t];
-        const int a_pages = td.n_rows >> 3;
-        const int chunk_pages = (P.dual + 1) * a_pages + b_pages;
-        const int pages = P.kpi * chunk_pages;
+        const int w_pages = (P.dual + 1) * (td.n_rows >> 3);
+        const int pages = P.kpi * (w_pages + b_pages);
         for (int gi = 0; gi < P.n_groups; ++gi) {
           int fp;
           const uint32_t it = rp.item;
@@ -518,11 +521,17 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
           if (!__all_sync(0xffffffffu, ok)) return;
           const int k0 = P.group_at(gi) * P.kpi, nk = min(P.kc, k0 + P.kpi) - k0;
           const uint32_t full = tc::smem_u32(&sh->full[it % NB]);
-          if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)nk * b_bytes);
-          __syncwarp();
-          if (lane < nk)
-            tc::tma_load_2d(ring_base + (uint32_t)(at + lane * chunk_pages + (P.dual + 1) * a_pages) * PAGE, bmaps[bmap],
-                            full, (k0 + lane) * BK, 0, pol);
+          const uint32_t dst = ring_base + (uint32_t)(at + P.kpi * w_pages) * PAGE;
+          if (d3) {
+            if (lane == 0) {
+              tc::mbar_expect_tx(full, (uint32_t)P.kpi * b_bytes);
+              tma_load_3d(dst, bmaps3[bmap], full, 0, 0, k0, pol);
+            }
+          } else {
+            if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)nk * b_bytes);
+            __syncwarp();
+            if (lane < nk) tc::tma_load_2d(dst + (uint32_t)lane * b_bytes, bmaps[bmap], full, (k0 + lane) * BK, 0, pol);
+          }
           __syncwarp();
         }
       }
@@ -549,16 +558,17 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
       for (int t = 0; t < P.n_tiles; ++t) {
         const TileDesc td = tiles[P.tile0 + t];
         const int a_pages = td.n_rows >> 3;
-        const int chunk_pages = (P.dual + 1) * a_pages + b_pages;
-        const int pages = P.kpi * chunk_pages;
+        const int w_pages = (P.dual + 1) * a_pages;
+        const int pages = P.kpi * (w_pages + b_pages);
         const uint32_t buf = n_acc & 1u;
         if (!wait_bar(&sh->acc_empty[buf], ((n_acc >> 1) & 1u) ^ 1u, p.ctl, sh)) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t acc = tmem_base + buf * 256u + (uint32_t)(which * (P.dual + 1) * c.BN);
         const uint32_t acc2 = acc + (uint32_t)c.BN;
-        const uint32_t up_lo = (uint32_t)a_pages * (PAGE / 16);                  // gate rows -> up rows
-        const uint32_t b_off = (uint32_t)((P.dual + 1) * a_pages) * (PAGE / 16);  // weight rows -> operand tile
-        const uint32_t chunk_lo = (uint32_t)chunk_pages * (PAGE / 16);
+        const uint32_t up_lo = (uint32_t)a_pages * (PAGE / 16);          // gate rows -> up rows
+        const uint32_t w_lo = (uint32_t)w_pages * (PAGE / 16);           // weights of one chunk
+        const uint32_t x_lo = (uint32_t)b_pages * (PAGE / 16);           // operand tile of one chunk
+        const uint32_t x0_lo = (uint32_t)P.kpi * w_lo;                   // first weight chunk -> first operand tile
         for (int gi = 0; gi < P.n_groups; ++gi) {
           int fp;
           const uint32_t it = rp.item;
@@ -569,23 +579,27 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
           const int k0 = P.group_at(gi) * P.kpi;
           const int nk = min(P.kc, k0 + P.kpi) - k0;
           uint32_t a_lo = desc_lo(ring_base + (uint32_t)at * PAGE);
+          uint32_t b_lo = a_lo + x0_lo;
           int k = 0;
           if (gi < c.n_iss) {  // this issuer's first item of the tile overwrites its accumulator
-            mma_chunk<true>(acc, a_lo, a_lo + b_off, idesc);
-            if (P.dual) mma_chunk<true>(acc2, a_lo + up_lo, a_lo + b_off, idesc);
-            a_lo += chunk_lo;
+            mma_chunk<true>(acc, a_lo, b_lo, idesc);
+            if (P.dual) mma_chunk<true>(acc2, a_lo + up_lo, b_lo, idesc);
+            a_lo += w_lo;
+            b_lo += x_lo;
             k = 1;
           }
           if (P.dual) {
             for (; k < nk; ++k) {
-              mma_chunk<false>(acc, a_lo, a_lo + b_off, idesc);
-              mma_chunk<false>(acc2, a_lo + up_lo, a_lo + b_off, idesc);
-              a_lo += chunk_lo;
+              mma_chunk<false>(acc, a_lo, b_lo, idesc);
+              mma_chunk<false>(acc2, a_lo + up_lo, b_lo, idesc);
+              a_lo += w_lo;
+              b_lo += x_lo;
             }
           } else {
             for (; k < nk; ++k) {
-              mma_chunk<false>(acc, a_lo, a_lo + b_off, idesc);
-              a_lo += chunk_lo;
+              mma_chunk<false>(acc, a_lo, b_lo, idesc);
+              a_lo += w_lo;
+              b_lo += x_lo;
             }
           }
           tc::mma_commit(tc::smem_u32(&sh->empty[it % NB]));
@@ -1068,28 +1082,14 @@ struct Worker {
     const long long kvld = c.kvd;
     const int qkvd = c.qd + 2 * c.kvd;
     const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;
-    const int qunits = c.split_units[S_QKV];
+    // every row's q, k, v exist once all CTAs have published their slice of the projections
+    if (!wait_all(F_QKV, J.tgt[F_QKV])) return false;
+    mark(T_ATT_READY);
     for (int it = blockIdx.x; it < n_items; it += c.G) {
       const int pbg = it % n_pbg;
       const int chunk = (it / n_pbg) % n_chunks;
       const int kvh = it / (n_pbg * n_chunks);
       const bool own = chunk >= n_runs;
-      // producers of this kv head's q heads, k head and v head
-      {
-        const int q0 = kvh * Gq * HD, q1 = q0 + Gq * HD - 1;
-        const int k0 = c.qd + kvh * HD, v0 = c.qd + c.kvd + kvh * HD;
-        const int a0 = owner_of(qunits, c.G, q0), a1 = owner_of(qunits, c.G, q1);
-        const int b0 = owner_of(qunits, c.G, k0), b1 = owner_of(qunits, c.G, k0 + HD - 1);
-        const int d0 = owner_of(qunits, c.G, v0), d1 = owner_of(qunits, c.G, v0 + HD - 1);
-        bool ok = true;
-        const int na = a1 - a0 + 1, nb2 = b1 - b0 + 1, nd = d1 - d0 + 1;
-        for (int k = wtid; k < na + nb2 + nd; k += WORKERS) {
-          const int cc = k < na ? a0 + k : (k < na + nb2 ? b0 + (k - na) : d0 + (k - na - nb2));
-          ok = wait_flag(p.b.flags + F_QKV * c.G + cc, jb + 1, p.ctl, sh) && ok;
-        }
-        if (!worker_and(ok)) return false;
-      }
-      mark(T_ATT_READY);
       const int p0 = (pbg * 8 + ww) * 16;
       const bool active = p0 < Pn;
       int rr[2], hq[2];
@@ -1478,7 +1478,10 @@ struct Worker {
 __global__ void __launch_bounds__(THREADS, 1)
 engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constant__ CUtensorMap map_attn,
               const __grid_constant__ CUtensorMap map_xn_m, const __grid_constant__ CUtensorMap map_act,
-              const __grid_constant__ CUtensorMap map_head, const __grid_constant__ Params p) {
+              const __grid_constant__ CUtensorMap map_head, const __grid_constant__ CUtensorMap map3_xn_a,
+              const __grid_constant__ CUtensorMap map3_attn, const __grid_constant__ CUtensorMap map3_xn_m,
+              const __grid_constant__ CUtensorMap map3_act, const __grid_constant__ CUtensorMap map3_head,
+              const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ Shared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1516,7 +1519,8 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
     producer_a(p, &sh, ring_base, lane);
   } else if (warp == 1) {
     const CUtensorMap* bmaps[5] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head};
-    producer_b(p, &sh, ring_base, bmaps, lane);
+    const CUtensorMap* bmaps3[5] = {&map3_xn_a, &map3_attn, &map3_xn_m, &map3_act, &map3_head};
+    producer_b(p, &sh, ring_base, bmaps, bmaps3, lane);
   } else if (warp == 2 || warp == 3) {
     if (lane == 0) mma_issuer(p, &sh, ring_base, tmem_base, warp - 2);
   } else if (warp >= 4) {

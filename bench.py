@@ -34,7 +34,8 @@ import datagen  # noqa: E402
 WORKLOADS = {
     # BASELINE configs[1]: 8B shape, 512-token context, M = 12, one objective token
     "8b-c512-M12": dict(model="8b", ctx=512, M=12, T=1, K=4),
-    # small stand-ins for quick checks (not bench lines)
+    # small stand-ins for quick checks and profiler captures (not bench lines)
+    "8b-l6-c512-M3": dict(model="8b-l6", ctx=512, M=3, T=1, K=4),
     "mini8b-c128-M2": dict(model="mini8b", ctx=128, M=2, T=1, K=3),
     "tiny-c64-M2": dict(model="tiny", ctx=64, M=2, T=1, K=4),
 }
@@ -153,12 +154,14 @@ def run_ours(args, rank, world):
     sampler.start()
     barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()   # lets `ncu --profile-from-start off` list only the timed region's launches
     ev0.record(eng.stream)
     new_tokens = 0
     for _ in range(steps):
         new_tokens += len(dec.round())
     ev1.record(eng.stream)
     barrier()
+    torch.cuda.profiler.stop()
     total_ms = ev0.elapsed_time(ev1)
     clocks = sampler.stop()
     launches = eng.launch_count() - launches0

@@ -86,6 +86,10 @@ CONFIGS: Dict[str, ModelConfig] = {
     # configs[1], [2], [4]: LLaMA3-8B shape
     "8b": ModelConfig("8b", L=32, d_model=4096, n_q_heads=32, n_kv_heads=8, head_dim=128,
                       d_ffn=14336, vocab=128256, dtype="bf16", scale_out_proj=True, seed=2),
+    # the 8B layer shape with few layers and a small vocabulary: a profiler capture saves and
+    # restores device memory per pass, so it runs on ~3 GB of weights instead of 16 GB
+    "8b-l6": ModelConfig("8b-l6", L=6, d_model=4096, n_q_heads=32, n_kv_heads=8, head_dim=128,
+                         d_ffn=14336, vocab=16384, dtype="bf16", scale_out_proj=True, seed=2),
     # configs[3]: LLaMA3-70B shape
     "70b": ModelConfig("70b", L=80, d_model=8192, n_q_heads=64, n_kv_heads=8, head_dim=128,
                        d_ffn=28672, vocab=128256, dtype="bf16", scale_out_proj=True, seed=3),

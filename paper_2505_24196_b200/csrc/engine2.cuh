@@ -66,7 +66,11 @@ enum { S_QKV = 0, S_D = 1, S_F = 2, S_V = 3, N_SPLITS = 4 };
 enum { F_PREP = 0, F_QKV, F_ATTN, F_MERGE, F_O, F_GU, F_DOWN, F_SELECT, F_HEAD, N_FLAGS };
 // trace slots of a job (time stamps of the workers' step boundaries)
 enum { T_START = 0, T_QKV, T_ATT_READY, T_ATT_Q, T_ATT_TILES, T_ATT_PUB, T_MERGE, T_O, T_GU, T_DOWN, T_DP_PUB,
-       T_DP_ALL, T_DP_DECIDED, T_DP_DONE, T_HEAD };
+       T_DP_ALL, T_DP_DECIDED, T_DP_DONE, T_HEAD,
+       // per product ph = 0..3 (q/k/v, o, gate/up, down): first ring item of the product ready for the MMA issuer,
+       // its last MMA issued, and the product's first accumulator complete (seen by the workers)
+       T_MMA_FIRST = 16, T_MMA_LAST = 20, T_ACC = 24 };
+constexpr int TRACE_SLOTS = 32;  // time stamps per job
 
 struct TileDesc {      // one accumulator's worth of a CTA's feature range: rows y0.. of one weight matrix
   int f0;              // first feature in the product's feature space
@@ -539,6 +543,15 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
   }
 }
 
+__device__ __forceinline__ void issuer_mark(const Params& p, int jb, int slot) {
+  const int idx = jb * TRACE_SLOTS + slot;
+  if (p.trace != nullptr && idx < p.trace_cap) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    p.trace[(long long)blockIdx.x * p.trace_cap + idx] = t;
+  }
+}
+
 // MMA issuer `which` (0 or 1) takes the ring items of each tile with that parity and adds them up
 // in accumulator `which` of the tile's buffer: buffer b holds accumulator a at column
 // b * 256 + a * (dual + 1) * BN  (gate at +0, up at +BN).
@@ -576,6 +589,7 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
           if ((gi & (c.n_iss - 1)) != which) continue;
           if (!wait_bar(&sh->full[it % NB], (it / NB) & 1u, p.ctl, sh)) return;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          if (t == 0 && gi == 0) issuer_mark(p, jb, T_MMA_FIRST + ph);
           const int k0 = P.group_at(gi) * P.kpi;
           const int nk = min(P.kc, k0 + P.kpi) - k0;
           uint32_t a_lo = desc_lo(ring_base + (uint32_t)at * PAGE);
@@ -605,6 +619,7 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
           tc::mma_commit(tc::smem_u32(&sh->empty[it % NB]));
         }
         tc::mma_commit(tc::smem_u32(&sh->acc_full[buf]));  // both issuers arrive, with or without items
+        if (which == 0 && t == P.n_tiles - 1) issuer_mark(p, jb, T_MMA_LAST + ph);
         ++n_acc;
       }
     }
@@ -621,9 +636,9 @@ struct Worker {
   uint32_t n_acc;
   int n_mark;
 
-  // time stamp of step `slot` (one of the T_* below) of the current job: 16 slots per job
+  // time stamp of step `slot` (one of the T_* above) of the current job
   __device__ __forceinline__ void mark(int slot) {
-    const int idx = n_mark * 16 + slot;
+    const int idx = n_mark * TRACE_SLOTS + slot;
     if (p.trace != nullptr && wtid == 0 && idx < p.trace_cap) {
       unsigned long long t;
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -749,6 +764,7 @@ struct Worker {
     ok = worker_and(ok);
     if (!ok) return false;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (tile_no == 0 && P.kind < 4) mark(T_ACC + P.kind);
     if ((P.kind == G_QKV || P.kind == G_GU || P.kind == G_HEAD) && tile_no == 0) {
       // the reduction consumed every operand column, so every CTA's sums of squares are published
       row_scales((P.kind == G_GU ? p.b.ss_m : p.b.ss_a) + (long long)jb * c.Rcap, J.R, P.kind == G_HEAD ? J.row_off : 0);

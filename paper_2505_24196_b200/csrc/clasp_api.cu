@@ -667,7 +667,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   int ring_pages = (optin - ctx->e_static_smem - 1024 - pk::SCRATCH_BYTES) / pk::PAGE;
   if (const char* e = getenv("CLASP_ENGINE_PAGES")) {
     const int v = atoi(e);
-    if (v >= 64 && v < ring_pages) ring_pages = v;
+    if (v >= 64 && v < ring_pages && BN <= 32) ring_pages = v;
   }
   // an item (gate + up rows and the operand tiles of kpi chunks) must fit the ring twice over
   const int b_pages = BN * pk::BK * 2 / pk::PAGE;
@@ -718,6 +718,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   P.c.G = ctx->e_G; P.c.Rcap = ws.e_rcap; P.c.run_len = ws.e_run_len; P.c.chunk_cap = ws.e_chunk_cap;
   P.c.BN = BN; P.c.ring_pages = ring_pages; P.c.n_iss = BN <= 64 ? 2 : 1;
   if (getenv("CLASP_ENGINE_ONE_ISSUER")) P.c.n_iss = 1;
+
   for (int s = 0; s < pk::N_SPLITS; ++s) { P.c.split_lo[s] = ctx->e_split_lo[s]; P.c.split_units[s] = ctx->e_split_units[s]; }
   for (int k = 0; k < 5; ++k) { P.c.tile_idx[k] = ctx->e_tile_idx[k]; P.c.kpi[k] = ctx->e_kpi[k]; P.c.use3d[k] = ctx->e_use3d[k]; }
   P.c.tiles_off = ctx->e_tiles_off; P.c.map3d_off = (int)(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS);
@@ -977,6 +978,7 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
       J.i = i; J.ell = ell; J.diag = i <= M ? 1 : 0; J.M = M;
       J.x_i = hidden_states + (int64_t)i * layer_stride;
       J.x_im1 = hidden_states + (int64_t)(i - 1) * layer_stride;
+      J.x_ip1 = i < L ? hidden_states + (int64_t)(i + 1) * layer_stride : nullptr;
       J.x_tok_stride = token_stride;
       J.g_prev = ws.grow[cur]; J.g_next = ws.grow[cur ^ 1];
       J.D = scores + (int64_t)i * (M + 1);

@@ -151,6 +151,7 @@ struct Job {
   int i, ell, diag, M;
   const float* x_i;
   const float* x_im1;
+  const float* x_ip1;      // objective rows of the next step (null at the last one)
   long long x_tok_stride;
   const float* g_prev;
   float* g_next;
@@ -288,6 +289,7 @@ struct Shared {
   volatile int a_issued;    // ring items whose weight loads have been issued (warp 0 -> warp 1)
   int flag;                 // broadcast of a one-thread decision to the workers
   float rs[MAX_ROWS];       // per-row norm factors of the current product
+  float rs_next[MAX_ROWS];  // Eq. 2 step: norm factors of the rows it hands to the next layer
   int choice[MAX_ROWS + 2];
   int foot[NB];             // warp 0: ring pages each item in flight gives back when it retires
   int job_words[(sizeof(Job) + 3) / 4];  // the workers' copy of the current job descriptor
@@ -403,6 +405,49 @@ struct RingPos {
   }
 };
 
+// Position in the sequence of ring items of a launch: (job, product, tile, chunk group).
+struct ItemCursor {
+  int jb, ph, nph, t, gi;
+  bool valid;
+  Phase P;
+  TileDesc td;
+  __device__ __forceinline__ void settle(const Params& p, const TileDesc* tiles, bool new_tile) {
+    for (;;) {
+      if (jb >= p.n_jobs) { valid = false; return; }
+      if (ph >= nph) {
+        ++jb; ph = 0; t = 0; gi = 0; new_tile = true;
+        if (jb < p.n_jobs) {
+          nph = n_gemm_phases(p.jobs[jb]);
+          if (nph > 0) P.init(p, p.jobs[jb], 0);
+        }
+        continue;
+      }
+      if (t >= P.n_tiles) {
+        ++ph; t = 0; gi = 0; new_tile = true;
+        if (ph < nph) P.init(p, p.jobs[jb], ph);
+        continue;
+      }
+      if (gi >= P.n_groups) { ++t; gi = 0; new_tile = true; continue; }
+      if (new_tile) td = tiles[P.tile0 + t];
+      return;
+    }
+  }
+  __device__ __forceinline__ void first(const Params& p, const TileDesc* tiles) {
+    jb = 0; ph = 0; t = 0; gi = 0; valid = true;
+    nph = n_gemm_phases(p.jobs[0]);
+    if (nph > 0) P.init(p, p.jobs[0], 0);
+    settle(p, tiles, true);
+  }
+  __device__ __forceinline__ int a_pages() const { return td.n_rows >> 3; }
+  __device__ __forceinline__ int w_pages() const { return (P.dual + 1) * (td.n_rows >> 3); }  // weight pages of one chunk
+  __device__ __forceinline__ int k0() const { return P.group_at(gi) * P.kpi; }
+  __device__ __forceinline__ int nk() const { return min(P.kc, k0() + P.kpi) - k0(); }
+  __device__ __forceinline__ void next(const Params& p, const TileDesc* tiles) {
+    ++gi;
+    settle(p, tiles, false);
+  }
+};
+
 // Ring item of tile (rows n) of a product: kpi chunks of weight rows, then kpi operand tiles:
 //   [W chunk 0 | W chunk 1 | ...]  each (dual + 1) * n / 8 pages (gate rows, then up rows)
 //   [X chunk 0 | X chunk 1 | ...]  each BN / 8 pages
@@ -419,57 +464,49 @@ __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base, int 
   uint32_t tail = 0;
   int* foot = sh->foot;
   const int b_pages = (c.BN * BK * 2) / PAGE;
-  for (int jb = 0; jb < p.n_jobs; ++jb) {
-    const Job& J = p.jobs[jb];
-    const int nph = n_gemm_phases(J);
-    for (int ph = 0; ph < nph; ++ph) {
-      Phase P;
-      P.init(p, J, ph);
-      const bool d3 = c.use3d[P.kind] != 0;
-      for (int t = 0; t < P.n_tiles; ++t) {
-        const TileDesc td = tiles[P.tile0 + t];
-        const int a_pages = td.n_rows >> 3;
-        const int w_pages = (P.dual + 1) * a_pages;       // weight pages of one chunk
-        const int pages = P.kpi * (w_pages + b_pages);
-        const CUtensorMap* map2 = p.wmaps + P.map_base + td.map_local;
-        const CUtensorMap* map3 = map2 + c.map3d_off;
-        for (int gi = 0; gi < P.n_groups; ++gi) {
-          // make room: items leave the ring in the order they entered it
-          int fp;
-          RingPos probe = rp;
-          probe.place(pages, c.ring_pages, fp);
-          while (used + fp > c.ring_pages || rp.item - tail >= (uint32_t)NB) {
-            const bool ok = wait_bar(&sh->empty[tail % NB], (tail / NB) & 1u, p.ctl, sh);
-            if (!__all_sync(0xffffffffu, ok)) return;
-            used -= foot[tail % NB];
-            ++tail;
-          }
-          const uint32_t it = rp.item;
-          const int at = rp.place(pages, c.ring_pages, fp);
-          __syncwarp();
-          if (lane == 0) foot[it % NB] = fp;
-          used += fp;
-          const int k0 = P.group_at(gi) * P.kpi, nk = min(P.kc, k0 + P.kpi) - k0;
-          const uint32_t full = tc::smem_u32(&sh->full[it % NB]);
-          const uint32_t dst = ring_base + (uint32_t)at * PAGE;
-          if (d3) {  // boxes always span kpi chunks; chunks beyond K arrive as zeros
-            if (lane == 0) {
-              tc::mbar_expect_tx(full, (uint32_t)(P.kpi * w_pages * PAGE));
-              tma_load_3d(dst, map3, full, 0, td.y0, k0, pol);
-            }
-          } else {
-            if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)(nk * w_pages * PAGE));
-            __syncwarp();
-            const int kk = lane >> 1, half = lane & 1;     // lane -> (chunk, gate / up)
-            if (kk < nk && half <= P.dual)
-              tc::tma_load_2d(dst + (uint32_t)((kk * w_pages + half * a_pages) * PAGE), map2 + half * N_HEIGHTS, full,
-                              (k0 + kk) * BK, td.y0, pol);
-          }
-          __syncwarp();
-          if (lane == 0) sh->a_issued = (int)(it + 1);
-        }
-      }
+  ItemCursor L;
+  L.first(p, tiles);
+  while (L.valid) {
+    const Phase& P = L.P;
+    const TileDesc& td = L.td;
+    const bool d3 = c.use3d[P.kind] != 0;
+    const int a_pages = L.a_pages(), w_pages = L.w_pages();
+    const int pages = P.kpi * (w_pages + b_pages);
+    // make room: items leave the ring in the order they entered it
+    int fp;
+    RingPos probe = rp;
+    probe.place(pages, c.ring_pages, fp);
+    while (used + fp > c.ring_pages || rp.item - tail >= (uint32_t)NB) {
+      const bool ok = wait_bar(&sh->empty[tail % NB], (tail / NB) & 1u, p.ctl, sh);
+      if (!__all_sync(0xffffffffu, ok)) return;
+      used -= foot[tail % NB];
+      ++tail;
     }
+    const uint32_t it = rp.item;
+    const int at = rp.place(pages, c.ring_pages, fp);
+    __syncwarp();
+    if (lane == 0) foot[it % NB] = fp;
+    used += fp;
+    const int k0 = L.k0(), nk = L.nk();
+    const uint32_t full = tc::smem_u32(&sh->full[it % NB]);
+    const uint32_t dst = ring_base + (uint32_t)at * PAGE;
+    const CUtensorMap* map2 = p.wmaps + P.map_base + td.map_local;
+    if (d3) {  // boxes always span kpi chunks; chunks beyond K arrive as zeros
+      if (lane == 0) {
+        tc::mbar_expect_tx(full, (uint32_t)(P.kpi * w_pages * PAGE));
+        tma_load_3d(dst, map2 + c.map3d_off, full, 0, td.y0, k0, pol);
+      }
+    } else {
+      if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)(nk * w_pages * PAGE));
+      __syncwarp();
+      const int kk = lane >> 1, half = lane & 1;     // lane -> (chunk, gate / up)
+      if (kk < nk && half <= P.dual)
+        tc::tma_load_2d(dst + (uint32_t)((kk * w_pages + half * a_pages) * PAGE), map2 + half * N_HEIGHTS, full,
+                        (k0 + kk) * BK, td.y0, pol);
+    }
+    __syncwarp();
+    if (lane == 0) sh->a_issued = (int)(it + 1);
+    L.next(p, tiles);
   }
 }
 
@@ -679,6 +716,36 @@ struct Worker {
     const long long q = __double2ll_rn((double)v * SS_FIX);
     asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(dst), "l"(q) : "memory");
   }
+  // Sums of v[0..31] over the warp: lane l returns the total of v[l].  31 shuffles, independent within
+  // a stage, instead of 32 five-step butterflies.
+  __device__ __forceinline__ static float warp_reduce32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int w = 16; w >= 1; w >>= 1) {
+      const bool up = (lane & w) != 0;
+#pragma unroll
+      for (int i = 0; i < w; ++i) {
+        const float send = up ? v[i] : v[i + w];
+        const float keep = up ? v[i + w] : v[i];
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, w);
+      }
+    }
+    return v[0];
+  }
+  // Same for 16 values: every lane l returns the total of v[l & 15].
+  __device__ __forceinline__ static float warp_reduce16(float (&v)[16], int lane) {
+#pragma unroll
+    for (int w = 8; w >= 1; w >>= 1) {
+      const bool up = (lane & w) != 0;
+#pragma unroll
+      for (int i = 0; i < w; ++i) {
+        const float send = up ? v[i] : v[i + w];
+        const float keep = up ? v[i + w] : v[i];
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, w);
+      }
+    }
+    return v[0] + __shfl_xor_sync(0xffffffffu, v[0], 16);
+  }
+
   // per-row factors rsqrt(mean(x^2) + eps) from the accumulated sums of squares
   __device__ void row_scales(const long long* ss, int R, int row_off) {
     const Cfg& c = p.c;
@@ -726,7 +793,7 @@ struct Worker {
     const int f = td.f0 + fl;
     const bool dpd = P.kind == G_DOWN && J.dp;
     const int rows_all = J.R + ((dpd && J.diag) ? J.T : 0);   // Eq. 2: plus the rows of the diagonal state
-    const int ncb = (rows_all + 15) >> 4;
+    const int ncb = (J.R + 15) >> 4;
     const bool resid = P.kind == G_O || P.kind == G_DOWN;
     // Eq. 2: objective row and skip candidate of every row of the first block, fetched early
     float xi[16];
@@ -765,7 +832,11 @@ struct Worker {
     if (!ok) return false;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (tile_no == 0 && P.kind < 4) mark(T_ACC + P.kind);
-    if ((P.kind == G_QKV || P.kind == G_GU || P.kind == G_HEAD) && tile_no == 0) {
+    if (P.kind == G_QKV && tile_no == 0 && J.src_flag == F_SELECT) {
+      // the rows come from an Eq. 2 step: it left their factors in shared memory
+      for (int r = wtid; r < J.R; r += WORKERS) sh->rs[r] = sh->rs_next[r];
+      worker_sync();
+    } else if ((P.kind == G_QKV || P.kind == G_GU || P.kind == G_HEAD) && tile_no == 0) {
       // the reduction consumed every operand column, so every CTA's sums of squares are published
       row_scales((P.kind == G_GU ? p.b.ss_m : p.b.ss_a) + (long long)jb * c.Rcap, J.R, P.kind == G_HEAD ? J.row_off : 0);
     }
@@ -803,18 +874,19 @@ struct Worker {
           }
         }
       } else if (P.kind == G_O) {
+        float sq[16];
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
           const int r = cb * 16 + k;
-          if (r >= J.R) break;
-          const float y = fv ? res[k] + v[k] : 0.f;
-          if (fv) {
+          const float y = (fv && r < J.R) ? res[k] + v[k] : 0.f;
+          if (fv && r < J.R) {
             __stcg(p.b.x1 + (long long)r * c.d + f, y);
             p.b.xn_m[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
           }
-          const float s2 = warp_sum(y * y);
-          if (lane == 0) T->red[quarter][r][0] = s2;
+          sq[k] = y * y;
         }
+        const float tot = warp_reduce16(sq, lane);
+        if (lane < 16 && cb * 16 + lane < J.R) T->red[quarter][cb * 16 + lane][0] = tot;
       } else if (P.kind == G_GU) {
         if (fv) {
 #pragma unroll
@@ -827,52 +899,42 @@ struct Worker {
           }
         }
       } else if (dpd) {
-        // candidate states: layer output y, skip candidate sv; five partial dot products per row
-        float sv[16];
+        // layer outputs of the candidate states; per row the two sums of Eq. 2 that involve them
+        // (x.y and y.y; the sums over the skip candidates were added when those were written)
         if (cb != group) {
 #pragma unroll
           for (int k = 0; k < 16; ++k) {
             const int r = cb * 16 + k;
-            xi[k] = 0.f;
-            sv[k] = 0.f;
-            if (fv && r < rows_all) {
-              xi[k] = __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f);
-              sv[k] = __ldcg(skip_src(J, r / J.T + 1, r % J.T) + f);
-            }
+            xi[k] = (fv && r < J.R) ? __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f) : 0.f;
           }
-        } else {
-#pragma unroll
-          for (int k = 0; k < 16; ++k) sv[k] = keep_s[k];
         }
+        float pr[32];
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
           const int r = cb * 16 + k;
-          if (r < rows_all) {
-            const float y = (fv && r < J.R) ? res[k] + v[k] : 0.f;
-            if (fv && r < J.R) __stcg(p.b.Gbuf + (long long)r * c.d + f, y);
-            if (cb == group) keep_y[k] = y;
-            const float s0 = warp_sum(xi[k] * y), s1 = warp_sum(y * y), s2 = warp_sum(xi[k] * sv[k]);
-            const float s3 = warp_sum(sv[k] * sv[k]), s4 = warp_sum(xi[k] * xi[k]);
-            if (lane == 0) {
-              float* dst = T->red[quarter][r];
-              dst[0] = s0; dst[1] = s1; dst[2] = s2; dst[3] = s3; dst[4] = s4;
-            }
-          }
+          const float y = (fv && r < J.R) ? res[k] + v[k] : 0.f;
+          if (fv && r < J.R && ncb > 2) __stcg(p.b.Gbuf + (long long)r * c.d + f, y);
+          if (cb == group) keep_y[k] = y;
+          pr[k] = xi[k] * y;
+          pr[16 + k] = y * y;
         }
+        const float tot = warp_reduce32(pr, lane);
+        if (cb * 16 + (lane & 15) < J.R) T->red[quarter][cb * 16 + (lane & 15)][lane >> 4] = tot;
       } else if (P.kind == G_DOWN) {
+        float sq[16];
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
           const int r = cb * 16 + k;
-          if (r >= J.R) break;
-          const float y = fv ? res[k] + v[k] : 0.f;
-          if (fv) {
+          const float y = (fv && r < J.R) ? res[k] + v[k] : 0.f;
+          if (fv && r < J.R) {
             __stcg(J.x_out + r * J.ldo + f, y);
             if (J.norm_next) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
           }
-          if (J.norm_next) {
-            const float s2 = warp_sum(y * y);
-            if (lane == 0) T->red[quarter][r][0] = s2;
-          }
+          sq[k] = y * y;
+        }
+        if (J.norm_next) {
+          const float tot = warp_reduce16(sq, lane);
+          if (lane < 16 && cb * 16 + lane < J.R) T->red[quarter][cb * 16 + lane][0] = tot;
         }
       } else {  // G_HEAD: best logit of this tile per row (lowest index on ties) and sum of exp
 #pragma unroll
@@ -940,11 +1002,63 @@ struct Worker {
     return j == 1 ? J.x_im1 + t * J.x_tok_stride : J.g_prev + ((long long)(j - 1) * J.T + t) * p.c.d;
   }
 
+  static constexpr double COS_FIX = 268435456.0;  // 2^28: sums up to 3e10 with 4e-9 resolution
+  __device__ __forceinline__ static void cos_add(unsigned long long* dst, float part) {
+    const long long q = __double2ll_rn((double)part * COS_FIX);
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(dst), "l"(q) : "memory");
+  }
+
+  // This CTA's share of the three sums of Eq. 2 that do not involve a layer output, for the step of
+  // job `tgt` with `rows` candidate rows: x.s, s.s and x.x, where x = x_new[t] is that step's objective
+  // row and s the skip candidate of state j: x_old[t] for j = 1, else g[j - 1][t].  They are added
+  // to the job's accumulators as soon as the candidates exist, off the step's critical path.
+  __device__ void pre_sums(int tgt, int rows, int Tn, const float* x_new, const float* x_old, long long xs,
+                           const float* g, bool fv, int f) {
+    const Cfg& c = p.c;
+    RedTables* T = tables();
+    const int quarter = ww & 3, group = ww >> 2;
+    const int ncb = (rows + 15) >> 4;
+    for (int cb = group; cb < ncb; cb += 2) {
+      float pa[32], pb[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int r = cb * 16 + k;
+        float xv = 0.f, sv = 0.f;
+        if (fv && r < rows) {
+          const int j = r / Tn + 1, t = r % Tn;
+          xv = __ldg(x_new + t * xs + f);
+          sv = __ldcg((j == 1 ? x_old + t * xs : g + ((long long)(j - 1) * Tn + t) * c.d) + f);
+        }
+        pa[k] = xv * sv;
+        pa[16 + k] = sv * sv;
+        pb[k] = xv * xv;
+      }
+      const float ta = warp_reduce32(pa, lane);
+      const float tb = warp_reduce16(pb, lane);
+      const int r = cb * 16 + (lane & 15);
+      if (r < rows) {
+        T->red[quarter][r][2 + (lane >> 4)] = ta;
+        if (lane < 16) T->red[quarter][r][4] = tb;
+      }
+    }
+    worker_sync();
+    unsigned long long* acc =
+        reinterpret_cast<unsigned long long*>(p.b.cosacc) + (long long)tgt * ((long long)(c.Rcap + MAX_ROWS) * 5);
+    for (int idx = wtid; idx < rows * 3; idx += WORKERS) {
+      const int r = idx / 3, k = 2 + idx % 3;
+      cos_add(acc + r * 5 + k, T->red[0][r][k] + T->red[1][r][k] + T->red[2][r][k] + T->red[3][r][k]);
+    }
+    worker_sync();  // the tables are reused
+  }
+
   // ---- Eq. 2 step i over this CTA's slice of the d features (thread <-> feature as in the
   // epilogue):
-  //   (1) per-CTA partial dot products, added to the job's fixed-point accumulators, publish;
-  //   (2) wait for every CTA, read the totals, decide (every CTA decides alike);
-  //   (3) write this CTA's slice of g[i][.] and of the next step's operand, publish.
+  //   (1) this CTA's share of x.y and y.y goes to the job's fixed-point accumulators, publish;
+  //   (2) wait for every CTA, read the totals, decide (every CTA decides alike); the chosen row's
+  //       sum of squares is also the next layer's norm factor;
+  //   (3) write this CTA's slice of the next layer's operand, publish;
+  //   (4) off the critical path: this CTA's slice of g[i][.], and its share of the next step's sums
+  //       over the skip candidates.
   // from_epilogue: the down product's epilogue left the partials of this CTA in the tables and
   // the thread's layer outputs / skip candidates of its first row block in keep_y / keep_s.
   __device__ bool dp_step(const Job& J, int jb, bool from_epilogue, float (&keep_y)[16], float (&keep_s)[16]) {
@@ -958,44 +1072,22 @@ struct Worker {
     const int n_states = J.ell + (J.diag ? 1 : 0);
     const int rows = n_states * J.T;
     const int ncb = (rows + 15) >> 4;
-    const long long cstride = (long long)(c.Rcap + MAX_ROWS) * 5;
-    constexpr double COS_FIX = 268435456.0;  // 2^28: sums up to 3e10 with 4e-9 resolution
+    unsigned long long* acc =
+        reinterpret_cast<unsigned long long*>(p.b.cosacc) + (long long)jb * ((long long)(c.Rcap + MAX_ROWS) * 5);
+    if (jb == 0) pre_sums(0, rows, J.T, J.x_i, J.x_im1, J.x_tok_stride, J.g_prev, fv, f);  // nobody prepared the first step
     if (!from_epilogue) {
-      // (1) no layer ran for this CTA's features: only skip candidates exist
-      for (int cb = group; cb < ncb; cb += 2) {
-        float xi[16], sv[16];
+      // no layer ran for this CTA's features: only skip candidates exist
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
-          xi[k] = 0.f;
-          sv[k] = 0.f;
-          if (fv && r < rows) {
-            xi[k] = __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f);
-            sv[k] = __ldcg(skip_src(J, r / J.T + 1, r % J.T) + f);
-          }
-          if (cb == group) { keep_s[k] = sv[k]; keep_y[k] = 0.f; }
-        }
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
-          if (r < rows) {
-            const float s2 = warp_sum(xi[k] * sv[k]), s3 = warp_sum(sv[k] * sv[k]), s4 = warp_sum(xi[k] * xi[k]);
-            if (lane == 0) {
-              float* dst = T->red[quarter][r];
-              dst[0] = 0.f; dst[1] = 0.f; dst[2] = s2; dst[3] = s3; dst[4] = s4;
-            }
-          }
-        }
+      for (int k = 0; k < 16; ++k) {
+        const int r = group * 16 + k;
+        keep_y[k] = 0.f;
+        keep_s[k] = (fv && r < rows) ? __ldcg(skip_src(J, r / J.T + 1, r % J.T) + f) : 0.f;
       }
-    }
-    worker_sync();
-    // this CTA's share of every dot product goes into the job's accumulators
-    unsigned long long* acc = reinterpret_cast<unsigned long long*>(p.b.cosacc) + (long long)jb * cstride;
-    for (int idx = wtid; idx < rows * 5; idx += WORKERS) {
-      const int r = idx / 5, k = idx % 5;
-      const float part = T->red[0][r][k] + T->red[1][r][k] + T->red[2][r][k] + T->red[3][r][k];
-      const long long q = __double2ll_rn((double)part * COS_FIX);
-      asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(acc + idx), "l"(q) : "memory");
+    } else {
+      for (int idx = wtid; idx < J.R * 2; idx += WORKERS) {
+        const int r = idx >> 1, k = idx & 1;
+        cos_add(acc + r * 5 + k, T->red[0][r][k] + T->red[1][r][k] + T->red[2][r][k] + T->red[3][r][k]);
+      }
     }
     publish(F_DOWN, jb + 1);
     mark(T_DP_PUB);
@@ -1021,6 +1113,10 @@ struct Worker {
         if (J.forced && J.forced[j] != 255) take = (J.forced[j] == 0);
       }
       sh->choice[j] = take;
+      for (int t = 0; t < J.T; ++t) {
+        const double* v = T->cosv[(j - 1) * J.T + t];
+        sh->rs_next[(j - 1) * J.T + t] = rsqrtf((float)(take ? v[1] : v[3]) / (float)c.d + c.eps);
+      }
       if (blockIdx.x == 0) {
         J.D[j] = take ? s_app : s_skip;
         J.choice[j] = take ? 0 : 1;
@@ -1033,44 +1129,47 @@ struct Worker {
     }
     worker_sync();
     mark(T_DP_DECIDED);
-    // (3) write-back: the first block of rows comes from registers
+    // (3) the next layer's operand: the first block of rows comes from registers
     const float wn = (fv && J.norm_next) ? __ldg(J.norm_next + f) : 0.f;
-    for (int cb = group; cb < ncb; cb += 2) {
-      float y16[16];
+    float y16[16];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        const int r = cb * 16 + k;
-        y16[k] = 0.f;
-        if (fv && r < rows) {
-          const int j = r / J.T + 1, t = r % J.T;
-          if (cb == group) y16[k] = sh->choice[j] ? keep_y[k] : keep_s[k];
-          else y16[k] = sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f);
-        }
-      }
+    for (int k = 0; k < 16; ++k) {
+      const int r = group * 16 + k;
+      y16[k] = 0.f;
+      if (fv && r < rows) y16[k] = sh->choice[r / J.T + 1] ? keep_y[k] : keep_s[k];
+    }
+    if (J.norm_next && fv) {
+      for (int cb = group; cb < ncb; cb += 2) {
 #pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        const int r = cb * 16 + k;
-        if (r < rows) {
-          const int j = r / J.T + 1, t = r % J.T;
-          const float y = y16[k];
-          if (fv) {
-            __stcg(J.g_next + ((long long)j * J.T + t) * c.d + f, y);
-            if (J.g_final && j == J.M) J.g_final[(long long)t * c.d + f] = y;
-            if (J.norm_next) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
-          }
-          if (J.norm_next) {
-            const float s2 = warp_sum(y * y);
-            if (lane == 0) T->red[quarter][r][0] = s2;
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          if (r < rows) {
+            const int j = r / J.T + 1, t = r % J.T;
+            const float y = cb == group ? y16[k]
+                                        : (sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f));
+            p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
           }
         }
       }
     }
-    worker_sync();
-    if (J.norm_next)
-      for (int r = wtid; r < rows; r += WORKERS)
-        ss_add(p.b.ss_a + (long long)(jb + 1) * c.Rcap + r,
-               T->red[0][r][0] + T->red[1][r][0] + T->red[2][r][0] + T->red[3][r][0]);
     publish(F_SELECT, jb + 1);
+    // (4) g[i][.] for the next step (read back only by this thread: same feature in every step)
+    if (fv) {
+      for (int cb = group; cb < ncb; cb += 2) {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          if (r < rows) {
+            const int j = r / J.T + 1, t = r % J.T;
+            const float y = cb == group ? y16[k]
+                                        : (sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f));
+            __stcg(J.g_next + ((long long)j * J.T + t) * c.d + f, y);
+            if (J.g_final && j == J.M) J.g_final[(long long)t * c.d + f] = y;
+          }
+        }
+      }
+    }
+    if (J.x_ip1) pre_sums(jb + 1, min(J.i + 1, J.M) * J.T, J.T, J.x_ip1, J.x_i, J.x_tok_stride, J.g_next, fv, f);
     return true;
   }
 

@@ -17,10 +17,10 @@
 //               the weight rows once the CTAs that produce those columns have published them.
 //   warps 2, 3  lane 0 of each issues tcgen05.mma: M = 128 weight rows (rows beyond the CTA's
 //               range are whatever bytes follow in the ring; their accumulator lanes are never
-//               read), N = BN activation rows, K = 16.  One thread can issue an MMA only every
-//               ~55 cycles while the tensor pipe takes ~39 for this shape, so the two warps take
-//               alternate ring items and accumulate into separate accumulators, which the
-//               epilogue adds in a fixed order.  Warp 3 also allocates / frees tensor memory.
+//               read; tiles of at most 64 rows use M = 64), N = BN activation rows, K = 16.  One
+//               thread can issue an MMA only every ~55 cycles, so the two warps take alternate
+//               ring items and accumulate into separate accumulators, which the epilogue adds in
+//               a fixed order.  Warp 3 also allocates / frees tensor memory.
 //   warps 4-11  "workers": epilogues, attention, Eq. 2 select, arg-max.
 //
 // Synchronisation between CTAs is through global memory: after finishing step s of job j a
@@ -594,7 +594,7 @@ __device__ __forceinline__ void issuer_mark(const Params& p, int jb, int slot) {
 // b * 256 + a * (dual + 1) * BN  (gate at +0, up at +BN).
 __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint32_t tmem_base, int which) {
   const Cfg& c = p.c;
-  const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.BN >> 3) << 17) | (8u << 24);
+  const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.BN >> 3) << 17);
   const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
   RingPos rp{0, 0};
   const int b_pages = (c.BN * BK * 2) / PAGE;
@@ -610,6 +610,9 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
         const int a_pages = td.n_rows >> 3;
         const int w_pages = (P.dual + 1) * a_pages;
         const int pages = P.kpi * (w_pages + b_pages);
+        // tiles of at most 64 weight rows take the M = 64 shape: the multiply reads half the operand
+        // rows from shared memory (row r of its accumulator sits in lane 32 (r / 16) + r % 16)
+        const uint32_t idesc = idesc0 | ((td.n_rows <= 64 ? 4u : 8u) << 24);
         const uint32_t buf = n_acc & 1u;
         if (!wait_bar(&sh->acc_empty[buf], ((n_acc >> 1) & 1u) ^ 1u, p.ctl, sh)) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -707,6 +710,12 @@ struct Worker {
     return worker_and(ok);
   }
 
+  // Feature (row of an accumulator of n rows) that thread `lane` of lane quarter `quarter` owns, or -1:
+  // an M = 128 accumulator has row r in lane r, an M = 64 one (n <= 64) in lane 32 (r / 16) + r % 16.
+  __device__ __forceinline__ static int feat_local(int n, int quarter, int lane) {
+    const int fl = n <= 64 ? (lane < 16 ? quarter * 16 + lane : n) : quarter * 32 + lane;
+    return fl < n ? fl : -1;
+  }
   __device__ __forceinline__ const int* split_lo(int split) const { return p.tabs + p.c.split_lo[split]; }
   __device__ __forceinline__ RedTables* tables() const { return reinterpret_cast<RedTables*>(scratch); }
 
@@ -788,8 +797,8 @@ struct Worker {
     const Cfg& c = p.c;
     RedTables* T = tables();
     const int quarter = ww & 3, group = ww >> 2;
-    const int fl = quarter * 32 + lane;
-    const bool fv = fl < td.n_rows;
+    const int fl = feat_local(td.n_rows, quarter, lane);
+    const bool fv = fl >= 0;
     const int f = td.f0 + fl;
     const bool dpd = P.kind == G_DOWN && J.dp;
     const int rows_all = J.R + ((dpd && J.diag) ? J.T : 0);   // Eq. 2: plus the rows of the diagonal state
@@ -827,7 +836,9 @@ struct Worker {
       else if (P.kind == G_DOWN && !J.dp && J.norm_next) wn = __ldg(J.norm_next + f);
     }
     const uint32_t buf = n_acc & 1u;
-    bool ok = wait_bar(&sh->acc_full[buf], (n_acc >> 1) & 1u, p.ctl, sh);
+    // one thread polls the barrier, the others sleep in the hardware barrier behind it
+    bool ok = true;
+    if (wtid == 0) ok = wait_bar(&sh->acc_full[buf], (n_acc >> 1) & 1u, p.ctl, sh);
     ok = worker_and(ok);
     if (!ok) return false;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -1066,8 +1077,8 @@ struct Worker {
     RedTables* T = tables();
     const int f_lo = __ldg(split_lo(S_D) + blockIdx.x), f_hi = __ldg(split_lo(S_D) + blockIdx.x + 1);
     const int quarter = ww & 3, group = ww >> 2;
-    const int fl = quarter * 32 + lane;
-    const bool fv = fl < f_hi - f_lo;   // a slice has at most 128 features (checked on the host)
+    const int fl = feat_local(f_hi - f_lo, quarter, lane);   // a slice has at most 128 features (checked on the host)
+    const bool fv = fl >= 0;
     const int f = f_lo + fl;
     const int n_states = J.ell + (J.diag ? 1 : 0);
     const int rows = n_states * J.T;

@@ -268,7 +268,8 @@ int64_t clasp_launch_count(const clasp_ctx* ctx);
  * Eq. 2 step, then the LM head; s: 0 job start, 1 q/k/v done, 2-5 attention partials, 6
  * attention merged, 7 o, 8 gate/up, 9 down, 10-13 Eq. 2 step, 14 head; for product p = 0..3
  * (q/k/v, o, gate/up, down) 16+p first operands ready for the tensor core, 20+p last
- * multiply issued, 24+p first accumulator complete; entries a CTA does
+ * multiply issued, 24+p first accumulator complete; 28 Eq. 2 step published the next operand;
+ * 29-31 operand of q/k/v, o, gate/up seen complete by the operand loader; entries a CTA does
  * not reach stay as the caller left them, entries beyond cap_per_cta are not recorded).  *n_ctas (HOST, may be NULL) receives the grid
  * size, 0 when the context does not use the persistent kernel. */
 int clasp_engine_trace(clasp_ctx* ctx, uint64_t* stamps, int32_t cap_per_cta, int32_t* n_ctas);

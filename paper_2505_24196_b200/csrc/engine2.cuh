@@ -69,7 +69,10 @@ enum { T_START = 0, T_QKV, T_ATT_READY, T_ATT_Q, T_ATT_TILES, T_ATT_PUB, T_MERGE
        T_DP_ALL, T_DP_DECIDED, T_DP_DONE, T_HEAD,
        // per product ph = 0..3 (q/k/v, o, gate/up, down): first ring item of the product ready for the MMA issuer,
        // its last MMA issued, and the product's first accumulator complete (seen by the workers)
-       T_MMA_FIRST = 16, T_MMA_LAST = 20, T_ACC = 24 };
+       T_MMA_FIRST = 16, T_MMA_LAST = 20, T_ACC = 24,
+       // the Eq. 2 step has published the next layer's operand; the operand producer has seen the operands
+       // of the q/k/v, o and gate/up products complete
+       T_SEL_PUB = 28, T_B_READY = 29 };
 constexpr int TRACE_SLOTS = 32;  // time stamps per job
 
 struct TileDesc {      // one accumulator's worth of a CTA's feature range: rows y0.. of one weight matrix
@@ -235,6 +238,15 @@ __device__ __forceinline__ uint2 pack4(float a, float b, float c2, float d2) {
   u.y = *reinterpret_cast<uint32_t*>(&hi);
   return u;
 }
+
+// r / T and r % T for the small row counts of a job (r * T < 65536) without the integer-division sequence
+struct RowDiv {
+  unsigned inv;
+  int T;
+  __device__ __forceinline__ explicit RowDiv(int t) : inv((65536u + (unsigned)t - 1u) / (unsigned)t), T(t) {}
+  __device__ __forceinline__ int div(int r) const { return (int)(((unsigned)r * inv) >> 16); }
+  __device__ __forceinline__ int mod(int r) const { return r - div(r) * T; }
+};
 
 // tcgen05.mma with the operand descriptors given by their low words (start address and leading
 // byte offset; the high word -- 1024-byte group stride, version, 128B swizzle -- is the same for
@@ -510,6 +522,15 @@ __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base, int 
   }
 }
 
+__device__ __forceinline__ void issuer_mark(const Params& p, int jb, int slot) {
+  const int idx = jb * TRACE_SLOTS + slot;
+  if (p.trace != nullptr && idx < p.trace_cap) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    p.trace[(long long)blockIdx.x * p.trace_cap + idx] = t;
+  }
+}
+
 // Warp 1, all lanes: lane k issues the operand tile of an item's chunk k.
 __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, const CUtensorMap* const* bmaps,
                            const CUtensorMap* const* bmaps3, int lane) {
@@ -538,6 +559,7 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
         bool ok = true;
         if (lane == 0) ok = wait_count(p, fkind, tgt, sh);
         if (!__all_sync(0xffffffffu, ok)) return;
+        if (lane == 0 && P.kind < 3) issuer_mark(p, jb, T_B_READY + P.kind);
       }
       fence_proxy_async();  // the producers' ordinary stores before this warp's TMA reads
       const bool d3 = c.use3d[P.kind] != 0;
@@ -577,15 +599,6 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
         }
       }
     }
-  }
-}
-
-__device__ __forceinline__ void issuer_mark(const Params& p, int jb, int slot) {
-  const int idx = jb * TRACE_SLOTS + slot;
-  if (p.trace != nullptr && idx < p.trace_cap) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    p.trace[(long long)blockIdx.x * p.trace_cap + idx] = t;
   }
 }
 
@@ -804,6 +817,7 @@ struct Worker {
     const int rows_all = J.R + ((dpd && J.diag) ? J.T : 0);   // Eq. 2: plus the rows of the diagonal state
     const int ncb = (J.R + 15) >> 4;
     const bool resid = P.kind == G_O || P.kind == G_DOWN;
+    const RowDiv rd(J.T);
     // Eq. 2: objective row and skip candidate of every row of the first block, fetched early
     float xi[16];
     if (dpd) {
@@ -814,8 +828,8 @@ struct Worker {
         keep_s[k] = 0.f;
         keep_y[k] = 0.f;
         if (fv && r < rows_all) {
-          xi[k] = __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f);
-          keep_s[k] = __ldcg(skip_src(J, r / J.T + 1, r % J.T) + f);
+          xi[k] = __ldg(J.x_i + rd.mod(r) * J.x_tok_stride + f);
+          keep_s[k] = __ldcg(skip_src(J, rd.div(r) + 1, rd.mod(r)) + f);
         }
       }
     }
@@ -916,7 +930,7 @@ struct Worker {
 #pragma unroll
           for (int k = 0; k < 16; ++k) {
             const int r = cb * 16 + k;
-            xi[k] = (fv && r < J.R) ? __ldg(J.x_i + (r % J.T) * J.x_tok_stride + f) : 0.f;
+            xi[k] = (fv && r < J.R) ? __ldg(J.x_i + rd.mod(r) * J.x_tok_stride + f) : 0.f;
           }
         }
         float pr[32];
@@ -1029,6 +1043,7 @@ struct Worker {
     RedTables* T = tables();
     const int quarter = ww & 3, group = ww >> 2;
     const int ncb = (rows + 15) >> 4;
+    const RowDiv rd(Tn);
     for (int cb = group; cb < ncb; cb += 2) {
       float pa[32], pb[16];
 #pragma unroll
@@ -1036,7 +1051,7 @@ struct Worker {
         const int r = cb * 16 + k;
         float xv = 0.f, sv = 0.f;
         if (fv && r < rows) {
-          const int j = r / Tn + 1, t = r % Tn;
+          const int j = rd.div(r) + 1, t = rd.mod(r);
           xv = __ldg(x_new + t * xs + f);
           sv = __ldcg((j == 1 ? x_old + t * xs : g + ((long long)(j - 1) * Tn + t) * c.d) + f);
         }
@@ -1085,6 +1100,8 @@ struct Worker {
     const int ncb = (rows + 15) >> 4;
     unsigned long long* acc =
         reinterpret_cast<unsigned long long*>(p.b.cosacc) + (long long)jb * ((long long)(c.Rcap + MAX_ROWS) * 5);
+    const RowDiv rd(J.T);
+    const float wn = (fv && J.norm_next) ? __ldg(J.norm_next + f) : 0.f;   // needed right after the decision
     if (jb == 0) pre_sums(0, rows, J.T, J.x_i, J.x_im1, J.x_tok_stride, J.g_prev, fv, f);  // nobody prepared the first step
     if (!from_epilogue) {
       // no layer ran for this CTA's features: only skip candidates exist
@@ -1092,7 +1109,7 @@ struct Worker {
       for (int k = 0; k < 16; ++k) {
         const int r = group * 16 + k;
         keep_y[k] = 0.f;
-        keep_s[k] = (fv && r < rows) ? __ldcg(skip_src(J, r / J.T + 1, r % J.T) + f) : 0.f;
+        keep_s[k] = (fv && r < rows) ? __ldcg(skip_src(J, rd.div(r) + 1, rd.mod(r)) + f) : 0.f;
       }
     } else {
       for (int idx = wtid; idx < J.R * 2; idx += WORKERS) {
@@ -1110,14 +1127,15 @@ struct Worker {
     worker_sync();
     if (wtid < n_states) {
       const int j = wtid + 1;
-      double app = 0.0, skp = 0.0;
+      // the sums are exact to the fixed-point step; the few operations on them run in float
+      float app = 0.f, skp = 0.f;
       for (int t = 0; t < J.T; ++t) {
         const double* v = T->cosv[(j - 1) * J.T + t];
-        const double nx = fmax(sqrt(v[4]), 1e-12);
-        app += v[0] / (nx * fmax(sqrt(v[1]), 1e-12));
-        skp += v[2] / (nx * fmax(sqrt(v[3]), 1e-12));
+        const float nx = fmaxf(sqrtf((float)v[4]), 1e-12f);
+        app += (float)v[0] / (nx * fmaxf(sqrtf((float)v[1]), 1e-12f));
+        skp += (float)v[2] / (nx * fmaxf(sqrtf((float)v[3]), 1e-12f));
       }
-      const float s_app = (float)(app / J.T), s_skip = (float)(skp / J.T);
+      const float s_app = app / (float)J.T, s_skip = skp / (float)J.T;
       int take = 0;
       if (j <= J.ell) {
         take = s_app > s_skip;
@@ -1141,13 +1159,12 @@ struct Worker {
     worker_sync();
     mark(T_DP_DECIDED);
     // (3) the next layer's operand: the first block of rows comes from registers
-    const float wn = (fv && J.norm_next) ? __ldg(J.norm_next + f) : 0.f;
     float y16[16];
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
       const int r = group * 16 + k;
       y16[k] = 0.f;
-      if (fv && r < rows) y16[k] = sh->choice[r / J.T + 1] ? keep_y[k] : keep_s[k];
+      if (fv && r < rows) y16[k] = sh->choice[rd.div(r) + 1] ? keep_y[k] : keep_s[k];
     }
     if (J.norm_next && fv) {
       for (int cb = group; cb < ncb; cb += 2) {
@@ -1155,7 +1172,7 @@ struct Worker {
         for (int k = 0; k < 16; ++k) {
           const int r = cb * 16 + k;
           if (r < rows) {
-            const int j = r / J.T + 1, t = r % J.T;
+            const int j = rd.div(r) + 1, t = rd.mod(r);
             const float y = cb == group ? y16[k]
                                         : (sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f));
             p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
@@ -1164,6 +1181,7 @@ struct Worker {
       }
     }
     publish(F_SELECT, jb + 1);
+    mark(T_SEL_PUB);
     // (4) g[i][.] for the next step (read back only by this thread: same feature in every step)
     if (fv) {
       for (int cb = group; cb < ncb; cb += 2) {
@@ -1171,7 +1189,7 @@ struct Worker {
         for (int k = 0; k < 16; ++k) {
           const int r = cb * 16 + k;
           if (r < rows) {
-            const int j = r / J.T + 1, t = r % J.T;
+            const int j = rd.div(r) + 1, t = rd.mod(r);
             const float y = cb == group ? y16[k]
                                         : (sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f));
             __stcg(J.g_next + ((long long)j * J.T + t) * c.d + f, y);
@@ -1208,6 +1226,32 @@ struct Worker {
     const long long kvld = c.kvd;
     const int qkvd = c.qd + 2 * c.kvd;
     const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;
+    const RowDiv rdT(J.T);
+    // The cache does not depend on this layer's projections: the first K/V tile of this CTA's first
+    // item is on its way from HBM while the CTA waits for them.
+    constexpr int FILL = ATT_KEYS * (HD / 8) / WORKERS;   // 16-byte pieces of a tile per thread
+    static_assert(FILL * WORKERS == ATT_KEYS * (HD / 8), "tile pieces must divide among the workers");
+    uint4 pre_k[FILL], pre_v[FILL];
+    bool pre_ok = false;
+    if ((int)blockIdx.x < n_items) {
+      const int chunk = ((int)blockIdx.x / n_pbg) % n_chunks;
+      const int kvh = (int)blockIdx.x / (n_pbg * n_chunks);
+      if (chunk < n_runs) {
+        const int key_lo = chunk * c.run_len;
+        pre_ok = true;
+#pragma unroll
+        for (int e = 0; e < FILL; ++e) {
+          const int vv = wtid + e * WORKERS;
+          const int key = key_lo + vv / (HD / 8), cv8 = vv % (HD / 8);
+          pre_k[e] = make_uint4(0, 0, 0, 0);
+          pre_v[e] = make_uint4(0, 0, 0, 0);
+          if (key < J.C) {   // positions this launch never writes
+            pre_k[e] = __ldcg(reinterpret_cast<const uint4*>(J.ck + (long long)key * kvld + kvh * HD + cv8 * 8));
+            pre_v[e] = __ldcg(reinterpret_cast<const uint4*>(J.cv + (long long)key * kvld + kvh * HD + cv8 * 8));
+          }
+        }
+      }
+    }
     // every row's q, k, v exist once all CTAs have published their slice of the projections
     if (!wait_all(F_QKV, J.tgt[F_QKV])) return false;
     mark(T_ATT_READY);
@@ -1218,7 +1262,7 @@ struct Worker {
       const bool own = chunk >= n_runs;
       const int p0 = (pbg * 8 + ww) * 16;
       const bool active = p0 < Pn;
-      int rr[2], hq[2];
+      int rr[2], hq[2], tq[2], sq[2];   // row, query head, position and state of the row
       bool pv[2];
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
@@ -1226,28 +1270,46 @@ struct Worker {
         pv[h] = pp < Pn;
         rr[h] = pv[h] ? pp / Gq : 0;
         hq[h] = kvh * Gq + (pv[h] ? pp % Gq : 0);
+        sq[h] = rdT.div(rr[h]);
+        tq[h] = rr[h] - sq[h] * J.T;
       }
       // q fragments, rotated.  Element i of the first half pairs with element i + HD/2: one load
       // of each gives the rotated values of both, i.e. the fragments of k-steps ks and ks + KS/2.
       uint32_t qh[KS][4], ql[KS][4];
+      {
+        // all loads first (one trip to L2), then the rotation
+        float2 raw_lo[KS / 2][4], raw_hi[KS / 2][4];
 #pragma unroll
-      for (int ks = 0; ks < KS / 2; ++ks) {
+        for (int ks = 0; ks < KS / 2; ++ks) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+          for (int h = 0; h < 2; ++h) {
 #pragma unroll
-          for (int kh = 0; kh < 2; ++kh) {
-            float2 v0 = make_float2(0.f, 0.f), v1 = v0;
-            if (active && pv[h]) {
-              const int i = ks * 16 + kh * 8 + c4 * 2;           // dims i, i + 1 of the first half
-              const float* qr = p.b.qkv + (long long)rr[h] * qkvd + hq[h] * HD;
-              const float2 lo2 = __ldcg(reinterpret_cast<const float2*>(qr + i));
-              const float2 hi2 = __ldcg(reinterpret_cast<const float2*>(qr + i + HALF));
-              const float4 cs = *reinterpret_cast<const float4*>(p.b.rope + (long long)(rr[h] % J.T) * HALF + i);
-              v0 = make_float2((lo2.x * cs.x - hi2.x * cs.y) * qscale, (lo2.y * cs.z - hi2.y * cs.w) * qscale);
-              v1 = make_float2((hi2.x * cs.x + lo2.x * cs.y) * qscale, (hi2.y * cs.z + lo2.y * cs.w) * qscale);
+            for (int kh = 0; kh < 2; ++kh) {
+              raw_lo[ks][h + kh * 2] = make_float2(0.f, 0.f);
+              raw_hi[ks][h + kh * 2] = make_float2(0.f, 0.f);
+              if (active && pv[h]) {
+                const int i = ks * 16 + kh * 8 + c4 * 2;           // dims i, i + 1 of the first half
+                const float* qr = p.b.qkv + (long long)rr[h] * qkvd + hq[h] * HD;
+                raw_lo[ks][h + kh * 2] = __ldcg(reinterpret_cast<const float2*>(qr + i));
+                raw_hi[ks][h + kh * 2] = __ldcg(reinterpret_cast<const float2*>(qr + i + HALF));
+              }
             }
-            split2(v0.x, v0.y, qh[ks][h + kh * 2], ql[ks][h + kh * 2]);
-            split2(v1.x, v1.y, qh[ks + KS / 2][h + kh * 2], ql[ks + KS / 2][h + kh * 2]);
+          }
+        }
+#pragma unroll
+        for (int ks = 0; ks < KS / 2; ++ks) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+              const int i = ks * 16 + kh * 8 + c4 * 2;
+              const float2 lo2 = raw_lo[ks][h + kh * 2], hi2 = raw_hi[ks][h + kh * 2];
+              const float4 cs = *reinterpret_cast<const float4*>(p.b.rope + (long long)tq[h] * HALF + i);
+              const float2 v0 = make_float2((lo2.x * cs.x - hi2.x * cs.y) * qscale, (lo2.y * cs.z - hi2.y * cs.w) * qscale);
+              const float2 v1 = make_float2((hi2.x * cs.x + lo2.x * cs.y) * qscale, (hi2.y * cs.z + lo2.y * cs.w) * qscale);
+              split2(v0.x, v0.y, qh[ks][h + kh * 2], ql[ks][h + kh * 2]);
+              split2(v1.x, v1.y, qh[ks + KS / 2][h + kh * 2], ql[ks + KS / 2][h + kh * 2]);
+            }
           }
         }
       }
@@ -1264,15 +1326,23 @@ struct Worker {
         const int nkeys = min(ATT_KEYS, key_hi - key0);
         worker_sync();  // previous tile consumed
         // K/V tile: cache rows as they are; rows of this call rotated / rounded from the projections
-        for (int vv = wtid; vv < ATT_KEYS * (HD / 8); vv += WORKERS) {
+        const bool use_pre = pre_ok && it == (int)blockIdx.x && key0 == key_lo;
+#pragma unroll
+        for (int e = 0; e < FILL; ++e) {
+          const int vv = wtid + e * WORKERS;
           const int row = vv / (HD / 8), cv8 = vv % (HD / 8);
           uint4 kk = make_uint4(0, 0, 0, 0), vq = make_uint4(0, 0, 0, 0);
           if (row < nkeys) {
             const int key = key0 + row;
             const int new_row = own ? key : (J.uniform ? key - J.C : -1);
             if (new_row < 0) {
-              kk = __ldcg(reinterpret_cast<const uint4*>(J.ck + (long long)key * kvld + kvh * HD + cv8 * 8));
-              vq = __ldcg(reinterpret_cast<const uint4*>(J.cv + (long long)key * kvld + kvh * HD + cv8 * 8));
+              if (use_pre) {
+                kk = pre_k[e];
+                vq = pre_v[e];
+              } else {
+                kk = __ldcg(reinterpret_cast<const uint4*>(J.ck + (long long)key * kvld + kvh * HD + cv8 * 8));
+                vq = __ldcg(reinterpret_cast<const uint4*>(J.cv + (long long)key * kvld + kvh * HD + cv8 * 8));
+              }
             } else {
               const float* kr = p.b.qkv + (long long)new_row * qkvd + c.qd + kvh * HD;
               const float* vr = kr + c.kvd;
@@ -1290,7 +1360,7 @@ struct Worker {
               float kro[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e) {
-                const float2 cs = p.b.rope[(long long)(new_row % J.T) * HALF + i0 + e];
+                const float2 cs = p.b.rope[(long long)rdT.mod(new_row) * HALF + i0 + e];
                 kro[e] = d0 < HALF ? ka[e] * cs.x - kb[e] * cs.y : kb[e] * cs.x + ka[e] * cs.y;
               }
               const uint2 k01 = pack4(kro[0], kro[1], kro[2], kro[3]), k23 = pack4(kro[4], kro[5], kro[6], kro[7]);
@@ -1329,7 +1399,7 @@ struct Worker {
             const int h = e >> 1;
             const int key = key0 + nb * 8 + c4 * 2 + (e & 1);
             bool vis = pv[h] && key < key_hi;
-            if (own) vis = vis && (key / J.T == rr[h] / J.T) && key <= rr[h];
+            if (own) vis = vis && (rdT.div(key) == sq[h]) && key <= rr[h];
             else if (J.uniform) vis = vis && key <= J.C + rr[h];
             if (!vis) s[nb][e] = -INFINITY;
             mx[h] = fmaxf(mx[h], s[nb][e]);
@@ -1413,15 +1483,18 @@ struct Worker {
     const int k_tot = J.uniform ? J.C + J.T : J.C;
     const int n_runs = (k_tot + c.run_len - 1) / c.run_len;
     const int n_chunks = n_runs + (J.uniform ? 0 : (J.R + ATT_KEYS - 1) / ATT_KEYS);
-    for (int hq = blockIdx.x; hq < c.nq; hq += c.G) {
-      // the items of this head's kv head ran on CTAs (item index) % G
-      const int kvh = hq / Gq;
-      const int it0 = kvh * n_chunks * n_pbg, n_it = n_chunks * n_pbg;
-      bool ok = true;
-      for (int k = wtid; k < min(n_it, c.G); k += WORKERS)
-        ok = wait_flag(p.b.flags + F_ATTN * c.G + (it0 + k) % c.G, jb + 1, p.ctl, sh) && ok;
-      if (!worker_and(ok)) return false;
-      for (int r = ww; r < J.R; r += 8) {
+    // One warp per (row, head) pair; the pairs are dealt out to all CTAs and, inside a CTA, to its warps.
+    bool all_ok = true;
+    for (int u = (int)blockIdx.x + c.G * ww; u < J.R * c.nq; u += c.G * 8) {
+      const int r = u / c.nq, hq = u - r * c.nq;
+      {
+        // the items of this head's kv head ran on CTAs (item index) % G
+        const int kvh = hq / Gq;
+        const int it0 = kvh * n_chunks * n_pbg, n_it = n_chunks * n_pbg;
+        bool ok = true;
+        for (int k = lane; k < min(n_it, c.G); k += 32)
+          ok = wait_flag(p.b.flags + F_ATTN * c.G + (it0 + k) % c.G, jb + 1, p.ctl, sh) && ok;
+        if (!__all_sync(0xffffffffu, ok)) { all_ok = false; break; }
         const long long pr = (long long)r * c.nq + hq;
         const float2* ml = p.b.att_ml + pr * c.chunk_cap;
         float2 v0 = make_float2(-INFINITY, 0.f), v1 = v0;
@@ -1470,6 +1543,7 @@ struct Worker {
         }
       }
     }
+    if (!worker_and(all_ok)) return false;
     publish(F_MERGE, jb + 1);
     return true;
   }

@@ -603,8 +603,15 @@ int engine_setup(clasp_ctx* ctx) {
       for (int h = 0; h < pk::N_HEIGHTS; ++h) ctx->e_heights[5][h] = ctx->e_heights[4][h];
     const int a_pages = (k == pk::G_GU ? 2 : 1) * (max_rows / 8);
     ctx->e_wpages[k] = a_pages;   // weight pages of one chunk of the kind's tallest tile
-    int kpi = 16 / a_pages;
-    ctx->e_kpi[k] = kpi < 1 ? 1 : (kpi > 4 ? 4 : kpi);
+    // ring items of about 32 KB of weights: every item costs the MMA issuers a barrier round trip, so
+    // small items waste issue time, while items beyond a sixth of the ring leave too few in flight
+    int kpi_budget = 32, kpi_max = 8;
+    if (const char* e = getenv("CLASP_ENGINE_KPI")) {
+      const int v = atoi(e);
+      if (v >= 4 && v <= 48) { kpi_budget = v; kpi_max = v / 4; }
+    }
+    int kpi = kpi_budget / a_pages;
+    ctx->e_kpi[k] = kpi < 1 ? 1 : (kpi > kpi_max ? kpi_max : kpi);
     // (the gate/up product interleaves two matrices per chunk, which one box cannot deliver)
     ctx->e_use3d[k] = (k != pk::G_GU && kind_K[k] % 64 == 0 && ctx->e_kpi[k] > 1 && !getenv("CLASP_ENGINE_NO3D")) ? 1 : 0;
   }
@@ -671,8 +678,17 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   }
   // an item (gate + up rows and the operand tiles of kpi chunks) must fit the ring twice over
   const int b_pages = BN * pk::BK * 2 / pk::PAGE;
-  for (int k = 0; k < 5; ++k)
-    if (ctx->e_kpi[k] * (ctx->e_wpages[k] + b_pages) * 2 > ring_pages) return CLASP_ERR_CAPACITY;
+  // chunks per ring item in this launch: the set-up value when two such items fit the ring, else fewer,
+  // loaded chunk by chunk through the 2-D maps (the 3-D boxes are built for the set-up value)
+  int kpi[5], use3d[5];
+  for (int k = 0; k < 5; ++k) {
+    kpi[k] = ctx->e_kpi[k];
+    use3d[k] = ctx->e_use3d[k];
+    while (kpi[k] > 1 && kpi[k] * (ctx->e_wpages[k] + b_pages) * 2 > ring_pages) --kpi[k];
+    if (kpi[k] * (ctx->e_wpages[k] + b_pages) * 2 > ring_pages) return CLASP_ERR_CAPACITY;
+    if (kpi[k] != ctx->e_kpi[k]) use3d[k] = 0;
+    if (!use3d[k] && kpi[k] > 16) kpi[k] = 16;   // one lane pair per chunk
+  }
   const size_t dyn = 1024 + (size_t)ring_pages * pk::PAGE + pk::SCRATCH_BYTES;
 
   const int qdim = qd;
@@ -720,7 +736,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   if (getenv("CLASP_ENGINE_ONE_ISSUER")) P.c.n_iss = 1;
 
   for (int s = 0; s < pk::N_SPLITS; ++s) { P.c.split_lo[s] = ctx->e_split_lo[s]; P.c.split_units[s] = ctx->e_split_units[s]; }
-  for (int k = 0; k < 5; ++k) { P.c.tile_idx[k] = ctx->e_tile_idx[k]; P.c.kpi[k] = ctx->e_kpi[k]; P.c.use3d[k] = ctx->e_use3d[k]; }
+  for (int k = 0; k < 5; ++k) { P.c.tile_idx[k] = ctx->e_tile_idx[k]; P.c.kpi[k] = kpi[k]; P.c.use3d[k] = use3d[k]; }
   P.c.tiles_off = ctx->e_tiles_off; P.c.map3d_off = (int)(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS);
   P.b.xn_a = (bf16*)ws.xn; P.b.xn_m = (bf16*)ws.xn_m; P.b.attn = (bf16*)ws.attn; P.b.act = (bf16*)ws.act;
   P.b.qkv = ws.qkv; P.b.x1 = ws.x1; P.b.Gbuf = ws.G; P.b.att_acc = ws.e_att_acc; P.b.att_ml = ws.e_att_ml;

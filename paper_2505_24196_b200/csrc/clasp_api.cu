@@ -188,7 +188,7 @@ struct clasp_ctx {
   int e_heights[8][clasp::pk::N_HEIGHTS];   // tile heights per matrix slot (wq wk wv wo gate up down head)
   std::vector<CUtensorMap> e_wmaps_host;
   bool e_wmaps_dirty = true;
-  std::map<int, std::array<CUtensorMap, 8>> e_bmaps;           // by BN: 2-D maps of the four operands, then 3-D
+  std::map<int, std::array<CUtensorMap, 10>> e_bmaps;          // by BN: 2-D maps of the four operands, then 3-D, then xn with 2 BN rows (2-D, 3-D)
   std::map<std::pair<int, int>, std::array<CUtensorMap, 2>> e_headmaps;  // by (row offset, BN): 2-D, 3-D
   std::vector<clasp::pk::Job> e_jobs;
   unsigned long long* e_trace = nullptr;
@@ -680,12 +680,15 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   const int b_pages = BN * pk::BK * 2 / pk::PAGE;
   // chunks per ring item in this launch: the set-up value when two such items fit the ring, else fewer,
   // loaded chunk by chunk through the 2-D maps (the 3-D boxes are built for the set-up value)
+  bool any_dual = false;
+  for (const pk::Job& J : ctx->e_jobs) any_dual = any_dual || J.dual_src;
   int kpi[5], use3d[5];
   for (int k = 0; k < 5; ++k) {
     kpi[k] = ctx->e_kpi[k];
     use3d[k] = ctx->e_use3d[k];
-    while (kpi[k] > 1 && kpi[k] * (ctx->e_wpages[k] + b_pages) * 2 > ring_pages) --kpi[k];
-    if (kpi[k] * (ctx->e_wpages[k] + b_pages) * 2 > ring_pages) return CLASP_ERR_CAPACITY;
+    const int bp = (k == pk::G_QKV && any_dual ? 2 : 1) * b_pages;
+    while (kpi[k] > 1 && kpi[k] * (ctx->e_wpages[k] + bp) * 2 > ring_pages) --kpi[k];
+    if (kpi[k] * (ctx->e_wpages[k] + bp) * 2 > ring_pages) return CLASP_ERR_CAPACITY;
     if (kpi[k] != ctx->e_kpi[k]) use3d[k] = 0;
     if (!use3d[k] && kpi[k] > 16) kpi[k] = 16;   // one lane pair per chunk
   }
@@ -694,7 +697,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   const int qdim = qd;
   auto bm = ctx->e_bmaps.find(BN);
   if (bm == ctx->e_bmaps.end()) {
-    std::array<CUtensorMap, 8> m{};
+    std::array<CUtensorMap, 10> m{};
     int rc = 0;
     rc |= make_map(ctx, ws.xn, rows_cap, d, BN, &m[0]);
     rc |= make_map(ctx, ws.attn, rows_cap, qdim, BN, &m[1]);
@@ -704,6 +707,10 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
     if (ctx->e_use3d[pk::G_O]) rc |= make_map3(ctx, ws.attn, rows_cap, qdim, BN, ctx->e_kpi[pk::G_O], &m[5]);
     if (ctx->e_use3d[pk::G_GU]) rc |= make_map3(ctx, ws.xn_m, rows_cap, d, BN, ctx->e_kpi[pk::G_GU], &m[6]);
     if (ctx->e_use3d[pk::G_DOWN]) rc |= make_map3(ctx, ws.act, rows_cap, c.d_ffn, BN, ctx->e_kpi[pk::G_DOWN], &m[7]);
+    if (2 * BN <= 256) {
+      rc |= make_map(ctx, ws.xn, rows_cap, d, 2 * BN, &m[8]);
+      if (ctx->e_use3d[pk::G_QKV]) rc |= make_map3(ctx, ws.xn, rows_cap, d, 2 * BN, ctx->e_kpi[pk::G_QKV], &m[9]);
+    }
     if (rc) return CLASP_ERR_CUDA;
     bm = ctx->e_bmaps.emplace(BN, m).first;
   }
@@ -752,7 +759,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   }
   void* args[] = {(void*)&bm->second[0], (void*)&bm->second[1], (void*)&bm->second[2], (void*)&bm->second[3],
                   (void*)&hm->second[0], (void*)&bm->second[4], (void*)&bm->second[5], (void*)&bm->second[6],
-                  (void*)&bm->second[7], (void*)&hm->second[1], (void*)&P};
+                  (void*)&bm->second[7], (void*)&hm->second[1], (void*)&bm->second[8], (void*)&bm->second[9], (void*)&P};
   cudaError_t err = cudaLaunchCooperativeKernel((const void*)pk::engine_kernel, dim3(ctx->e_G), dim3(pk::THREADS),
                                                 args, dyn, ctx->stream);
   if (ctx->profiling) {
@@ -782,7 +789,7 @@ void link_jobs(std::vector<pk::Job>& jobs) {
     int src_tgt = 0, src_flag = pk::F_PREP;
     if (k > 0) {
       const pk::Job& prev = jobs[k - 1];
-      const bool from_select = prev.type == pk::JOB_SELECT || (prev.type == pk::JOB_LAYER && prev.dp);
+      const bool from_select = (prev.type == pk::JOB_SELECT || (prev.type == pk::JOB_LAYER && prev.dp)) && !prev.defer;
       src_flag = from_select ? pk::F_SELECT : pk::F_DOWN;
       src_tgt = n_pub[src_flag];
     }
@@ -790,7 +797,7 @@ void link_jobs(std::vector<pk::Job>& jobs) {
       if (J.prep) ++n_pub[pk::F_PREP];
       ++n_pub[pk::F_QKV]; ++n_pub[pk::F_ATTN]; ++n_pub[pk::F_MERGE]; ++n_pub[pk::F_O]; ++n_pub[pk::F_GU];
       ++n_pub[pk::F_DOWN];
-      if (J.dp) ++n_pub[pk::F_SELECT];
+      if (J.dp && !J.defer) ++n_pub[pk::F_SELECT];
       if (J.prep) { src_flag = pk::F_PREP; src_tgt = n_pub[pk::F_PREP]; }
     } else if (J.type == pk::JOB_SELECT) {
       ++n_pub[pk::F_DOWN]; ++n_pub[pk::F_SELECT];
@@ -994,7 +1001,6 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
       J.i = i; J.ell = ell; J.diag = i <= M ? 1 : 0; J.M = M;
       J.x_i = hidden_states + (int64_t)i * layer_stride;
       J.x_im1 = hidden_states + (int64_t)(i - 1) * layer_stride;
-      J.x_ip1 = i < L ? hidden_states + (int64_t)(i + 1) * layer_stride : nullptr;
       J.x_tok_stride = token_stride;
       J.g_prev = ws.grow[cur]; J.g_next = ws.grow[cur ^ 1];
       J.D = scores + (int64_t)i * (M + 1);
@@ -1006,6 +1012,15 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
       ctx->e_jobs.push_back(J);
       cur ^= 1;
     }
+    // a layer job followed by another layer job hands over both candidates of every state instead of
+    // making the next layer wait for the Eq. 2 decision (needs 2 BN operand rows and accumulator columns)
+    const int BNs = M * T <= 16 ? 16 : (M * T + 15) / 16 * 16;
+    if (2 * BNs <= c.max_rows && 2 * BNs <= 128 && !getenv("CLASP_ENGINE_NODEFER"))
+      for (size_t k = 0; k + 1 < ctx->e_jobs.size(); ++k)
+        if (ctx->e_jobs[k].type == pk::JOB_LAYER && ctx->e_jobs[k + 1].type == pk::JOB_LAYER) {
+          ctx->e_jobs[k].defer = 1;
+          ctx->e_jobs[k + 1].dual_src = 1;
+        }
     link_jobs(ctx->e_jobs);
     if ((rc = engine_launch(ctx, M * T, 0))) return rc;
     clasp::backtrack_kernel<<<1, 32, 0, ctx->stream>>>(ws.choice, L, M, skip_mask);

@@ -137,6 +137,10 @@ struct Job {
   int uniform;   // 1: the rows' K/V go into the cache and attention is causal by position
   int prep;      // 1: build the first operand from x_in when the job starts
   int dp;        // 1: the layer output feeds the Eq. 2 step below
+  int defer;     // 1 (with dp): the next layer does not wait for the Eq. 2 decision.  Its q/k/v product takes
+                 // both candidates of every state -- operand rows [0, BN) the layer outputs (written by the
+                 // down epilogue), rows [BN, 2 BN) the skip candidates -- and its epilogue keeps the chosen one
+  int dual_src;  // 1: this job's q/k/v operand has those two row blocks (the previous job has `defer`)
   int row_off;   // JOB_HEAD: first row (of the previous job's rows) that goes through the head
   int src_flag;  // step kind that publishes this job's first operand (F_PREP / F_DOWN / F_SELECT)
   int src_tgt;   // how often every CTA has published that step once the operand is complete
@@ -154,7 +158,6 @@ struct Job {
   int i, ell, diag, M;
   const float* x_i;
   const float* x_im1;
-  const float* x_ip1;      // objective rows of the next step (null at the last one)
   long long x_tok_stride;
   const float* g_prev;
   float* g_next;
@@ -377,6 +380,9 @@ __device__ __forceinline__ int kind_map_base(const Cfg& c, int kind, int layer) 
 
 struct Phase {   // one product of one job, as seen by this CTA
   int kind, dual, kc, kpi, n_groups;  // chunks, chunks per item, items per tile
+  int bmul;                           // operand row blocks of BN rows (2 for a q/k/v product over both candidates)
+  int width;                          // accumulator columns of one MMA issuer
+  int n_iss;                          // issuers that take items of this product
   int tile0, n_tiles;                 // this CTA's TileDesc range
   int map_base;
   int g0;                             // chunk group this CTA starts its reduction at: CTAs walk the
@@ -389,6 +395,9 @@ struct Phase {   // one product of one job, as seen by this CTA
     kc = (kind_K(c, kind) + BK - 1) / BK;
     kpi = c.kpi[kind];
     n_groups = (kc + kpi - 1) / kpi;
+    bmul = (kind == G_QKV && J.dual_src) ? 2 : 1;
+    width = (dual + 1) * bmul * c.BN;
+    n_iss = 2 * width <= 256 ? c.n_iss : 1;
     const int* ti = p.tabs + c.tile_idx[kind] + blockIdx.x;
     tile0 = __ldg(ti);
     n_tiles = __ldg(ti + 1) - tile0;
@@ -483,7 +492,7 @@ __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base, int 
     const TileDesc& td = L.td;
     const bool d3 = c.use3d[P.kind] != 0;
     const int a_pages = L.a_pages(), w_pages = L.w_pages();
-    const int pages = P.kpi * (w_pages + b_pages);
+    const int pages = P.kpi * (w_pages + P.bmul * b_pages);
     // make room: items leave the ring in the order they entered it
     int fp;
     RingPos probe = rp;
@@ -550,7 +559,7 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
       if (P.n_tiles == 0) continue;
       // the operand exists once every CTA has published the step that writes it
       int fkind, tgt, bmap;
-      if (P.kind == G_QKV) { fkind = J.src_flag; tgt = J.src_tgt; bmap = 0; }
+      if (P.kind == G_QKV) { fkind = J.src_flag; tgt = J.src_tgt; bmap = J.dual_src ? 5 : 0; }
       else if (P.kind == G_O) { fkind = F_MERGE; tgt = J.tgt[F_MERGE]; bmap = 1; }
       else if (P.kind == G_GU) { fkind = F_O; tgt = J.tgt[F_O]; bmap = 2; }
       else if (P.kind == G_DOWN) { fkind = F_GU; tgt = J.tgt[F_GU]; bmap = 3; }
@@ -566,7 +575,8 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
       for (int t = 0; t < P.n_tiles; ++t) {
         const TileDesc td = tiles[P.tile0 + t];
         const int w_pages = (P.dual + 1) * (td.n_rows >> 3);
-        const int pages = P.kpi * (w_pages + b_pages);
+        const int pages = P.kpi * (w_pages + P.bmul * b_pages);
+        const uint32_t pb_bytes = (uint32_t)P.bmul * b_bytes;   // operand tile of one chunk
         for (int gi = 0; gi < P.n_groups; ++gi) {
           int fp;
           const uint32_t it = rp.item;
@@ -587,13 +597,13 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
           const uint32_t dst = ring_base + (uint32_t)(at + P.kpi * w_pages) * PAGE;
           if (d3) {
             if (lane == 0) {
-              tc::mbar_expect_tx(full, (uint32_t)P.kpi * b_bytes);
+              tc::mbar_expect_tx(full, (uint32_t)P.kpi * pb_bytes);
               tma_load_3d(dst, bmaps3[bmap], full, 0, 0, k0, pol);
             }
           } else {
-            if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)nk * b_bytes);
+            if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)nk * pb_bytes);
             __syncwarp();
-            if (lane < nk) tc::tma_load_2d(dst + (uint32_t)lane * b_bytes, bmaps[bmap], full, (k0 + lane) * BK, 0, pol);
+            if (lane < nk) tc::tma_load_2d(dst + (uint32_t)lane * pb_bytes, bmaps[bmap], full, (k0 + lane) * BK, 0, pol);
           }
           __syncwarp();
         }
@@ -607,7 +617,7 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
 // b * 256 + a * (dual + 1) * BN  (gate at +0, up at +BN).
 __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint32_t tmem_base, int which) {
   const Cfg& c = p.c;
-  const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(c.BN >> 3) << 17);
+  const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10);
   const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
   RingPos rp{0, 0};
   const int b_pages = (c.BN * BK * 2) / PAGE;
@@ -622,24 +632,24 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
         const TileDesc td = tiles[P.tile0 + t];
         const int a_pages = td.n_rows >> 3;
         const int w_pages = (P.dual + 1) * a_pages;
-        const int pages = P.kpi * (w_pages + b_pages);
+        const int pages = P.kpi * (w_pages + P.bmul * b_pages);
         // tiles of at most 64 weight rows take the M = 64 shape: the multiply reads half the operand
         // rows from shared memory (row r of its accumulator sits in lane 32 (r / 16) + r % 16)
-        const uint32_t idesc = idesc0 | ((td.n_rows <= 64 ? 4u : 8u) << 24);
+        const uint32_t idesc = idesc0 | ((uint32_t)((P.bmul * c.BN) >> 3) << 17) | ((td.n_rows <= 64 ? 4u : 8u) << 24);
         const uint32_t buf = n_acc & 1u;
         if (!wait_bar(&sh->acc_empty[buf], ((n_acc >> 1) & 1u) ^ 1u, p.ctl, sh)) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t acc = tmem_base + buf * 256u + (uint32_t)(which * (P.dual + 1) * c.BN);
+        const uint32_t acc = tmem_base + buf * 256u + (uint32_t)(which * P.width);
         const uint32_t acc2 = acc + (uint32_t)c.BN;
         const uint32_t up_lo = (uint32_t)a_pages * (PAGE / 16);          // gate rows -> up rows
         const uint32_t w_lo = (uint32_t)w_pages * (PAGE / 16);           // weights of one chunk
-        const uint32_t x_lo = (uint32_t)b_pages * (PAGE / 16);           // operand tile of one chunk
+        const uint32_t x_lo = (uint32_t)(P.bmul * b_pages) * (PAGE / 16);  // operand tile of one chunk
         const uint32_t x0_lo = (uint32_t)P.kpi * w_lo;                   // first weight chunk -> first operand tile
         for (int gi = 0; gi < P.n_groups; ++gi) {
           int fp;
           const uint32_t it = rp.item;
           const int at = rp.place(pages, c.ring_pages, fp);
-          if ((gi & (c.n_iss - 1)) != which) continue;
+          if ((gi & (P.n_iss - 1)) != which) continue;
           if (!wait_bar(&sh->full[it % NB], (it / NB) & 1u, p.ctl, sh)) return;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           if (t == 0 && gi == 0) issuer_mark(p, jb, T_MMA_FIRST + ph);
@@ -648,7 +658,7 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
           uint32_t a_lo = desc_lo(ring_base + (uint32_t)at * PAGE);
           uint32_t b_lo = a_lo + x0_lo;
           int k = 0;
-          if (gi < c.n_iss) {  // this issuer's first item of the tile overwrites its accumulator
+          if (gi < P.n_iss) {  // this issuer's first item of the tile overwrites its accumulator
             mma_chunk<true>(acc, a_lo, b_lo, idesc);
             if (P.dual) mma_chunk<true>(acc2, a_lo + up_lo, b_lo, idesc);
             a_lo += w_lo;
@@ -832,6 +842,23 @@ struct Worker {
           keep_s[k] = __ldcg(skip_src(J, rd.div(r) + 1, rd.mod(r)) + f);
         }
       }
+      if (J.defer && fv) {   // the skip candidates' rows of the next layer's operand
+        const float wq = __ldg(J.norm_next + f);
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = group * 16 + k;
+          if (r < rows_all) p.b.xn_a[(long long)(c.BN + r) * c.d + f] = __float2bfloat16_rn(keep_s[k] * wq);
+        }
+        for (int cb = group + 2; cb * 16 < rows_all; cb += 2) {
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            const int r = cb * 16 + k;
+            if (r < rows_all)
+              p.b.xn_a[(long long)(c.BN + r) * c.d + f] =
+                  __float2bfloat16_rn(__ldcg(skip_src(J, rd.div(r) + 1, rd.mod(r)) + f) * wq);
+          }
+        }
+      }
     }
     // residual rows of the first block are fetched before the accumulator is ready
     float res[16];
@@ -847,7 +874,7 @@ struct Worker {
     float wn = 0.f;
     if (fv) {
       if (P.kind == G_O) wn = __ldg(J.norm_mlp + f);
-      else if (P.kind == G_DOWN && !J.dp && J.norm_next) wn = __ldg(J.norm_next + f);
+      else if (P.kind == G_DOWN && (!J.dp || J.defer) && J.norm_next) wn = __ldg(J.norm_next + f);
     }
     const uint32_t buf = n_acc & 1u;
     // one thread polls the barrier, the others sleep in the hardware barrier behind it
@@ -857,7 +884,7 @@ struct Worker {
     if (!ok) return false;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (tile_no == 0 && P.kind < 4) mark(T_ACC + P.kind);
-    if (P.kind == G_QKV && tile_no == 0 && J.src_flag == F_SELECT) {
+    if (P.kind == G_QKV && tile_no == 0 && (J.src_flag == F_SELECT || J.dual_src)) {
       // the rows come from an Eq. 2 step: it left their factors in shared memory
       for (int r = wtid; r < J.R; r += WORKERS) sh->rs[r] = sh->rs_next[r];
       worker_sync();
@@ -869,17 +896,26 @@ struct Worker {
     for (int cb = group; cb < ncb; cb += 2) {
       float v[16], u[16];
       tc::tmem_ld16(t_lane + (uint32_t)(cb * 16), v);
-      if (P.dual) tc::tmem_ld16(t_lane + (uint32_t)(c.BN + cb * 16), u);
-      if (c.n_iss == 2 && P.n_groups >= 2) {  // the second MMA issuer's share of the reduction
-        const uint32_t off = (uint32_t)((P.dual + 1) * c.BN + cb * 16);
+      if (P.dual || P.bmul == 2) tc::tmem_ld16(t_lane + (uint32_t)(c.BN + cb * 16), u);
+      if (P.n_iss == 2 && P.n_groups >= 2) {  // the second MMA issuer's share of the reduction
+        const uint32_t off = (uint32_t)(P.width + cb * 16);
         float w[16];
         tc::tmem_ld16(t_lane + off, w);
 #pragma unroll
         for (int k = 0; k < 16; ++k) v[k] += w[k];
-        if (P.dual) {
+        if (P.dual || P.bmul == 2) {
           tc::tmem_ld16(t_lane + off + (uint32_t)c.BN, w);
 #pragma unroll
           for (int k = 0; k < 16; ++k) u[k] += w[k];
+        }
+      }
+      if (P.bmul == 2) {
+        // both candidates of every state went through the product (v: layer output, u: skip candidate):
+        // keep the one the Eq. 2 step chose
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = cb * 16 + k;
+          if (r < J.R && !sh->choice[rd.div(r) + 1]) v[k] = u[k];
         }
       }
       if (cb != group && resid && fv) {
@@ -939,6 +975,7 @@ struct Worker {
           const int r = cb * 16 + k;
           const float y = (fv && r < J.R) ? res[k] + v[k] : 0.f;
           if (fv && r < J.R && ncb > 2) __stcg(p.b.Gbuf + (long long)r * c.d + f, y);
+          if (J.defer && fv && r < J.R) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
           if (cb == group) keep_y[k] = y;
           pr[k] = xi[k] * y;
           pr[16 + k] = y * y;
@@ -1083,8 +1120,9 @@ struct Worker {
   //   (2) wait for every CTA, read the totals, decide (every CTA decides alike); the chosen row's
   //       sum of squares is also the next layer's norm factor;
   //   (3) write this CTA's slice of the next layer's operand, publish;
-  //   (4) off the critical path: this CTA's slice of g[i][.], and its share of the next step's sums
-  //       over the skip candidates.
+  //   (4) this CTA's slice of g[i][.].
+  // The sums over the skip candidates (x.s, s.s, x.x) were added earlier: by a layer job while it waited
+  // for its o product, by a select-only job at its start.
   // from_epilogue: the down product's epilogue left the partials of this CTA in the tables and
   // the thread's layer outputs / skip candidates of its first row block in keep_y / keep_s.
   __device__ bool dp_step(const Job& J, int jb, bool from_epilogue, float (&keep_y)[16], float (&keep_s)[16]) {
@@ -1102,7 +1140,8 @@ struct Worker {
         reinterpret_cast<unsigned long long*>(p.b.cosacc) + (long long)jb * ((long long)(c.Rcap + MAX_ROWS) * 5);
     const RowDiv rd(J.T);
     const float wn = (fv && J.norm_next) ? __ldg(J.norm_next + f) : 0.f;   // needed right after the decision
-    if (jb == 0) pre_sums(0, rows, J.T, J.x_i, J.x_im1, J.x_tok_stride, J.g_prev, fv, f);  // nobody prepared the first step
+    // (a layer job adds its sums over the skip candidates while it waits for its o product)
+    if (J.type == JOB_SELECT) pre_sums(jb, rows, J.T, J.x_i, J.x_im1, J.x_tok_stride, J.g_prev, fv, f);
     if (!from_epilogue) {
       // no layer ran for this CTA's features: only skip candidates exist
 #pragma unroll
@@ -1166,7 +1205,7 @@ struct Worker {
       y16[k] = 0.f;
       if (fv && r < rows) y16[k] = sh->choice[rd.div(r) + 1] ? keep_y[k] : keep_s[k];
     }
-    if (J.norm_next && fv) {
+    if (J.norm_next && fv && !J.defer) {
       for (int cb = group; cb < ncb; cb += 2) {
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
@@ -1180,7 +1219,7 @@ struct Worker {
         }
       }
     }
-    publish(F_SELECT, jb + 1);
+    if (!J.defer) publish(F_SELECT, jb + 1);   // (a deferred step's successor reads both candidates: nobody waits)
     mark(T_SEL_PUB);
     // (4) g[i][.] for the next step (read back only by this thread: same feature in every step)
     if (fv) {
@@ -1198,7 +1237,6 @@ struct Worker {
         }
       }
     }
-    if (J.x_ip1) pre_sums(jb + 1, min(J.i + 1, J.M) * J.T, J.T, J.x_ip1, J.x_i, J.x_tok_stride, J.g_next, fv, f);
     return true;
   }
 
@@ -1647,6 +1685,13 @@ struct Worker {
       for (int ph = 0; ph < 4; ++ph) {
         Phase P;
         P.init(p, J, ph);
+        if (ph == G_O && J.dp) {
+          // idle time (the o product is being multiplied): this CTA's share of the sums of this job's
+          // Eq. 2 step over the skip candidates, which the previous step left in g
+          const int f_lo = __ldg(split_lo(S_D) + blockIdx.x), f_hi = __ldg(split_lo(S_D) + blockIdx.x + 1);
+          const int fl = feat_local(f_hi - f_lo, ww & 3, lane);
+          pre_sums(jb, (J.ell + (J.diag ? 1 : 0)) * J.T, J.T, J.x_i, J.x_im1, J.x_tok_stride, J.g_prev, fl >= 0, f_lo + fl);
+        }
         for (int t = 0; t < P.n_tiles; ++t)
           if (!epilogue(J, jb, P, tiles[P.tile0 + t], t, keep_y, keep_s)) return false;
         mark(ph == G_QKV ? T_QKV : (ph == G_O ? T_O : (ph == G_GU ? T_GU : T_DOWN)));
@@ -1681,6 +1726,7 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
               const __grid_constant__ CUtensorMap map_head, const __grid_constant__ CUtensorMap map3_xn_a,
               const __grid_constant__ CUtensorMap map3_attn, const __grid_constant__ CUtensorMap map3_xn_m,
               const __grid_constant__ CUtensorMap map3_act, const __grid_constant__ CUtensorMap map3_head,
+              const __grid_constant__ CUtensorMap map_xn_a2, const __grid_constant__ CUtensorMap map3_xn_a2,
               const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ Shared sh;
@@ -1718,8 +1764,8 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
   if (warp == 0) {
     producer_a(p, &sh, ring_base, lane);
   } else if (warp == 1) {
-    const CUtensorMap* bmaps[5] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head};
-    const CUtensorMap* bmaps3[5] = {&map3_xn_a, &map3_attn, &map3_xn_m, &map3_act, &map3_head};
+    const CUtensorMap* bmaps[6] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head, &map_xn_a2};
+    const CUtensorMap* bmaps3[6] = {&map3_xn_a, &map3_attn, &map3_xn_m, &map3_act, &map3_head, &map3_xn_a2};
     producer_b(p, &sh, ring_base, bmaps, bmaps3, lane);
   } else if (warp == 2 || warp == 3) {
     if (lane == 0) mma_issuer(p, &sh, ring_base, tmem_base, warp - 2);

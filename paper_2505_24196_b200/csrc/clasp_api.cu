@@ -135,7 +135,7 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
     w.e_rcap = (int)rcap;
     w.xn_m = take(R * d * 2);
     w.e_run_len = pk::ATT_KEYS * ((c.max_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32));
-    w.e_chunk_cap = (c.max_ctx + w.e_run_len - 1) / w.e_run_len + (int)((rcap + pk::ATT_KEYS - 1) / pk::ATT_KEYS);
+    w.e_chunk_cap = 32 + (int)((rcap + pk::ATT_KEYS - 1) / pk::ATT_KEYS);   // at most 32 runs of cache keys + own rows
     w.e_att_acc = (float*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * c.head_dim * 4);
     w.e_att_ml = (float2*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * sizeof(float2));
     // fixed-point accumulators, zeroed before every launch: ss_a, ss_m, cosacc are contiguous
@@ -660,7 +660,7 @@ double job_bytes(const clasp_ctx* ctx, const pk::Job& J) {
 
 // Launch the engine over ctx->e_jobs.  Rmax: most rows of any job; head_off: first row of the
 // previous job that the head job (if any) reads.
-int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
+int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   const clasp_config& c = ctx->cfg;
   Workspace& ws = ctx->ws;
   if (ctx->e_jobs.empty()) return CLASP_OK;
@@ -739,6 +739,12 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off) {
   P.c.L = c.L; P.c.d = d; P.c.qd = qd; P.c.kvd = c.n_kv_heads * c.head_dim; P.c.hd = c.head_dim;
   P.c.nq = c.n_q_heads; P.c.nkv = c.n_kv_heads; P.c.dffn = c.d_ffn; P.c.vocab = c.vocab; P.c.eps = c.rms_eps;
   P.c.G = ctx->e_G; P.c.Rcap = ws.e_rcap; P.c.run_len = ws.e_run_len; P.c.chunk_cap = ws.e_chunk_cap;
+  // The forward passes cut the cache into runs of a length fixed by the context capacity, so that a
+  // position's attention is summed in the same order whichever call computes it (verification and
+  // one-token decoding must agree bit for bit).  The search only has to agree with itself: it cuts
+  // the keys it sees into at most 32 runs, which spreads a short context over many more CTAs.
+  if (search_ctx >= 0) P.c.run_len = pk::ATT_KEYS * ((search_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32) > 0
+                                                       ? (search_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32) : 1);
   P.c.BN = BN; P.c.ring_pages = ring_pages; P.c.n_iss = BN <= 64 ? 2 : 1;
   if (getenv("CLASP_ENGINE_ONE_ISSUER")) P.c.n_iss = 1;
 
@@ -1022,7 +1028,7 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
           ctx->e_jobs[k + 1].dual_src = 1;
         }
     link_jobs(ctx->e_jobs);
-    if ((rc = engine_launch(ctx, M * T, 0))) return rc;
+    if ((rc = engine_launch(ctx, M * T, 0, ctx_len))) return rc;
     clasp::backtrack_kernel<<<1, 32, 0, ctx->stream>>>(ws.choice, L, M, skip_mask);
     return launch_check(ctx);
   }

@@ -1360,11 +1360,25 @@ struct Worker {
       int key_lo, key_hi;
       if (!own) { key_lo = chunk * c.run_len; key_hi = min(k_tot, key_lo + c.run_len); }
       else { key_lo = (chunk - n_runs) * ATT_KEYS; key_hi = min(J.R, key_lo + ATT_KEYS); }
+      // cache pieces of the tile at k0 into the rolling registers (issued one tile ahead of their use)
+      auto load_cache_tile = [&](int k0) {
+#pragma unroll
+        for (int e = 0; e < FILL; ++e) {
+          const int vv = wtid + e * WORKERS;
+          const int key = k0 + vv / (HD / 8), cv8 = vv % (HD / 8);
+          pre_k[e] = make_uint4(0, 0, 0, 0);
+          pre_v[e] = make_uint4(0, 0, 0, 0);
+          if (key < key_hi && key < J.C) {
+            pre_k[e] = __ldcg(reinterpret_cast<const uint4*>(J.ck + (long long)key * kvld + kvh * HD + cv8 * 8));
+            pre_v[e] = __ldcg(reinterpret_cast<const uint4*>(J.cv + (long long)key * kvld + kvh * HD + cv8 * 8));
+          }
+        }
+      };
+      if (!own && !(pre_ok && it == (int)blockIdx.x)) load_cache_tile(key_lo);
       for (int key0 = key_lo; key0 < key_hi; key0 += ATT_KEYS) {
         const int nkeys = min(ATT_KEYS, key_hi - key0);
         worker_sync();  // previous tile consumed
         // K/V tile: cache rows as they are; rows of this call rotated / rounded from the projections
-        const bool use_pre = pre_ok && it == (int)blockIdx.x && key0 == key_lo;
 #pragma unroll
         for (int e = 0; e < FILL; ++e) {
           const int vv = wtid + e * WORKERS;
@@ -1374,13 +1388,8 @@ struct Worker {
             const int key = key0 + row;
             const int new_row = own ? key : (J.uniform ? key - J.C : -1);
             if (new_row < 0) {
-              if (use_pre) {
-                kk = pre_k[e];
-                vq = pre_v[e];
-              } else {
-                kk = __ldcg(reinterpret_cast<const uint4*>(J.ck + (long long)key * kvld + kvh * HD + cv8 * 8));
-                vq = __ldcg(reinterpret_cast<const uint4*>(J.cv + (long long)key * kvld + kvh * HD + cv8 * 8));
-              }
+              kk = pre_k[e];
+              vq = pre_v[e];
             } else {
               const float* kr = p.b.qkv + (long long)new_row * qkvd + c.qd + kvh * HD;
               const float* vr = kr + c.kvd;
@@ -1414,6 +1423,7 @@ struct Worker {
           *reinterpret_cast<uint4*>(k_s + row * LD + cv8 * 8) = kk;
           *reinterpret_cast<uint4*>(v_s + row * LD + cv8 * 8) = vq;
         }
+        if (!own && key0 + ATT_KEYS < key_hi) load_cache_tile(key0 + ATT_KEYS);   // in flight during the tile's math
         worker_sync();
         if (!active) continue;
         float s[4][4];

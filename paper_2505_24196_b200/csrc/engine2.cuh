@@ -305,7 +305,8 @@ struct Shared {
   int flag;                 // broadcast of a one-thread decision to the workers
   float rs[MAX_ROWS];       // per-row norm factors of the current product
   float rs_next[MAX_ROWS];  // Eq. 2 step: norm factors of the rows it hands to the next layer
-  int choice[MAX_ROWS + 2];
+  int choice[MAX_ROWS + 2];   // Eq. 2 decision per state (1: the layer output was taken)
+  int choice_row[MAX_ROWS + 16];  // the same per candidate row
   int foot[NB];             // warp 0: ring pages each item in flight gives back when it retires
   int job_words[(sizeof(Job) + 3) / 4];  // the workers' copy of the current job descriptor
 };
@@ -839,7 +840,7 @@ struct Worker {
         keep_y[k] = 0.f;
         if (fv && r < rows_all) {
           xi[k] = __ldg(J.x_i + rd.mod(r) * J.x_tok_stride + f);
-          keep_s[k] = __ldcg(skip_src(J, rd.div(r) + 1, rd.mod(r)) + f);
+          keep_s[k] = __ldcg(skip_row(J, r) + f);
         }
       }
       if (J.defer && fv) {   // the skip candidates' rows of the next layer's operand
@@ -855,7 +856,7 @@ struct Worker {
             const int r = cb * 16 + k;
             if (r < rows_all)
               p.b.xn_a[(long long)(c.BN + r) * c.d + f] =
-                  __float2bfloat16_rn(__ldcg(skip_src(J, rd.div(r) + 1, rd.mod(r)) + f) * wq);
+                  __float2bfloat16_rn(__ldcg(skip_row(J, r) + f) * wq);
           }
         }
       }
@@ -915,7 +916,7 @@ struct Worker {
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
           const int r = cb * 16 + k;
-          if (r < J.R && !sh->choice[rd.div(r) + 1]) v[k] = u[k];
+          if (r < J.R && !sh->choice_row[r]) v[k] = u[k];
         }
       }
       if (cb != group && resid && fv) {
@@ -1060,6 +1061,11 @@ struct Worker {
   }
 
   // skip candidate of state j (1-based) at row t: g[i-1][j-1]
+  // the same by row r = (j - 1) T + t of the step: state 1's candidates are the objective rows of the step
+  // before, the others row r - T ... of g, i.e. row r of the array that starts at g[i-1][0]
+  __device__ __forceinline__ const float* skip_row(const Job& J, int r) const {
+    return r < J.T ? J.x_im1 + r * J.x_tok_stride : J.g_prev + (long long)r * p.c.d;
+  }
   __device__ __forceinline__ const float* skip_src(const Job& J, int j, int t) const {
     return j == 1 ? J.x_im1 + t * J.x_tok_stride : J.g_prev + ((long long)(j - 1) * J.T + t) * p.c.d;
   }
@@ -1148,7 +1154,7 @@ struct Worker {
       for (int k = 0; k < 16; ++k) {
         const int r = group * 16 + k;
         keep_y[k] = 0.f;
-        keep_s[k] = (fv && r < rows) ? __ldcg(skip_src(J, rd.div(r) + 1, rd.mod(r)) + f) : 0.f;
+        keep_s[k] = (fv && r < rows) ? __ldcg(skip_row(J, r) + f) : 0.f;
       }
     } else {
       for (int idx = wtid; idx < J.R * 2; idx += WORKERS) {
@@ -1181,6 +1187,7 @@ struct Worker {
         if (J.forced && J.forced[j] != 255) take = (J.forced[j] == 0);
       }
       sh->choice[j] = take;
+      for (int t = 0; t < J.T; ++t) sh->choice_row[(j - 1) * J.T + t] = take;
       for (int t = 0; t < J.T; ++t) {
         const double* v = T->cosv[(j - 1) * J.T + t];
         sh->rs_next[(j - 1) * J.T + t] = rsqrtf((float)(take ? v[1] : v[3]) / (float)c.d + c.eps);
@@ -1203,7 +1210,7 @@ struct Worker {
     for (int k = 0; k < 16; ++k) {
       const int r = group * 16 + k;
       y16[k] = 0.f;
-      if (fv && r < rows) y16[k] = sh->choice[rd.div(r) + 1] ? keep_y[k] : keep_s[k];
+      if (fv && r < rows) y16[k] = sh->choice_row[r] ? keep_y[k] : keep_s[k];
     }
     if (J.norm_next && fv && !J.defer) {
       for (int cb = group; cb < ncb; cb += 2) {
@@ -1211,9 +1218,8 @@ struct Worker {
         for (int k = 0; k < 16; ++k) {
           const int r = cb * 16 + k;
           if (r < rows) {
-            const int j = rd.div(r) + 1, t = rd.mod(r);
             const float y = cb == group ? y16[k]
-                                        : (sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f));
+                                        : (sh->choice_row[r] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_row(J, r) + f));
             p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
           }
         }
@@ -1222,17 +1228,19 @@ struct Worker {
     if (!J.defer) publish(F_SELECT, jb + 1);   // (a deferred step's successor reads both candidates: nobody waits)
     mark(T_SEL_PUB);
     // (4) g[i][.] for the next step (read back only by this thread: same feature in every step)
+    float* const g_out = J.g_next + (long long)J.T * c.d + f;
+    const int gf_lo = (J.M - 1) * J.T;                              // first row of state M, if the step has it
+    float* const gf_out = (J.g_final && rows > gf_lo) ? J.g_final + f : nullptr;
     if (fv) {
       for (int cb = group; cb < ncb; cb += 2) {
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
           const int r = cb * 16 + k;
-          if (r < rows) {
-            const int j = rd.div(r) + 1, t = rd.mod(r);
+          if (r < rows) {   // row r of the step is g[i][j][t] with j T + t = r + T
             const float y = cb == group ? y16[k]
-                                        : (sh->choice[j] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_src(J, j, t) + f));
-            __stcg(J.g_next + ((long long)j * J.T + t) * c.d + f, y);
-            if (J.g_final && j == J.M) J.g_final[(long long)t * c.d + f] = y;
+                                        : (sh->choice_row[r] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_row(J, r) + f));
+            __stcg(g_out + (long long)r * c.d, y);
+            if (gf_out && r >= gf_lo) gf_out[(long long)(r - gf_lo) * c.d] = y;
           }
         }
       }

@@ -6,6 +6,7 @@ self-speculative loop.  One JSON line per measurement.
     python -m paper_2505_24196_b200.sweep dp     --model 8b  --ctx 512 2048 8192 --M 8 12 16 --T 1
     python -m paper_2505_24196_b200.sweep dp     --model 70b --ctx 1024 --M 32 40
     python -m paper_2505_24196_b200.sweep decode --model 8b  --prompt 512 --new 256 --K 4 8 --M 12
+    python -m paper_2505_24196_b200.sweep trace  --model 8b  --ctx 512 --M 12 --job 20
 
 Weights are seeded random-init tensors and the prompts uniform random token ids (see `datagen`).
 Times come from CUDA events on the library's stream; the per-layer split comes from the
@@ -123,6 +124,54 @@ def cmd_dp(args):
     eng.close()
 
 
+STAMP_NAMES = (["job_start", "qkv_epilogue_done", "attention_ready", "attention_q_loaded", "attention_tiles_done",
+                "attention_published", "attention_merged", "o_epilogue_done", "gate_up_epilogue_done",
+                "down_epilogue_done", "eq2_sums_published", "eq2_sums_complete", "eq2_decided", "eq2_step_done",
+                "head_done", "-"]
+               + [f"{a}_{b}" for a in ("mma_first", "mma_last", "accumulator_ready") for b in ("qkv", "o", "gate_up", "down")]
+               + ["eq2_next_operand_point", "operand_ready_qkv", "operand_ready_o", "operand_ready_gate_up"])
+
+
+def cmd_trace(args):
+    """Time line of one job of a search: per stamp the min / median / max over the CTAs, in
+    microseconds after the job's first stamp."""
+    import numpy as np
+    C, M, T = args.ctx[0], args.M[0], args.T[0]
+    cfg, ccfg, eng, keep = build_engine(args.model, C + 64, M, T)
+    kv = clasp.KVCache(ccfg, device=eng.device)
+    toks = datagen.token_ids(cfg, C).to(eng.device)
+    hid = prefill_to(eng, kv, toks, 0, C, T)[-T:].contiguous()
+    d, L = cfg.d_model, cfg.L
+    p0 = C - T
+    run = lambda: eng.dp_search(hid, d, (L + 1) * d, kv, p0, p0, T, M, want_margins=False, want_g=False)
+    for _ in range(3):
+        run()
+    G = eng.engine_ctas()
+    cap = (L + 4) * TRACE_SLOTS
+    st = torch.zeros((G, cap), dtype=torch.int64, device=eng.device)
+    eng.set_trace(st, cap)
+    run()
+    torch.cuda.synchronize()
+    eng.set_trace(None, 0)
+    s = st.cpu().numpy().astype(np.float64)
+    jb = args.job
+    blk = s[:, jb * TRACE_SLOTS:(jb + 1) * TRACE_SLOTS]
+    base = blk[blk > 0].min()
+    rows = []
+    for k, name in enumerate(STAMP_NAMES):
+        col = blk[:, k]
+        col = col[col > 0]
+        if len(col):
+            col = (col - base) / 1e3
+            rows.append((float(np.median(col)), name, float(col.min()), float(col.max())))
+    print(f"# job {jb} (DP step {jb + 1}, layer {jb}) of a search: model {cfg.name}, ctx {C}, M {M}, T {T}; us after the job's first stamp")
+    for med, name, lo, hi in sorted(rows):
+        print(f"{name:28s} min {lo:8.2f}  median {med:8.2f}  max {hi:8.2f}")
+    starts = [s[:, j * TRACE_SLOTS][s[:, j * TRACE_SLOTS] > 0].min() for j in range(L) if (s[:, j * TRACE_SLOTS] > 0).any()]
+    print("job durations (us):", " ".join(f"{(starts[i + 1] - starts[i]) / 1e3:.0f}" for i in range(len(starts) - 1)))
+    eng.close()
+
+
 def cmd_decode(args):
     max_ctx = args.prompt + args.new + 4 * (max(args.K) + 1) + 64
     cfg, ccfg, eng, keep = build_engine(args.model, max_ctx, max(args.M), 1, max_head_rows=max(args.K) + 1)
@@ -158,11 +207,15 @@ def cmd_decode(args):
             ms = a.elapsed_time(b)
             out = out[:args.new]
             acc = [r["accepted"] for r in dec.rounds]
+            # Sparse Persistence (Sec. 3.7): Jaccard similarity of the skip sets of consecutive searches
+            sets = [frozenset(i for i, b in enumerate(r["S"]) if b) for r in dec.rounds[::args.dp_interval]]
+            jac = [len(x & y) / max(len(x | y), 1) for x, y in zip(sets, sets[1:])]
             print(json.dumps({"what": "self_speculative", "model": cfg.name, "prompt": args.prompt, "new": args.new,
                               "M": M, "K": K, "dp_interval": args.dp_interval, "identical_to_autoregressive": out == ar,
                               "decode_ms": round(ms, 2), "prefill_and_first_search_ms": round(prefill_ms, 2),
                               "tokens_per_s": round((args.new - 1) / ms * 1e3, 2), "rounds": len(dec.rounds),
                               "mean_accepted_drafts": round(sum(acc) / max(len(acc), 1), 3),
+                              "mean_jaccard_of_consecutive_skip_sets": round(sum(jac) / max(len(jac), 1), 3),
                               "stage_ms_total": {k: round(v, 2) for k, v in dec.stage_ms.items()},
                               "device_status": eng.device_status()}), flush=True)
     eng.close()
@@ -177,6 +230,12 @@ def main():
     p.add_argument("--M", type=int, nargs="+", default=[12])
     p.add_argument("--T", type=int, nargs="+", default=[1])
     p.add_argument("--reps", type=int, default=10)
+    p = sub.add_parser("trace")
+    p.add_argument("--model", default="8b")
+    p.add_argument("--ctx", type=int, nargs="+", default=[512])
+    p.add_argument("--M", type=int, nargs="+", default=[12])
+    p.add_argument("--T", type=int, nargs="+", default=[1])
+    p.add_argument("--job", type=int, default=20)
     p = sub.add_parser("decode")
     p.add_argument("--model", default="8b")
     p.add_argument("--prompt", type=int, default=512)
@@ -185,7 +244,7 @@ def main():
     p.add_argument("--M", type=int, nargs="+", default=[12])
     p.add_argument("--dp-interval", type=int, default=1)
     args = ap.parse_args()
-    {"dp": cmd_dp, "decode": cmd_decode}[args.cmd](args)
+    {"dp": cmd_dp, "decode": cmd_decode, "trace": cmd_trace}[args.cmd](args)
 
 
 if __name__ == "__main__":

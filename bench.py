@@ -212,13 +212,7 @@ def run_ours(args, rank, world):
 
     # max over ranks of the time-like numbers, sum of the throughput
     tok_s = new_tokens / (total_ms * 1e-3)
-    if world > 1:
-        t = torch.tensor([total_ms, dp_ms, e2e_val], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms, dp_ms, e2e_val = t.tolist()
-        s = torch.tensor([tok_s], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(s, op=torch.distributed.ReduceOp.SUM)
-        tok_s = float(s[0])
+    total_ms, dp_ms, e2e_val, tok_s = combine_replicas(total_ms, dp_ms, e2e_val, tok_s, world, dev)
     out = {
         "metric": "dp_search_ms_per_verify", "value": round(dp_ms, 4), "unit": "ms",
         "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": round(total_ms / steps, 4),
@@ -244,6 +238,19 @@ def run_ours(args, rank, world):
         out["cpu_baseline"] = cpu_baseline(cfg, wl, layers=layers, head=head)
     if rank == 0:
         print(json.dumps(out), flush=True)
+
+
+def combine_replicas(total_ms, dp_ms, e2e_ms, tok_s, world, device):
+    """Replicas only: every rank runs the same independent job.  Time-like numbers are the maximum
+    over the ranks (the slowest replica), throughput is the sum.  No data crosses between replicas."""
+    if world > 1:
+        t = torch.tensor([total_ms, dp_ms, e2e_ms], device=device, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms, dp_ms, e2e_ms = t.tolist()
+        s = torch.tensor([tok_s], device=device, dtype=torch.float64)
+        torch.distributed.all_reduce(s, op=torch.distributed.ReduceOp.SUM)
+        tok_s = float(s[0])
+    return total_ms, dp_ms, e2e_ms, tok_s
 
 
 def dp_only(args, eng, dec, kv, cfg, wl):

@@ -55,6 +55,8 @@ constexpr int NB = 32;                // items in flight (mbarrier pairs)
 constexpr int ATT_KEYS = 32;
 constexpr int SCRATCH_BYTES = 2 * ATT_KEYS * 136 * 2 + 2048;  // two padded K/V tiles + slack (>= 16 KB guard)
 constexpr int MAX_ROWS = 128;         // rows one launch may push through a layer
+constexpr int RB = 8;                 // rows (accumulator columns) a worker group finishes per pass: the two groups
+                                      // of four warps take alternate blocks, so 9 to 16 rows keep both busy
 constexpr int N_HEIGHTS = 4;          // distinct tile heights (TMA box heights) per weight matrix
 constexpr int MAX_CTAS = 192;
 
@@ -779,6 +781,32 @@ struct Worker {
     return v[0] + __shfl_xor_sync(0xffffffffu, v[0], 16);
   }
 
+  // Same for 8 values: every lane l returns the total of v[l & 7].
+  __device__ __forceinline__ static float warp_reduce8(float (&v)[8], int lane) {
+#pragma unroll
+    for (int w = 4; w >= 1; w >>= 1) {
+      const bool up = (lane & w) != 0;
+#pragma unroll
+      for (int i = 0; i < w; ++i) {
+        const float send = up ? v[i] : v[i + w];
+        const float keep = up ? v[i + w] : v[i];
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, w);
+      }
+    }
+    float t = v[0] + __shfl_xor_sync(0xffffffffu, v[0], 8);
+    return t + __shfl_xor_sync(0xffffffffu, t, 16);
+  }
+  // eight accumulator columns of this thread's lane
+  __device__ __forceinline__ static void tmem_ld8(uint32_t taddr, float (&v)[8]) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+  }
+
   // per-row factors rsqrt(mean(x^2) + eps) from the accumulated sums of squares
   __device__ void row_scales(const long long* ss, int R, int row_off) {
     const Cfg& c = p.c;
@@ -812,12 +840,12 @@ struct Worker {
 
   // ---- epilogue of one accumulator: tile td of product P.kind.
   // Thread (quarter q, lane) owns feature td.f0 + 32 q + lane; the two warps of a quarter take
-  // alternating blocks of 16 rows (accumulator columns).  Per-row sums over the CTA's features
+  // alternating blocks of RB rows (accumulator columns).  Per-row sums over the CTA's features
   // (sums of squares, cosine partials, arg-max) go through RedTables: one entry per (quarter, row).
   // For the down product of an Eq. 2 job the thread's layer outputs (keep_y) and skip candidates
-  // (keep_s) of its first block of 16 rows stay in registers for dp_step.
-  __device__ bool epilogue(const Job& J, int jb, const Phase& P, const TileDesc& td, int tile_no, float (&keep_y)[16],
-                           float (&keep_s)[16]) {
+  // (keep_s) of its first block of RB rows stay in registers for dp_step.
+  __device__ bool epilogue(const Job& J, int jb, const Phase& P, const TileDesc& td, int tile_no, float (&keep_y)[RB],
+                           float (&keep_s)[RB]) {
     const Cfg& c = p.c;
     RedTables* T = tables();
     const int quarter = ww & 3, group = ww >> 2;
@@ -826,15 +854,15 @@ struct Worker {
     const int f = td.f0 + fl;
     const bool dpd = P.kind == G_DOWN && J.dp;
     const int rows_all = J.R + ((dpd && J.diag) ? J.T : 0);   // Eq. 2: plus the rows of the diagonal state
-    const int ncb = (J.R + 15) >> 4;
+    const int ncb = (J.R + RB - 1) / RB;
     const bool resid = P.kind == G_O || P.kind == G_DOWN;
     const RowDiv rd(J.T);
     // Eq. 2: objective row and skip candidate of every row of the first block, fetched early
-    float xi[16];
+    float xi[RB];
     if (dpd) {
 #pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        const int r = group * 16 + k;
+      for (int k = 0; k < RB; ++k) {
+        const int r = group * RB + k;
         xi[k] = 0.f;
         keep_s[k] = 0.f;
         keep_y[k] = 0.f;
@@ -846,14 +874,14 @@ struct Worker {
       if (J.defer && fv) {   // the skip candidates' rows of the next layer's operand
         const float wq = __ldg(J.norm_next + f);
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = group * 16 + k;
+        for (int k = 0; k < RB; ++k) {
+          const int r = group * RB + k;
           if (r < rows_all) p.b.xn_a[(long long)(c.BN + r) * c.d + f] = __float2bfloat16_rn(keep_s[k] * wq);
         }
-        for (int cb = group + 2; cb * 16 < rows_all; cb += 2) {
+        for (int cb = group + 2; cb * RB < rows_all; cb += 2) {
 #pragma unroll
-          for (int k = 0; k < 16; ++k) {
-            const int r = cb * 16 + k;
+          for (int k = 0; k < RB; ++k) {
+            const int r = cb * RB + k;
             if (r < rows_all)
               p.b.xn_a[(long long)(c.BN + r) * c.d + f] =
                   __float2bfloat16_rn(__ldcg(skip_row(J, r) + f) * wq);
@@ -862,13 +890,13 @@ struct Worker {
       }
     }
     // residual rows of the first block are fetched before the accumulator is ready
-    float res[16];
+    float res[RB];
 #pragma unroll
-    for (int k = 0; k < 16; ++k) res[k] = 0.f;
+    for (int k = 0; k < RB; ++k) res[k] = 0.f;
     if (resid && fv && group < ncb) {
 #pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        const int r = group * 16 + k;
+      for (int k = 0; k < RB; ++k) {
+        const int r = group * RB + k;
         if (r < J.R) res[k] = P.kind == G_O ? __ldcg(J.x_in + r * J.ldx + f) : __ldcg(p.b.x1 + (long long)r * c.d + f);
       }
     }
@@ -895,34 +923,34 @@ struct Worker {
     }
     const uint32_t t_lane = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
     for (int cb = group; cb < ncb; cb += 2) {
-      float v[16], u[16];
-      tc::tmem_ld16(t_lane + (uint32_t)(cb * 16), v);
-      if (P.dual || P.bmul == 2) tc::tmem_ld16(t_lane + (uint32_t)(c.BN + cb * 16), u);
+      float v[RB], u[RB];
+      tmem_ld8(t_lane + (uint32_t)(cb * RB), v);
+      if (P.dual || P.bmul == 2) tmem_ld8(t_lane + (uint32_t)(c.BN + cb * RB), u);
       if (P.n_iss == 2 && P.n_groups >= 2) {  // the second MMA issuer's share of the reduction
-        const uint32_t off = (uint32_t)(P.width + cb * 16);
-        float w[16];
-        tc::tmem_ld16(t_lane + off, w);
+        const uint32_t off = (uint32_t)(P.width + cb * RB);
+        float w[RB];
+        tmem_ld8(t_lane + off, w);
 #pragma unroll
-        for (int k = 0; k < 16; ++k) v[k] += w[k];
+        for (int k = 0; k < RB; ++k) v[k] += w[k];
         if (P.dual || P.bmul == 2) {
-          tc::tmem_ld16(t_lane + off + (uint32_t)c.BN, w);
+          tmem_ld8(t_lane + off + (uint32_t)c.BN, w);
 #pragma unroll
-          for (int k = 0; k < 16; ++k) u[k] += w[k];
+          for (int k = 0; k < RB; ++k) u[k] += w[k];
         }
       }
       if (P.bmul == 2) {
         // both candidates of every state went through the product (v: layer output, u: skip candidate):
         // keep the one the Eq. 2 step chose
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
+        for (int k = 0; k < RB; ++k) {
+          const int r = cb * RB + k;
           if (r < J.R && !sh->choice_row[r]) v[k] = u[k];
         }
       }
       if (cb != group && resid && fv) {
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
+        for (int k = 0; k < RB; ++k) {
+          const int r = cb * RB + k;
           res[k] = 0.f;
           if (r < J.R) res[k] = P.kind == G_O ? __ldcg(J.x_in + r * J.ldx + f) : __ldcg(p.b.x1 + (long long)r * c.d + f);
         }
@@ -930,16 +958,16 @@ struct Worker {
       if (P.kind == G_QKV) {
         if (fv) {
 #pragma unroll
-          for (int k = 0; k < 16; ++k) {
-            const int r = cb * 16 + k;
+          for (int k = 0; k < RB; ++k) {
+            const int r = cb * RB + k;
             if (r < J.R) __stcg(p.b.qkv + (long long)r * (c.qd + 2 * c.kvd) + f, v[k] * sh->rs[r]);
           }
         }
       } else if (P.kind == G_O) {
-        float sq[16];
+        float sq[RB];
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
+        for (int k = 0; k < RB; ++k) {
+          const int r = cb * RB + k;
           const float y = (fv && r < J.R) ? res[k] + v[k] : 0.f;
           if (fv && r < J.R) {
             __stcg(p.b.x1 + (long long)r * c.d + f, y);
@@ -947,13 +975,13 @@ struct Worker {
           }
           sq[k] = y * y;
         }
-        const float tot = warp_reduce16(sq, lane);
-        if (lane < 16 && cb * 16 + lane < J.R) T->red[quarter][cb * 16 + lane][0] = tot;
+        const float tot = warp_reduce8(sq, lane);
+        if (lane < RB && cb * RB + lane < J.R) T->red[quarter][cb * RB + lane][0] = tot;
       } else if (P.kind == G_GU) {
         if (fv) {
 #pragma unroll
-          for (int k = 0; k < 16; ++k) {
-            const int r = cb * 16 + k;
+          for (int k = 0; k < RB; ++k) {
+            const int r = cb * RB + k;
             if (r < J.R) {
               const float rs = sh->rs[r];
               p.b.act[(long long)r * c.dffn + f] = __float2bfloat16_rn(silu_f(rs * v[k]) * (rs * u[k]));
@@ -965,29 +993,29 @@ struct Worker {
         // (x.y and y.y; the sums over the skip candidates were added when those were written)
         if (cb != group) {
 #pragma unroll
-          for (int k = 0; k < 16; ++k) {
-            const int r = cb * 16 + k;
+          for (int k = 0; k < RB; ++k) {
+            const int r = cb * RB + k;
             xi[k] = (fv && r < J.R) ? __ldg(J.x_i + rd.mod(r) * J.x_tok_stride + f) : 0.f;
           }
         }
-        float pr[32];
+        float pr[2 * RB];
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
+        for (int k = 0; k < RB; ++k) {
+          const int r = cb * RB + k;
           const float y = (fv && r < J.R) ? res[k] + v[k] : 0.f;
           if (fv && r < J.R && ncb > 2) __stcg(p.b.Gbuf + (long long)r * c.d + f, y);
           if (J.defer && fv && r < J.R) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y * wn);
           if (cb == group) keep_y[k] = y;
           pr[k] = xi[k] * y;
-          pr[16 + k] = y * y;
+          pr[RB + k] = y * y;
         }
-        const float tot = warp_reduce32(pr, lane);
-        if (cb * 16 + (lane & 15) < J.R) T->red[quarter][cb * 16 + (lane & 15)][lane >> 4] = tot;
+        const float tot = warp_reduce16(pr, lane);
+        if (lane < 2 * RB && cb * RB + (lane & 7) < J.R) T->red[quarter][cb * RB + (lane & 7)][lane >> 3] = tot;
       } else if (P.kind == G_DOWN) {
-        float sq[16];
+        float sq[RB];
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
+        for (int k = 0; k < RB; ++k) {
+          const int r = cb * RB + k;
           const float y = (fv && r < J.R) ? res[k] + v[k] : 0.f;
           if (fv && r < J.R) {
             __stcg(J.x_out + r * J.ldo + f, y);
@@ -996,13 +1024,13 @@ struct Worker {
           sq[k] = y * y;
         }
         if (J.norm_next) {
-          const float tot = warp_reduce16(sq, lane);
-          if (lane < 16 && cb * 16 + lane < J.R) T->red[quarter][cb * 16 + lane][0] = tot;
+          const float tot = warp_reduce8(sq, lane);
+          if (lane < RB && cb * RB + lane < J.R) T->red[quarter][cb * RB + lane][0] = tot;
         }
       } else {  // G_HEAD: best logit of this tile per row (lowest index on ties) and sum of exp
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
+        for (int k = 0; k < RB; ++k) {
+          const int r = cb * RB + k;
           if (r >= J.R) break;
           const float mine = fv ? v[k] * sh->rs[r] : -INFINITY;
           float best = mine;
@@ -1085,13 +1113,13 @@ struct Worker {
     const Cfg& c = p.c;
     RedTables* T = tables();
     const int quarter = ww & 3, group = ww >> 2;
-    const int ncb = (rows + 15) >> 4;
+    const int ncb = (rows + RB - 1) / RB;
     const RowDiv rd(Tn);
     for (int cb = group; cb < ncb; cb += 2) {
-      float pa[32], pb[16];
+      float pa[2 * RB], pb[RB];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        const int r = cb * 16 + k;
+      for (int k = 0; k < RB; ++k) {
+        const int r = cb * RB + k;
         float xv = 0.f, sv = 0.f;
         if (fv && r < rows) {
           const int j = rd.div(r) + 1, t = rd.mod(r);
@@ -1099,15 +1127,15 @@ struct Worker {
           sv = __ldcg((j == 1 ? x_old + t * xs : g + ((long long)(j - 1) * Tn + t) * c.d) + f);
         }
         pa[k] = xv * sv;
-        pa[16 + k] = sv * sv;
+        pa[RB + k] = sv * sv;
         pb[k] = xv * xv;
       }
-      const float ta = warp_reduce32(pa, lane);
-      const float tb = warp_reduce16(pb, lane);
-      const int r = cb * 16 + (lane & 15);
-      if (r < rows) {
-        T->red[quarter][r][2 + (lane >> 4)] = ta;
-        if (lane < 16) T->red[quarter][r][4] = tb;
+      const float ta = warp_reduce16(pa, lane);
+      const float tb = warp_reduce8(pb, lane);
+      const int r = cb * RB + (lane & 7);
+      if (lane < 2 * RB && r < rows) {
+        T->red[quarter][r][2 + (lane >> 3)] = ta;
+        if (lane < RB) T->red[quarter][r][4] = tb;
       }
     }
     worker_sync();
@@ -1131,7 +1159,7 @@ struct Worker {
   // for its o product, by a select-only job at its start.
   // from_epilogue: the down product's epilogue left the partials of this CTA in the tables and
   // the thread's layer outputs / skip candidates of its first row block in keep_y / keep_s.
-  __device__ bool dp_step(const Job& J, int jb, bool from_epilogue, float (&keep_y)[16], float (&keep_s)[16]) {
+  __device__ bool dp_step(const Job& J, int jb, bool from_epilogue, float (&keep_y)[RB], float (&keep_s)[RB]) {
     const Cfg& c = p.c;
     RedTables* T = tables();
     const int f_lo = __ldg(split_lo(S_D) + blockIdx.x), f_hi = __ldg(split_lo(S_D) + blockIdx.x + 1);
@@ -1141,7 +1169,7 @@ struct Worker {
     const int f = f_lo + fl;
     const int n_states = J.ell + (J.diag ? 1 : 0);
     const int rows = n_states * J.T;
-    const int ncb = (rows + 15) >> 4;
+    const int ncb = (rows + RB - 1) / RB;
     unsigned long long* acc =
         reinterpret_cast<unsigned long long*>(p.b.cosacc) + (long long)jb * ((long long)(c.Rcap + MAX_ROWS) * 5);
     const RowDiv rd(J.T);
@@ -1151,8 +1179,8 @@ struct Worker {
     if (!from_epilogue) {
       // no layer ran for this CTA's features: only skip candidates exist
 #pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        const int r = group * 16 + k;
+      for (int k = 0; k < RB; ++k) {
+        const int r = group * RB + k;
         keep_y[k] = 0.f;
         keep_s[k] = (fv && r < rows) ? __ldcg(skip_row(J, r) + f) : 0.f;
       }
@@ -1205,18 +1233,18 @@ struct Worker {
     worker_sync();
     mark(T_DP_DECIDED);
     // (3) the next layer's operand: the first block of rows comes from registers
-    float y16[16];
+    float y16[RB];
 #pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      const int r = group * 16 + k;
+    for (int k = 0; k < RB; ++k) {
+      const int r = group * RB + k;
       y16[k] = 0.f;
       if (fv && r < rows) y16[k] = sh->choice_row[r] ? keep_y[k] : keep_s[k];
     }
     if (J.norm_next && fv && !J.defer) {
       for (int cb = group; cb < ncb; cb += 2) {
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
+        for (int k = 0; k < RB; ++k) {
+          const int r = cb * RB + k;
           if (r < rows) {
             const float y = cb == group ? y16[k]
                                         : (sh->choice_row[r] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_row(J, r) + f));
@@ -1234,8 +1262,8 @@ struct Worker {
     if (fv) {
       for (int cb = group; cb < ncb; cb += 2) {
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int r = cb * 16 + k;
+        for (int k = 0; k < RB; ++k) {
+          const int r = cb * RB + k;
           if (r < rows) {   // row r of the step is g[i][j][t] with j T + t = r + T
             const float y = cb == group ? y16[k]
                                         : (sh->choice_row[r] ? __ldcg(p.b.Gbuf + (long long)r * c.d + f) : __ldcg(skip_row(J, r) + f));
@@ -1670,9 +1698,9 @@ struct Worker {
   __device__ bool run() {
     const Cfg& c = p.c;
     const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
-    float keep_y[16], keep_s[16];
+    float keep_y[RB], keep_s[RB];
 #pragma unroll
-    for (int k = 0; k < 16; ++k) { keep_y[k] = 0.f; keep_s[k] = 0.f; }
+    for (int k = 0; k < RB; ++k) { keep_y[k] = 0.f; keep_s[k] = 0.f; }
     for (int jb = 0; jb < p.n_jobs; ++jb) {
       // the job descriptor goes to shared memory and from there into a local copy: its fields
       // must not look as if a store to global memory could change them

@@ -1591,11 +1591,12 @@ struct Worker {
         float num[DPL];
 #pragma unroll
         for (int k = 0; k < DPL; ++k) num[k] = 0.f;
+        constexpr int MB = 17;   // partials fetched per trip to L2 (a 512-key context has 17)
         const float* acc = p.b.att_acc + pr * c.chunk_cap * c.hd + lane * DPL;
-        for (int ch0 = 0; ch0 < n_chunks; ch0 += 8) {
-          float a[8][DPL];
+        for (int ch0 = 0; ch0 < n_chunks; ch0 += MB) {
+          float a[MB][DPL];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
+          for (int e = 0; e < MB; ++e) {
 #pragma unroll
             for (int k = 0; k < DPL; ++k) a[e][k] = 0.f;
             if (ch0 + e < n_chunks) {
@@ -1609,7 +1610,7 @@ struct Worker {
             }
           }
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
+          for (int e = 0; e < MB; ++e) {
             const int ch = ch0 + e;
             const float wa = __shfl_sync(0xffffffffu, w0, ch & 31), wb = __shfl_sync(0xffffffffu, w1, ch & 31);
             const float w = ch < 32 ? wa : wb;

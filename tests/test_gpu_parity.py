@@ -178,6 +178,34 @@ def test_dp_search_edge_cases(pair):
     assert torch.equal(ra["D"].nan_to_num(7.0), rb["D"].nan_to_num(7.0)) and torch.equal(ra["S"], rb["S"])
 
 
+def test_search_with_and_without_deferred_decision(pair, monkeypatch):
+    """The persistent kernel normally starts a layer's q/k/v product on both Eq. 2 candidates of every
+    state before the decision exists; CLASP_ENGINE_NODEFER=1 makes it wait for the decision instead.  Both
+    orders multiply the same operand bytes, so tables, mask and final state agree."""
+    cfg = pair.cfg
+    L, d = cfg.L, cfg.d_model
+    toks, ocache, am_o, hid_o, _, kv, am_g, hid_g = _prefill_both(pair, 48)
+    p0 = 47
+    M = min(3, L)
+    a = pair.engine.dp_search(hid_g[p0], d, 0, kv, p0, p0, 1, M)
+    monkeypatch.setenv("CLASP_ENGINE_NODEFER", "1")
+    b = pair.engine.dp_search(hid_g[p0], d, 0, kv, p0, p0, 1, M)
+    monkeypatch.delenv("CLASP_ENGINE_NODEFER")
+    torch.cuda.synchronize()
+    assert pair.engine.device_status() == 0
+    assert torch.equal(a["S"], b["S"])
+    np.testing.assert_allclose(a["D"].nan_to_num(7.0).cpu().numpy(), b["D"].nan_to_num(7.0).cpu().numpy(), atol=1e-6)
+    assert rel_l2(a["g_final"].cpu().numpy(), b["g_final"].cpu().numpy()) < 1e-6
+    ref = orc.dp_search(pair.oracle, hid_o[p0][:, None, :], ocache, p0, p0, M)
+    forced = torch.from_numpy(ref["choice"].copy()).cuda()
+    monkeypatch.setenv("CLASP_ENGINE_NODEFER", "1")
+    c = pair.engine.dp_search(hid_g[p0], d, 0, kv, p0, p0, 1, M, forced_choice=forced)
+    monkeypatch.delenv("CLASP_ENGINE_NODEFER")
+    Dc = c["D"].cpu().numpy()
+    np.testing.assert_allclose(Dc[~np.isnan(Dc)], ref["D"][~np.isnan(Dc)], atol=1e-3)
+    assert rel_l2(c["g_final"].cpu().numpy(), ref["g"][L, M]) < tol_hidden(cfg)
+
+
 def test_argument_errors(pair):
     import paper_2505_24196_b200 as clasp
     cfg = pair.cfg

@@ -525,11 +525,17 @@ int engine_setup(clasp_ctx* ctx) {
   const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
   if (d % 8 || c.d_ffn % 8 || c.vocab % 8) return CLASP_OK;
   cudaFuncAttributes fa;
-  CUDA_TRY(cudaFuncGetAttributes(&fa, pk::engine_kernel));
+  CUDA_TRY(cudaFuncGetAttributes(&fa, pk::engine_kernel<false>));
   ctx->e_static_smem = (int)fa.sharedSizeBytes;
+  {  // one shared-memory budget for the plain and the traced instantiation
+    cudaFuncAttributes ft;
+    CUDA_TRY(cudaFuncGetAttributes(&ft, pk::engine_kernel<true>));
+    if ((int)ft.sharedSizeBytes > ctx->e_static_smem) ctx->e_static_smem = (int)ft.sharedSizeBytes;
+  }
   const int dyn_max = optin - ctx->e_static_smem;
   if (dyn_max < 1024 + 64 * pk::PAGE + pk::SCRATCH_BYTES) return CLASP_OK;
-  CUDA_TRY(cudaFuncSetAttribute(pk::engine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
+  CUDA_TRY(cudaFuncSetAttribute(pk::engine_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
+  CUDA_TRY(cudaFuncSetAttribute(pk::engine_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
   int G = ctx->num_sms;
   if (const char* e = getenv("CLASP_ENGINE_CTAS")) {
     const int v = atoi(e);
@@ -766,7 +772,8 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   void* args[] = {(void*)&bm->second[0], (void*)&bm->second[1], (void*)&bm->second[2], (void*)&bm->second[3],
                   (void*)&hm->second[0], (void*)&bm->second[4], (void*)&bm->second[5], (void*)&bm->second[6],
                   (void*)&bm->second[7], (void*)&hm->second[1], (void*)&bm->second[8], (void*)&bm->second[9], (void*)&P};
-  cudaError_t err = cudaLaunchCooperativeKernel((const void*)pk::engine_kernel, dim3(ctx->e_G), dim3(pk::THREADS),
+  const void* kern = ctx->e_trace ? (const void*)pk::engine_kernel<true> : (const void*)pk::engine_kernel<false>;
+  cudaError_t err = cudaLaunchCooperativeKernel(kern, dim3(ctx->e_G), dim3(pk::THREADS),
                                                 args, dyn, ctx->stream);
   if (ctx->profiling) {
     cudaEventRecord(e1, ctx->stream);

@@ -534,7 +534,9 @@ __device__ void producer_a(const Params& p, Shared* sh, uint32_t ring_base, int 
   }
 }
 
+template <bool TR>
 __device__ __forceinline__ void issuer_mark(const Params& p, int jb, int slot) {
+  if (!TR) return;
   const int idx = jb * TRACE_SLOTS + slot;
   if (p.trace != nullptr && idx < p.trace_cap) {
     unsigned long long t;
@@ -544,6 +546,7 @@ __device__ __forceinline__ void issuer_mark(const Params& p, int jb, int slot) {
 }
 
 // Warp 1, all lanes: lane k issues the operand tile of an item's chunk k.
+template <bool TR>
 __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, const CUtensorMap* const* bmaps,
                            const CUtensorMap* const* bmaps3, int lane) {
   const Cfg& c = p.c;
@@ -571,7 +574,7 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
         bool ok = true;
         if (lane == 0) ok = wait_count(p, fkind, tgt, sh);
         if (!__all_sync(0xffffffffu, ok)) return;
-        if (lane == 0 && P.kind < 3) issuer_mark(p, jb, T_B_READY + P.kind);
+        if (lane == 0 && P.kind < 3) issuer_mark<TR>(p, jb, T_B_READY + P.kind);
       }
       fence_proxy_async();  // the producers' ordinary stores before this warp's TMA reads
       const bool d3 = c.use3d[P.kind] != 0;
@@ -618,6 +621,7 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
 // MMA issuer `which` (0 or 1) takes the ring items of each tile with that parity and adds them up
 // in accumulator `which` of the tile's buffer: buffer b holds accumulator a at column
 // b * 256 + a * (dual + 1) * BN  (gate at +0, up at +BN).
+template <bool TR>
 __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint32_t tmem_base, int which) {
   const Cfg& c = p.c;
   const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10);
@@ -655,7 +659,7 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
           if ((gi & (P.n_iss - 1)) != which) continue;
           if (!wait_bar(&sh->full[it % NB], (it / NB) & 1u, p.ctl, sh)) return;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          if (t == 0 && gi == 0) issuer_mark(p, jb, T_MMA_FIRST + ph);
+          if (t == 0 && gi == 0) issuer_mark<TR>(p, jb, T_MMA_FIRST + ph);
           const int k0 = P.group_at(gi) * P.kpi;
           const int nk = min(P.kc, k0 + P.kpi) - k0;
           uint32_t a_lo = desc_lo(ring_base + (uint32_t)at * PAGE);
@@ -685,7 +689,7 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
           tc::mma_commit(tc::smem_u32(&sh->empty[it % NB]));
         }
         tc::mma_commit(tc::smem_u32(&sh->acc_full[buf]));  // both issuers arrive, with or without items
-        if (which == 0 && t == P.n_tiles - 1) issuer_mark(p, jb, T_MMA_LAST + ph);
+        if (which == 0 && t == P.n_tiles - 1) issuer_mark<TR>(p, jb, T_MMA_LAST + ph);
         ++n_acc;
       }
     }
@@ -693,6 +697,9 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
 }
 
 // ------------------------------------------------------------------ worker steps
+// TR: the step stamps are compiled in (the kernel is sensitive to its code size, so the untraced
+// instantiation carries none of them)
+template <bool TR>
 struct Worker {
   const Params& p;
   Shared* sh;
@@ -704,6 +711,7 @@ struct Worker {
 
   // time stamp of step `slot` (one of the T_* above) of the current job
   __device__ __forceinline__ void mark(int slot) {
+    if (!TR) return;
     const int idx = n_mark * TRACE_SLOTS + slot;
     if (p.trace != nullptr && wtid == 0 && idx < p.trace_cap) {
       unsigned long long t;
@@ -1767,6 +1775,7 @@ struct Worker {
 };
 
 // ------------------------------------------------------------------ the kernel
+template <bool TR>
 __global__ void __launch_bounds__(THREADS, 1)
 engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constant__ CUtensorMap map_attn,
               const __grid_constant__ CUtensorMap map_xn_m, const __grid_constant__ CUtensorMap map_act,
@@ -1813,11 +1822,11 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
   } else if (warp == 1) {
     const CUtensorMap* bmaps[6] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head, &map_xn_a2};
     const CUtensorMap* bmaps3[6] = {&map3_xn_a, &map3_attn, &map3_xn_m, &map3_act, &map3_head, &map3_xn_a2};
-    producer_b(p, &sh, ring_base, bmaps, bmaps3, lane);
+    producer_b<TR>(p, &sh, ring_base, bmaps, bmaps3, lane);
   } else if (warp == 2 || warp == 3) {
-    if (lane == 0) mma_issuer(p, &sh, ring_base, tmem_base, warp - 2);
+    if (lane == 0) mma_issuer<TR>(p, &sh, ring_base, tmem_base, warp - 2);
   } else if (warp >= 4) {
-    Worker w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0};
+    Worker<TR> w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0};
     w.run();
   }
 

@@ -1641,31 +1641,6 @@ struct Worker {
     return true;
   }
 
-  // L2 prefetch of the cache lines this CTA's attention items will read
-  __device__ void attention_prefetch(const Job& J) {
-    const Cfg& c = p.c;
-    const int Gq = c.nq / c.nkv;
-    const int n_pbg = (J.R * Gq + 127) / 128;
-    const int k_tot = J.uniform ? J.C + J.T : J.C;
-    const int n_runs = (k_tot + c.run_len - 1) / c.run_len;
-    const int n_own = J.uniform ? 0 : (J.R + ATT_KEYS - 1) / ATT_KEYS;
-    const int n_chunks = n_runs + n_own;
-    const int n_items = c.nkv * n_chunks * n_pbg;
-    const int lpr = (c.hd * 2 + 127) / 128;
-    for (int it = blockIdx.x; it < n_items; it += c.G) {
-      const int chunk = (it / n_pbg) % n_chunks;
-      const int kvh = it / (n_pbg * n_chunks);
-      if (chunk >= n_runs) continue;
-      const int key_lo = chunk * c.run_len, key_hi = min(J.C, key_lo + c.run_len);
-      const int n_lines = (key_hi - key_lo) * lpr * 2;
-      for (int v = wtid; v < n_lines; v += WORKERS) {
-        const int which = v & 1, ln = (v >> 1) % lpr, key = key_lo + (v >> 1) / lpr;
-        const bf16* addr = (which ? J.cv : J.ck) + (long long)key * c.kvd + kvh * c.hd + ln * 64;
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(addr));
-      }
-    }
-  }
-
   // greedy token of each head row from every CTA's best (CTA 0, one warp per row)
   __device__ bool head_merge(const Job& J, int jb) {
     const Cfg& c = p.c;
@@ -1735,7 +1710,6 @@ struct Worker {
         mark(T_HEAD);
         continue;
       }
-      attention_prefetch(J);
       if (J.prep) prep(J, jb + 1);
       for (int ph = 0; ph < 4; ++ph) {
         Phase P;

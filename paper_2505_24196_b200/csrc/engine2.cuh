@@ -1749,6 +1749,14 @@ struct Worker {
 };
 
 // ------------------------------------------------------------------ the kernel
+#ifndef CLASP_REGS_SPECIAL
+#define CLASP_REGS_SPECIAL 72
+#endif
+constexpr int REGS_SPECIAL = CLASP_REGS_SPECIAL;
+constexpr int REGS_WORKER = (THREADS * 168 - 128 * REGS_SPECIAL) / 256 / 8 * 8;
+static_assert(THREADS == 384 && WORKER_T0 == 128, "register split assumes one special and two worker warp groups");
+static_assert(128 * REGS_SPECIAL + 256 * REGS_WORKER <= THREADS * 168, "register pool of the CTA");
+
 template <bool TR>
 __global__ void __launch_bounds__(THREADS, 1)
 engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constant__ CUtensorMap map_attn,
@@ -1791,15 +1799,22 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = sh.tmem_base;
 
-  if (warp == 0) {
-    producer_a(p, &sh, ring_base, lane);
-  } else if (warp == 1) {
-    const CUtensorMap* bmaps[6] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head, &map_xn_a2};
-    const CUtensorMap* bmaps3[6] = {&map3_xn_a, &map3_attn, &map3_xn_m, &map3_act, &map3_head, &map3_xn_a2};
-    producer_b<TR>(p, &sh, ring_base, bmaps, bmaps3, lane);
-  } else if (warp == 2 || warp == 3) {
-    if (lane == 0) mma_issuer<TR>(p, &sh, ring_base, tmem_base, warp - 2);
-  } else if (warp >= 4) {
+  // The register file is re-divided between the warp groups: the four loader / issuer warps keep
+  // REGS_SPECIAL registers per thread, the two worker groups take the rest
+  // (128 * REGS_SPECIAL + 256 * REGS_WORKER = 384 * 168, the allocation the CTA was launched with).
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SPECIAL));
+    if (warp == 0) {
+      producer_a(p, &sh, ring_base, lane);
+    } else if (warp == 1) {
+      const CUtensorMap* bmaps[6] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head, &map_xn_a2};
+      const CUtensorMap* bmaps3[6] = {&map3_xn_a, &map3_attn, &map3_xn_m, &map3_act, &map3_head, &map3_xn_a2};
+      producer_b<TR>(p, &sh, ring_base, bmaps, bmaps3, lane);
+    } else {
+      if (lane == 0) mma_issuer<TR>(p, &sh, ring_base, tmem_base, warp - 2);
+    }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_WORKER));
     Worker<TR> w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0};
     w.run();
   }

@@ -183,6 +183,7 @@ struct clasp_ctx {
   bool use_engine = false;
   int e_G = 0;              // CTAs of the cooperative grid (one per SM)
   int e_static_smem = 0;
+  const void* e_kernel[2] = {nullptr, nullptr};   // the layer kernel for this head dimension: plain, with step stamps
   int e_split_lo[clasp::pk::N_SPLITS], e_split_units[clasp::pk::N_SPLITS], e_tile_idx[5], e_tiles_off = 0,
       e_kpi[5], e_use3d[5], e_wpages[5];
   int e_heights[8][clasp::pk::N_HEIGHTS];   // tile heights per matrix slot (wq wk wv wo gate up down head)
@@ -524,18 +525,19 @@ int engine_setup(clasp_ctx* ctx) {
   if (!coop) return CLASP_OK;
   const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
   if (d % 8 || c.d_ffn % 8 || c.vocab % 8) return CLASP_OK;
-  cudaFuncAttributes fa;
-  CUDA_TRY(cudaFuncGetAttributes(&fa, pk::engine_kernel<false>));
-  ctx->e_static_smem = (int)fa.sharedSizeBytes;
-  {  // one shared-memory budget for the plain and the traced instantiation
-    cudaFuncAttributes ft;
-    CUDA_TRY(cudaFuncGetAttributes(&ft, pk::engine_kernel<true>));
-    if ((int)ft.sharedSizeBytes > ctx->e_static_smem) ctx->e_static_smem = (int)ft.sharedSizeBytes;
+  // the instantiations for this model's head dimension, without and with step stamps
+  ctx->e_kernel[0] = c.head_dim == 128 ? (const void*)pk::engine_kernel<false, 128> : (const void*)pk::engine_kernel<false, 64>;
+  ctx->e_kernel[1] = c.head_dim == 128 ? (const void*)pk::engine_kernel<true, 128> : (const void*)pk::engine_kernel<true, 64>;
+  ctx->e_static_smem = 0;
+  for (int k = 0; k < 2; ++k) {  // one shared-memory budget for both
+    cudaFuncAttributes fa;
+    CUDA_TRY(cudaFuncGetAttributes(&fa, ctx->e_kernel[k]));
+    if ((int)fa.sharedSizeBytes > ctx->e_static_smem) ctx->e_static_smem = (int)fa.sharedSizeBytes;
   }
   const int dyn_max = optin - ctx->e_static_smem;
   if (dyn_max < 1024 + 64 * pk::PAGE + pk::SCRATCH_BYTES) return CLASP_OK;
-  CUDA_TRY(cudaFuncSetAttribute(pk::engine_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
-  CUDA_TRY(cudaFuncSetAttribute(pk::engine_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
+  for (int k = 0; k < 2; ++k)
+    CUDA_TRY(cudaFuncSetAttribute(ctx->e_kernel[k], cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
   int G = ctx->num_sms;
   if (const char* e = getenv("CLASP_ENGINE_CTAS")) {
     const int v = atoi(e);
@@ -772,7 +774,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   void* args[] = {(void*)&bm->second[0], (void*)&bm->second[1], (void*)&bm->second[2], (void*)&bm->second[3],
                   (void*)&hm->second[0], (void*)&bm->second[4], (void*)&bm->second[5], (void*)&bm->second[6],
                   (void*)&bm->second[7], (void*)&hm->second[1], (void*)&bm->second[8], (void*)&bm->second[9], (void*)&P};
-  const void* kern = ctx->e_trace ? (const void*)pk::engine_kernel<true> : (const void*)pk::engine_kernel<false>;
+  const void* kern = ctx->e_kernel[ctx->e_trace ? 1 : 0];
   cudaError_t err = cudaLaunchCooperativeKernel(kern, dim3(ctx->e_G), dim3(pk::THREADS),
                                                 args, dyn, ctx->stream);
   if (ctx->profiling) {

@@ -697,9 +697,10 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
 }
 
 // ------------------------------------------------------------------ worker steps
-// TR: the step stamps are compiled in (the kernel is sensitive to its code size, so the untraced
-// instantiation carries none of them)
-template <bool TR>
+// TR: the step stamps are compiled in; HD: the model's head dimension (64 or 128).  The kernel is
+// sensitive to its code size, so an instantiation carries neither stamps it does not take nor the
+// attention code of the other head dimension.
+template <bool TR, int HD>
 struct Worker {
   const Params& p;
   Shared* sh;
@@ -1287,7 +1288,6 @@ struct Worker {
   // ---- attention: partial softmax over one run of cache keys or one chunk of own rows.
   // q, k, v of the rows come from the projection buffer (norm factor applied, not rotated): they
   // are rotated here; new keys / values are rounded to the cache type before use.
-  template <int HD>
   __device__ bool attention_partials(const Job& J, int jb) {
     const Cfg& c = p.c;
     constexpr int KS = HD / 16;
@@ -1567,8 +1567,8 @@ struct Worker {
   }
 
   // all chunks of query head h merged, one warp per row; head h is merged by CTA h % G
-  template <int DPL>
   __device__ bool attention_merge(const Job& J, int jb) {
+    constexpr int DPL = HD / 32;   // head dimensions per lane
     const Cfg& c = p.c;
     const int Gq = c.nq / c.nkv;
     const int n_pbg = (J.R * Gq + 127) / 128;
@@ -1600,7 +1600,7 @@ struct Worker {
 #pragma unroll
         for (int k = 0; k < DPL; ++k) num[k] = 0.f;
         constexpr int MB = 17;   // partials fetched per trip to L2 (a 512-key context has 17)
-        const float* acc = p.b.att_acc + pr * c.chunk_cap * c.hd + lane * DPL;
+        const float* acc = p.b.att_acc + pr * c.chunk_cap * HD + lane * DPL;
         for (int ch0 = 0; ch0 < n_chunks; ch0 += MB) {
           float a[MB][DPL];
 #pragma unroll
@@ -1609,10 +1609,10 @@ struct Worker {
             for (int k = 0; k < DPL; ++k) a[e][k] = 0.f;
             if (ch0 + e < n_chunks) {
               if (DPL == 4) {
-                const float4 t = __ldcg(reinterpret_cast<const float4*>(acc + (long long)(ch0 + e) * c.hd));
+                const float4 t = __ldcg(reinterpret_cast<const float4*>(acc + (long long)(ch0 + e) * HD));
                 a[e][0] = t.x; a[e][1] = t.y; a[e][2] = t.z; a[e][3] = t.w;
               } else {
-                const float2 t = __ldcg(reinterpret_cast<const float2*>(acc + (long long)(ch0 + e) * c.hd));
+                const float2 t = __ldcg(reinterpret_cast<const float2*>(acc + (long long)(ch0 + e) * HD));
                 a[e][0] = t.x; a[e][1] = t.y;
               }
             }
@@ -1626,7 +1626,7 @@ struct Worker {
             for (int k = 0; k < DPL; ++k) num[k] = fmaf(w, a[e][k], num[k]);
           }
         }
-        bf16* dst = p.b.attn + pr * c.hd + lane * DPL;
+        bf16* dst = p.b.attn + pr * HD + lane * DPL;
         const float inv = 1.0f / den;
         if (DPL == 4) {
           *reinterpret_cast<uint2*>(dst) = pack4(num[0] * inv, num[1] * inv, num[2] * inv, num[DPL - 1] * inv);
@@ -1726,9 +1726,9 @@ struct Worker {
         mark(ph == G_QKV ? T_QKV : (ph == G_O ? T_O : (ph == G_GU ? T_GU : T_DOWN)));
         if (ph == G_QKV) {
           publish(F_QKV, jb + 1);
-          if (!(c.hd == 128 ? attention_partials<128>(J, jb) : attention_partials<64>(J, jb))) return false;
+          if (!attention_partials(J, jb)) return false;
           mark(T_ATT_PUB);
-          if (!(c.hd == 128 ? attention_merge<4>(J, jb) : attention_merge<2>(J, jb))) return false;
+          if (!attention_merge(J, jb)) return false;
           mark(T_MERGE);
         } else if (ph == G_O) {
           publish(F_O, jb + 1);
@@ -1757,7 +1757,7 @@ constexpr int REGS_WORKER = (THREADS * 168 - 128 * REGS_SPECIAL) / 256 / 8 * 8;
 static_assert(THREADS == 384 && WORKER_T0 == 128, "register split assumes one special and two worker warp groups");
 static_assert(128 * REGS_SPECIAL + 256 * REGS_WORKER <= THREADS * 168, "register pool of the CTA");
 
-template <bool TR>
+template <bool TR, int HD>
 __global__ void __launch_bounds__(THREADS, 1)
 engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constant__ CUtensorMap map_attn,
               const __grid_constant__ CUtensorMap map_xn_m, const __grid_constant__ CUtensorMap map_act,
@@ -1815,7 +1815,7 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_WORKER));
-    Worker<TR> w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0};
+    Worker<TR, HD> w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0};
     w.run();
   }
 

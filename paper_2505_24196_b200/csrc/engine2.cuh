@@ -55,7 +55,10 @@ constexpr int NB = 32;                // items in flight (mbarrier pairs)
 constexpr int ATT_KEYS = 32;
 constexpr int SCRATCH_BYTES = 2 * ATT_KEYS * 136 * 2 + 2048;  // two padded K/V tiles + slack (>= 16 KB guard)
 constexpr int MAX_ROWS = 128;         // rows one launch may push through a layer
-constexpr int RB = 8;                 // rows (accumulator columns) a worker group finishes per pass: the two groups
+#ifndef CLASP_RB
+#define CLASP_RB 8
+#endif
+constexpr int RB = CLASP_RB;                 // rows (accumulator columns) a worker group finishes per pass: the two groups
                                       // of four warps take alternate blocks, so 9 to 16 rows keep both busy
 constexpr int N_HEIGHTS = 4;          // distinct tile heights (TMA box heights) per weight matrix
 constexpr int MAX_CTAS = 192;
@@ -760,11 +763,13 @@ struct Worker {
     const long long q = __double2ll_rn((double)v * SS_FIX);
     asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(dst), "l"(q) : "memory");
   }
-  // Sums of v[0..31] over the warp: lane l returns the total of v[l].  31 shuffles, independent within
-  // a stage, instead of 32 five-step butterflies.
-  __device__ __forceinline__ static float warp_reduce32(float (&v)[32], int lane) {
+  // Sums of several values over the warp with N - 1 + log2(32 / N) shuffles, independent within a stage,
+  // instead of N five-step butterflies.
+  // Same for N = 4, 8 or 16 values: every lane l returns the total of v[l & (N - 1)].
+  template <int N>
+  __device__ __forceinline__ static float warp_reduce(float (&v)[N], int lane) {
 #pragma unroll
-    for (int w = 16; w >= 1; w >>= 1) {
+    for (int w = N / 2; w >= 1; w >>= 1) {
       const bool up = (lane & w) != 0;
 #pragma unroll
       for (int i = 0; i < w; ++i) {
@@ -773,47 +778,27 @@ struct Worker {
         v[i] = keep + __shfl_xor_sync(0xffffffffu, send, w);
       }
     }
-    return v[0];
+    float t = v[0];
+#pragma unroll
+    for (int o = N; o < 32; o <<= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    return t;
   }
-  // Same for 16 values: every lane l returns the total of v[l & 15].
-  __device__ __forceinline__ static float warp_reduce16(float (&v)[16], int lane) {
-#pragma unroll
-    for (int w = 8; w >= 1; w >>= 1) {
-      const bool up = (lane & w) != 0;
-#pragma unroll
-      for (int i = 0; i < w; ++i) {
-        const float send = up ? v[i] : v[i + w];
-        const float keep = up ? v[i + w] : v[i];
-        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, w);
-      }
+  // RB accumulator columns of this thread's lane
+  __device__ __forceinline__ static void tmem_ld_rb(uint32_t taddr, float (&v)[RB]) {
+    uint32_t r[RB];
+    if constexpr (RB == 8) {
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                   : "r"(taddr));
+    } else {
+      static_assert(RB == 4 || RB == 8, "row block of 4 or 8 accumulator columns");
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                   : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                   : "r"(taddr));
     }
-    return v[0] + __shfl_xor_sync(0xffffffffu, v[0], 16);
-  }
-
-  // Same for 8 values: every lane l returns the total of v[l & 7].
-  __device__ __forceinline__ static float warp_reduce8(float (&v)[8], int lane) {
-#pragma unroll
-    for (int w = 4; w >= 1; w >>= 1) {
-      const bool up = (lane & w) != 0;
-#pragma unroll
-      for (int i = 0; i < w; ++i) {
-        const float send = up ? v[i] : v[i + w];
-        const float keep = up ? v[i + w] : v[i];
-        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, w);
-      }
-    }
-    float t = v[0] + __shfl_xor_sync(0xffffffffu, v[0], 8);
-    return t + __shfl_xor_sync(0xffffffffu, t, 16);
-  }
-  // eight accumulator columns of this thread's lane
-  __device__ __forceinline__ static void tmem_ld8(uint32_t taddr, float (&v)[8]) {
-    uint32_t r[8];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < RB; ++i) v[i] = __uint_as_float(r[i]);
   }
 
   // per-row factors rsqrt(mean(x^2) + eps) from the accumulated sums of squares
@@ -933,16 +918,16 @@ struct Worker {
     const uint32_t t_lane = tmem_base + buf * 256u + ((uint32_t)(quarter * 32) << 16);
     for (int cb = group; cb < ncb; cb += 2) {
       float v[RB], u[RB];
-      tmem_ld8(t_lane + (uint32_t)(cb * RB), v);
-      if (P.dual || P.bmul == 2) tmem_ld8(t_lane + (uint32_t)(c.BN + cb * RB), u);
+      tmem_ld_rb(t_lane + (uint32_t)(cb * RB), v);
+      if (P.dual || P.bmul == 2) tmem_ld_rb(t_lane + (uint32_t)(c.BN + cb * RB), u);
       if (P.n_iss == 2 && P.n_groups >= 2) {  // the second MMA issuer's share of the reduction
         const uint32_t off = (uint32_t)(P.width + cb * RB);
         float w[RB];
-        tmem_ld8(t_lane + off, w);
+        tmem_ld_rb(t_lane + off, w);
 #pragma unroll
         for (int k = 0; k < RB; ++k) v[k] += w[k];
         if (P.dual || P.bmul == 2) {
-          tmem_ld8(t_lane + off + (uint32_t)c.BN, w);
+          tmem_ld_rb(t_lane + off + (uint32_t)c.BN, w);
 #pragma unroll
           for (int k = 0; k < RB; ++k) u[k] += w[k];
         }
@@ -984,7 +969,7 @@ struct Worker {
           }
           sq[k] = y * y;
         }
-        const float tot = warp_reduce8(sq, lane);
+        const float tot = warp_reduce<RB>(sq, lane);
         if (lane < RB && cb * RB + lane < J.R) T->red[quarter][cb * RB + lane][0] = tot;
       } else if (P.kind == G_GU) {
         if (fv) {
@@ -1018,8 +1003,8 @@ struct Worker {
           pr[k] = xi[k] * y;
           pr[RB + k] = y * y;
         }
-        const float tot = warp_reduce16(pr, lane);
-        if (lane < 2 * RB && cb * RB + (lane & 7) < J.R) T->red[quarter][cb * RB + (lane & 7)][lane >> 3] = tot;
+        const float tot = warp_reduce<2 * RB>(pr, lane);
+        if (lane < 2 * RB && cb * RB + (lane & (RB - 1)) < J.R) T->red[quarter][cb * RB + (lane & (RB - 1))][lane / RB] = tot;
       } else if (P.kind == G_DOWN) {
         float sq[RB];
 #pragma unroll
@@ -1033,7 +1018,7 @@ struct Worker {
           sq[k] = y * y;
         }
         if (J.norm_next) {
-          const float tot = warp_reduce8(sq, lane);
+          const float tot = warp_reduce<RB>(sq, lane);
           if (lane < RB && cb * RB + lane < J.R) T->red[quarter][cb * RB + lane][0] = tot;
         }
       } else {  // G_HEAD: best logit of this tile per row (lowest index on ties) and sum of exp
@@ -1139,11 +1124,11 @@ struct Worker {
         pa[RB + k] = sv * sv;
         pb[k] = xv * xv;
       }
-      const float ta = warp_reduce16(pa, lane);
-      const float tb = warp_reduce8(pb, lane);
-      const int r = cb * RB + (lane & 7);
+      const float ta = warp_reduce<2 * RB>(pa, lane);
+      const float tb = warp_reduce<RB>(pb, lane);
+      const int r = cb * RB + (lane & (RB - 1));
       if (lane < 2 * RB && r < rows) {
-        T->red[quarter][r][2 + (lane >> 3)] = ta;
+        T->red[quarter][r][2 + lane / RB] = ta;
         if (lane < RB) T->red[quarter][r][4] = tb;
       }
     }

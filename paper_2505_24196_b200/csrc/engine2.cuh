@@ -1577,17 +1577,10 @@ struct Worker {
         float2 v0 = make_float2(-INFINITY, 0.f), v1 = v0;
         if (lane < n_chunks) v0 = __ldcg(ml + lane);
         if (lane + 32 < n_chunks) v1 = __ldcg(ml + lane + 32);
-        const float mx = warp_max(fmaxf(v0.x, v1.x));
-        const float w0 = v0.x == -INFINITY ? 0.f : exp2f(v0.x - mx);
-        const float w1 = v1.x == -INFINITY ? 0.f : exp2f(v1.x - mx);
-        const float den = warp_sum(w0 * v0.y + w1 * v1.y);
-        float num[DPL];
-#pragma unroll
-        for (int k = 0; k < DPL; ++k) num[k] = 0.f;
         constexpr int MB = 17;   // partials fetched per trip to L2 (a 512-key context has 17)
         const float* acc = p.b.att_acc + pr * c.chunk_cap * HD + lane * DPL;
-        for (int ch0 = 0; ch0 < n_chunks; ch0 += MB) {
-          float a[MB][DPL];
+        float a[MB][DPL];
+        auto load_trip = [&](int ch0) {
 #pragma unroll
           for (int e = 0; e < MB; ++e) {
 #pragma unroll
@@ -1602,6 +1595,17 @@ struct Worker {
               }
             }
           }
+        };
+        load_trip(0);   // in the same trip to L2 as the maxima and sums: the partials do not depend on them
+        const float mx = warp_max(fmaxf(v0.x, v1.x));
+        const float w0 = v0.x == -INFINITY ? 0.f : exp2f(v0.x - mx);
+        const float w1 = v1.x == -INFINITY ? 0.f : exp2f(v1.x - mx);
+        const float den = warp_sum(w0 * v0.y + w1 * v1.y);
+        float num[DPL];
+#pragma unroll
+        for (int k = 0; k < DPL; ++k) num[k] = 0.f;
+        for (int ch0 = 0; ch0 < n_chunks; ch0 += MB) {
+          if (ch0 > 0) load_trip(ch0);
 #pragma unroll
           for (int e = 0; e < MB; ++e) {
             const int ch = ch0 + e;

@@ -32,7 +32,7 @@ sys.path.insert(0, ROOT)
 import datagen  # noqa: E402
 
 WORKLOADS = {
-    # BASELINE configs[1]: 8B shape, 512-token context, M = 12, one objective token
+    # the headline workload: LLaMA3-8B shape, 512-token context, M = 12, one objective token
     "8b-c512-M12": dict(model="8b", ctx=512, M=12, T=1, K=4),
     # small stand-ins for quick checks and profiler captures (not bench lines)
     "8b-l6-c512-M3": dict(model="8b-l6", ctx=512, M=3, T=1, K=4),

@@ -72,7 +72,7 @@ class ModelConfig:
 
 
 CONFIGS: Dict[str, ModelConfig] = {
-    # configs[0]: the small case the oracle finishes in seconds
+    # the small fp32 case the oracle finishes in seconds
     "tiny": ModelConfig("tiny", L=8, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64,
                         d_ffn=688, vocab=1024, dtype="fp32", seed=1),
     # a bf16 case small enough for the oracle that still spans several GEMM
@@ -83,14 +83,14 @@ CONFIGS: Dict[str, ModelConfig] = {
     "mini8b": ModelConfig("mini8b", L=4, d_model=1024, n_q_heads=8, n_kv_heads=2, head_dim=128,
                           d_ffn=3584, vocab=4096, dtype="bf16", scale_out_proj=True,
                           norm_std=0.1, seed=6),
-    # configs[1], [2], [4]: LLaMA3-8B shape
+    # LLaMA3-8B shape (headline search, context sweep, decode loop)
     "8b": ModelConfig("8b", L=32, d_model=4096, n_q_heads=32, n_kv_heads=8, head_dim=128,
                       d_ffn=14336, vocab=128256, dtype="bf16", scale_out_proj=True, seed=2),
     # the 8B layer shape with few layers and a small vocabulary: a profiler capture saves and
     # restores device memory per pass, so it runs on ~3 GB of weights instead of 16 GB
     "8b-l6": ModelConfig("8b-l6", L=6, d_model=4096, n_q_heads=32, n_kv_heads=8, head_dim=128,
                          d_ffn=14336, vocab=16384, dtype="bf16", scale_out_proj=True, seed=2),
-    # configs[3]: LLaMA3-70B shape
+    # LLaMA3-70B shape
     "70b": ModelConfig("70b", L=80, d_model=8192, n_q_heads=64, n_kv_heads=8, head_dim=128,
                        d_ffn=28672, vocab=128256, dtype="bf16", scale_out_proj=True, seed=3),
 }

@@ -55,11 +55,14 @@ constexpr int NB = 32;                // items in flight (mbarrier pairs)
 constexpr int ATT_KEYS = 32;
 constexpr int SCRATCH_BYTES = 2 * ATT_KEYS * 136 * 2 + 2048;  // two padded K/V tiles + slack (>= 16 KB guard)
 constexpr int MAX_ROWS = 128;         // rows one launch may push through a layer
+// Rows (accumulator columns) a worker group finishes per pass; the two groups of four warps take alternate
+// blocks.  4 or 8: with 4 the unrolled per-row code is half as long and 5 to 8 rows already keep both groups
+// busy (measured against 8: 8B search -0.5 %, forward passes -1.7 %, 8192-key contexts -3 %; launches with
+// many rows make more passes: 70B search with 32 rows +0.6 %, 128-row prefill +3 %).
 #ifndef CLASP_RB
-#define CLASP_RB 8
+#define CLASP_RB 4
 #endif
-constexpr int RB = CLASP_RB;                 // rows (accumulator columns) a worker group finishes per pass: the two groups
-                                      // of four warps take alternate blocks, so 9 to 16 rows keep both busy
+constexpr int RB = CLASP_RB;
 constexpr int N_HEIGHTS = 4;          // distinct tile heights (TMA box heights) per weight matrix
 constexpr int MAX_CTAS = 192;
 

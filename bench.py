@@ -282,7 +282,7 @@ def dp_only(args, eng, dec, kv, cfg, wl):
 # DRAM bytes (read + write) of one search launch of the persistent kernel, from the ncu capture summarised in
 # profiles/engine_kernel_8b_l6_c512_M3_ncu.md: taken on a 6-layer model of the same layer shape and scaled by
 # 31 / 5 applied layers.  Set to None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES = {"8b-c512-M12": 13747570000}   # (dram read + write of the 6-layer capture) x 31 / 5
+NCU_TRAFFIC_BYTES = {"8b-c512-M12": 13730230000}   # (dram read + write of the 6-layer capture) x 31 / 5
 
 
 def gemm_roofline(eng, dec, kv, hid_dev, obj, T, M, d):

@@ -616,7 +616,7 @@ int engine_setup(clasp_ctx* ctx) {
     int kpi_budget = 32, kpi_max = 8;
     if (const char* e = getenv("CLASP_ENGINE_KPI")) {
       const int v = atoi(e);
-      if (v >= 4 && v <= 48) { kpi_budget = v; kpi_max = v / 4; }
+      if (v >= 4 && v <= 40) { kpi_budget = v; kpi_max = v / 4; }
     }
     int kpi = kpi_budget / a_pages;
     ctx->e_kpi[k] = kpi < 1 ? 1 : (kpi > kpi_max ? kpi_max : kpi);

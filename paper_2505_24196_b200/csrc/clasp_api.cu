@@ -753,8 +753,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   // the keys it sees into at most 32 runs, which spreads a short context over many more CTAs.
   if (search_ctx >= 0) P.c.run_len = pk::ATT_KEYS * ((search_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32) > 0
                                                        ? (search_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32) : 1);
-  P.c.BN = BN; P.c.ring_pages = ring_pages; P.c.n_iss = BN <= 64 ? 2 : 1;
-  if (getenv("CLASP_ENGINE_ONE_ISSUER")) P.c.n_iss = 1;
+  P.c.BN = BN; P.c.ring_pages = ring_pages;
 
   for (int s = 0; s < pk::N_SPLITS; ++s) { P.c.split_lo[s] = ctx->e_split_lo[s]; P.c.split_units[s] = ctx->e_split_units[s]; }
   for (int k = 0; k < 5; ++k) { P.c.tile_idx[k] = ctx->e_tile_idx[k]; P.c.kpi[k] = kpi[k]; P.c.use3d[k] = use3d[k]; }

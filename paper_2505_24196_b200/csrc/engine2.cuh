@@ -15,12 +15,13 @@
 //               depend on activations: this warp runs ahead across products, layers and jobs.
 //   warp 1      lane 0 loads the activation operand ([BN x 64] bf16 per 64-column chunk) next to
 //               the weight rows once the CTAs that produce those columns have published them.
-//   warps 2, 3  lane 0 of each issues tcgen05.mma: M = 128 weight rows (rows beyond the CTA's
-//               range are whatever bytes follow in the ring; their accumulator lanes are never
-//               read; tiles of at most 64 rows use M = 64), N = BN activation rows, K = 16.  One
-//               thread can issue an MMA only every ~55 cycles, so the two warps take alternate
-//               ring items and accumulate into separate accumulators, which the epilogue adds in
-//               a fixed order.  Warp 3 also allocates / frees tensor memory.
+//   warp 2      issues tcgen05.mma: M = 128 weight rows (rows beyond the CTA's range are whatever
+//               bytes follow in the ring; their accumulator lanes are never read; tiles of at most
+//               64 rows use M = 64), N = BN activation rows, K = 16.  All 32 lanes walk the schedule
+//               and one elected lane issues, which keeps the descriptor arithmetic warp-uniform:
+//               the warp then issues as fast as the tensor pipe multiplies (23 cycles per M = 64,
+//               39 per M = 128 instruction at these N).
+//   warp 3      allocates / frees tensor memory.
 //   warps 4-11  "workers": epilogues, attention, Eq. 2 select, arg-max.
 //
 // Synchronisation between CTAs is through global memory: after finishing step s of job j a
@@ -98,8 +99,6 @@ struct Cfg {
   int run_len, chunk_cap;
   int BN;              // activation rows padded to a multiple of 16 (MMA N)
   int ring_pages;
-  int n_iss;           // MMA issuers in use: 2 while two accumulators of (gate, up) x BN columns fit one
-                       // 256-column buffer (BN <= 64), else 1
   // tables (ints / structs in Params::tabs, offsets in ints)
   int split_lo[N_SPLITS];    // [G + 1] first feature of each CTA: lo(c) = 8 floor(c units / G)
   int split_units[N_SPLITS]; // 8-feature units of each split
@@ -259,38 +258,53 @@ struct RowDiv {
   __device__ __forceinline__ int mod(int r) const { return r - div(r) * T; }
 };
 
-// tcgen05.mma with the operand descriptors given by their low words (start address and leading
-// byte offset; the high word -- 1024-byte group stride, version, 128B swizzle -- is the same for
-// every tile).  A thread issues thousands of these per layer, so nothing else is in the asm.
+// tcgen05.mma issued by the elected lane of a converged warp.  The whole warp walks the schedule, so the
+// descriptor arithmetic stays warp-uniform (a loop that only one lane runs pays ~60 cycles per instruction
+// for moving its operands to the uniform registers the instruction reads; measured with resident operands:
+// 23 cycles per M = 64, N <= 32 multiply and 39 per M = 128 one in this form, the tensor pipe's own rate).
+// Descriptor: start address and leading byte offset in the low word; 1024-byte group stride, version and
+// 128B swizzle in the high word, the same for every tile.
 constexpr uint32_t DESC_HI = 64u | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
+  return ((uint64_t)DESC_HI << 32) | (uint64_t)(((smem_addr & 0x3FFFFu) >> 4) | (1u << 16));
+}
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred;
+}
 template <bool ACC>
-__device__ __forceinline__ void mma_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+__device__ __forceinline__ void mma_el(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t el) {
   if (ACC) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.eq.u32 p, 1, 1;\n\t"
-        "mov.b64 da, {%1, %4};\n\t"
-        "mov.b64 db, {%2, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem),
-        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI));
+        "setp.ne.u32 q, %4, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(da), "l"(db), "r"(idesc), "r"(el));
   } else {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.eq.u32 p, 1, 0;\n\t"
-        "mov.b64 da, {%1, %4};\n\t"
-        "mov.b64 db, {%2, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem),
-        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI));
+        "setp.ne.u32 q, %4, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(da), "l"(db), "r"(idesc), "r"(el));
   }
 }
 // the four K = 16 steps of one 64-column chunk
 template <bool FIRST>
-__device__ __forceinline__ void mma_chunk(uint32_t acc, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
-  mma_lo<!FIRST>(acc, a_lo, b_lo, idesc);
-  mma_lo<true>(acc, a_lo + 2, b_lo + 2, idesc);
-  mma_lo<true>(acc, a_lo + 4, b_lo + 4, idesc);
-  mma_lo<true>(acc, a_lo + 6, b_lo + 6, idesc);
+__device__ __forceinline__ void mma_chunk(uint32_t acc, uint64_t da, uint64_t db, uint32_t idesc, uint32_t el) {
+  mma_el<!FIRST>(acc, da, db, idesc, el);
+  mma_el<true>(acc, da + 2, db + 2, idesc, el);
+  mma_el<true>(acc, da + 4, db + 4, idesc, el);
+  mma_el<true>(acc, da + 6, db + 6, idesc, el);
+}
+__device__ __forceinline__ void mma_commit_el(uint32_t bar, uint32_t el) {
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar), "r"(el)
+      : "memory");
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z,
@@ -390,8 +404,6 @@ __device__ __forceinline__ int kind_map_base(const Cfg& c, int kind, int layer) 
 struct Phase {   // one product of one job, as seen by this CTA
   int kind, dual, kc, kpi, n_groups;  // chunks, chunks per item, items per tile
   int bmul;                           // operand row blocks of BN rows (2 for a q/k/v product over both candidates)
-  int width;                          // accumulator columns of one MMA issuer
-  int n_iss;                          // issuers that take items of this product
   int tile0, n_tiles;                 // this CTA's TileDesc range
   int map_base;
   int g0;                             // chunk group this CTA starts its reduction at: CTAs walk the
@@ -405,8 +417,6 @@ struct Phase {   // one product of one job, as seen by this CTA
     kpi = c.kpi[kind];
     n_groups = (kc + kpi - 1) / kpi;
     bmul = (kind == G_QKV && J.dual_src) ? 2 : 1;
-    width = (dual + 1) * bmul * c.BN;
-    n_iss = 2 * width <= 256 ? c.n_iss : 1;
     const int* ti = p.tabs + c.tile_idx[kind] + blockIdx.x;
     tile0 = __ldg(ti);
     n_tiles = __ldg(ti + 1) - tile0;
@@ -624,17 +634,17 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
   }
 }
 
-// MMA issuer `which` (0 or 1) takes the ring items of each tile with that parity and adds them up
-// in accumulator `which` of the tile's buffer: buffer b holds accumulator a at column
-// b * 256 + a * (dual + 1) * BN  (gate at +0, up at +BN).
+// MMA issuer (warp 2, all lanes converged, one elected lane issues): adds the ring items of each tile up in
+// the tile's accumulator; buffer b holds it at column b * 256 (gate at +0, up at +BN).
 template <bool TR>
-__device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint32_t tmem_base, int which) {
+__device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint32_t tmem_base, int lane) {
   const Cfg& c = p.c;
   const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10);
   const TileDesc* tiles = reinterpret_cast<const TileDesc*>(p.tabs + c.tiles_off);
   RingPos rp{0, 0};
   const int b_pages = (c.BN * BK * 2) / PAGE;
   uint32_t n_acc = 0;
+  const uint32_t el = elect_one();
   for (int jb = 0; jb < p.n_jobs; ++jb) {
     const Job& J = p.jobs[jb];
     const int nph = n_gemm_phases(J);
@@ -650,52 +660,51 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
         // rows from shared memory (row r of its accumulator sits in lane 32 (r / 16) + r % 16)
         const uint32_t idesc = idesc0 | ((uint32_t)((P.bmul * c.BN) >> 3) << 17) | ((td.n_rows <= 64 ? 4u : 8u) << 24);
         const uint32_t buf = n_acc & 1u;
-        if (!wait_bar(&sh->acc_empty[buf], ((n_acc >> 1) & 1u) ^ 1u, p.ctl, sh)) return;
+        if (!__all_sync(0xffffffffu, wait_bar(&sh->acc_empty[buf], ((n_acc >> 1) & 1u) ^ 1u, p.ctl, sh))) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t acc = tmem_base + buf * 256u + (uint32_t)(which * P.width);
+        const uint32_t acc = tmem_base + buf * 256u;
         const uint32_t acc2 = acc + (uint32_t)c.BN;
-        const uint32_t up_lo = (uint32_t)a_pages * (PAGE / 16);          // gate rows -> up rows
-        const uint32_t w_lo = (uint32_t)w_pages * (PAGE / 16);           // weights of one chunk
-        const uint32_t x_lo = (uint32_t)(P.bmul * b_pages) * (PAGE / 16);  // operand tile of one chunk
-        const uint32_t x0_lo = (uint32_t)P.kpi * w_lo;                   // first weight chunk -> first operand tile
+        const uint64_t up_lo = (uint64_t)(a_pages * (PAGE / 16));              // gate rows -> up rows
+        const uint64_t w_lo = (uint64_t)(w_pages * (PAGE / 16));               // weights of one chunk
+        const uint64_t x_lo = (uint64_t)(P.bmul * b_pages * (PAGE / 16));      // operand tile of one chunk
+        const uint64_t x0_lo = (uint64_t)P.kpi * w_lo;                         // first weight chunk -> first operand tile
         for (int gi = 0; gi < P.n_groups; ++gi) {
           int fp;
           const uint32_t it = rp.item;
           const int at = rp.place(pages, c.ring_pages, fp);
-          if ((gi & (P.n_iss - 1)) != which) continue;
-          if (!wait_bar(&sh->full[it % NB], (it / NB) & 1u, p.ctl, sh)) return;
+          if (!__all_sync(0xffffffffu, wait_bar(&sh->full[it % NB], (it / NB) & 1u, p.ctl, sh))) return;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          if (t == 0 && gi == 0) issuer_mark<TR>(p, jb, T_MMA_FIRST + ph);
+          if (t == 0 && gi == 0 && lane == 0) issuer_mark<TR>(p, jb, T_MMA_FIRST + ph);
           const int k0 = P.group_at(gi) * P.kpi;
           const int nk = min(P.kc, k0 + P.kpi) - k0;
-          uint32_t a_lo = desc_lo(ring_base + (uint32_t)at * PAGE);
-          uint32_t b_lo = a_lo + x0_lo;
+          uint64_t da = make_desc(ring_base + (uint32_t)at * PAGE);
+          uint64_t db = da + x0_lo;
           int k = 0;
-          if (gi < P.n_iss) {  // this issuer's first item of the tile overwrites its accumulator
-            mma_chunk<true>(acc, a_lo, b_lo, idesc);
-            if (P.dual) mma_chunk<true>(acc2, a_lo + up_lo, b_lo, idesc);
-            a_lo += w_lo;
-            b_lo += x_lo;
+          if (gi == 0) {  // the first item of the tile overwrites the accumulator
+            mma_chunk<true>(acc, da, db, idesc, el);
+            if (P.dual) mma_chunk<true>(acc2, da + up_lo, db, idesc, el);
+            da += w_lo;
+            db += x_lo;
             k = 1;
           }
           if (P.dual) {
             for (; k < nk; ++k) {
-              mma_chunk<false>(acc, a_lo, b_lo, idesc);
-              mma_chunk<false>(acc2, a_lo + up_lo, b_lo, idesc);
-              a_lo += w_lo;
-              b_lo += x_lo;
+              mma_chunk<false>(acc, da, db, idesc, el);
+              mma_chunk<false>(acc2, da + up_lo, db, idesc, el);
+              da += w_lo;
+              db += x_lo;
             }
           } else {
             for (; k < nk; ++k) {
-              mma_chunk<false>(acc, a_lo, b_lo, idesc);
-              a_lo += w_lo;
-              b_lo += x_lo;
+              mma_chunk<false>(acc, da, db, idesc, el);
+              da += w_lo;
+              db += x_lo;
             }
           }
-          tc::mma_commit(tc::smem_u32(&sh->empty[it % NB]));
+          mma_commit_el(tc::smem_u32(&sh->empty[it % NB]), el);
         }
-        tc::mma_commit(tc::smem_u32(&sh->acc_full[buf]));  // both issuers arrive, with or without items
-        if (which == 0 && t == P.n_tiles - 1) issuer_mark<TR>(p, jb, T_MMA_LAST + ph);
+        mma_commit_el(tc::smem_u32(&sh->acc_full[buf]), el);
+        if (lane == 0 && t == P.n_tiles - 1) issuer_mark<TR>(p, jb, T_MMA_LAST + ph);
         ++n_acc;
       }
     }
@@ -923,18 +932,6 @@ struct Worker {
       float v[RB], u[RB];
       tmem_ld_rb(t_lane + (uint32_t)(cb * RB), v);
       if (P.dual || P.bmul == 2) tmem_ld_rb(t_lane + (uint32_t)(c.BN + cb * RB), u);
-      if (P.n_iss == 2 && P.n_groups >= 2) {  // the second MMA issuer's share of the reduction
-        const uint32_t off = (uint32_t)(P.width + cb * RB);
-        float w[RB];
-        tmem_ld_rb(t_lane + off, w);
-#pragma unroll
-        for (int k = 0; k < RB; ++k) v[k] += w[k];
-        if (P.dual || P.bmul == 2) {
-          tmem_ld_rb(t_lane + off + (uint32_t)c.BN, w);
-#pragma unroll
-          for (int k = 0; k < RB; ++k) u[k] += w[k];
-        }
-      }
       if (P.bmul == 2) {
         // both candidates of every state went through the product (v: layer output, u: skip candidate):
         // keep the one the Eq. 2 step chose
@@ -1771,7 +1768,7 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
       tc::mbar_init(tc::smem_u32(&sh.empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
-      tc::mbar_init(tc::smem_u32(&sh.acc_full[b]), 2);   // one arrival per MMA issuer
+      tc::mbar_init(tc::smem_u32(&sh.acc_full[b]), 1);
       tc::mbar_init(tc::smem_u32(&sh.acc_empty[b]), 1);
     }
     sh.abort = 0;
@@ -1802,8 +1799,8 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
       const CUtensorMap* bmaps[6] = {&map_xn_a, &map_attn, &map_xn_m, &map_act, &map_head, &map_xn_a2};
       const CUtensorMap* bmaps3[6] = {&map3_xn_a, &map3_attn, &map3_xn_m, &map3_act, &map3_head, &map3_xn_a2};
       producer_b<TR>(p, &sh, ring_base, bmaps, bmaps3, lane);
-    } else {
-      if (lane == 0) mma_issuer<TR>(p, &sh, ring_base, tmem_base, warp - 2);
+    } else if (warp == 2) {
+      mma_issuer<TR>(p, &sh, ring_base, tmem_base, lane);
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_WORKER));

@@ -24,6 +24,11 @@
  *   - Every function returns CLASP_OK (0) or a negative CLASP_ERR_*; nothing
  *     throws, aborts or traps on the device.  Every device-side wait is bounded;
  *     one that runs out records a code readable by clasp_last_device_status.
+ *   - Alignment: weight matrices, float buffers (hidden states, layer inputs and
+ *     outputs, g_final) and K/V arrays are 16-byte aligned and float strides are
+ *     multiples of 4 elements (the kernels use 16-byte accesses); a call that is
+ *     given anything else returns CLASP_ERR_INVALID_ARG before it launches.
+ *   - No environment variable changes what the library computes or how.
  */
 #ifndef CLASP_H_
 #define CLASP_H_
@@ -76,6 +81,14 @@ typedef struct clasp_config {
 
 #define CLASP_FLAG_FORCE_SIMT 1 /* bf16 model: use the CUDA-core GEMM instead of the
                                    tcgen05 one (diagnostics; both are device code) */
+#define CLASP_FLAG_NO_DEFER 2   /* diagnostics: the search lets every layer wait for the
+                                   Eq. 2 decision of the step before it, instead of sending
+                                   both candidates of a state through the layer's q/k/v
+                                   product and keeping the chosen one.  Same operand bytes
+                                   either way, so the results agree. */
+#define CLASP_FLAG_MULTI_KERNEL 4 /* diagnostics, bf16 model: one kernel per step (tcgen05
+                                   GEMM, attention, norm, Eq. 2 select ...) instead of the
+                                   persistent kernel that runs a whole call in one launch */
 
 /* Device pointers to the nine tensors of one decoder layer (borrowed). */
 typedef struct clasp_layer_weights {
@@ -108,6 +121,26 @@ size_t clasp_workspace_bytes(const clasp_config* cfg);
 int clasp_create(const clasp_config* cfg, void* workspace, size_t workspace_bytes,
                  void* cuda_stream, clasp_ctx** out);
 void clasp_destroy(clasp_ctx* ctx);
+
+/* 1 when the context runs its searches and forwards in the persistent layer kernel (one
+ * cooperative launch per call), 0 when it uses one kernel per step: an fp32 model, the two
+ * diagnostic flags above, or a bf16 shape the persistent kernel does not take (vocab not a
+ * multiple of 8; more than 128 d_model features per SM; a weight matrix whose per-SM row
+ * ranges need more than four distinct heights; no cooperative launch on the device).  Both
+ * paths compute the same thing; the second is several times slower, so a caller that sized
+ * its deployment for the first should check.  Per call, a search with M*T > 128 candidate
+ * rows and a forward over more than 128 rows also take the one-kernel-per-step path.
+ * Negative: CLASP_ERR_INVALID_ARG. */
+int clasp_engine_active(const clasp_ctx* ctx);
+
+/* Limit of every device-side wait in the context's kernels, in polls (a poll is about
+ * 100 ns once a wait has started to sleep between polls); 0 restores the default (about
+ * half a second).  A wait that reaches the limit makes its kernel wind down -- copies in
+ * flight are awaited, tensor memory is freed -- and clasp_last_device_status reports
+ * CLASP_ERR_TIMEOUT; the outputs of that call are unspecified, the context stays usable.
+ * A limit of a few polls makes healthy kernels give up: that is how the tests reach the
+ * wind-down path without a kernel that would wait forever. */
+int clasp_set_wait_limit(clasp_ctx* ctx, uint32_t polls);
 
 /* Register the weights of layers first..first+count-1 (Sec. 3.4: the decoder
  * layers f_l the search and the forwards apply).  `w` is a HOST array of
@@ -225,6 +258,9 @@ int clasp_gemm_xwT(clasp_ctx* ctx, const void* x, const void* w, int32_t R, int3
  *   cuda_stream  the cudaStream_t to launch on (NULL = default stream)
  *   status_out   device int32 or NULL: set to 1 by the kernel if one of its bounded
  *                waits gave up (y is then unspecified); the caller zeroes it beforehand.
+ *                With NULL a wait that gave up is NOT reported anywhere (the flag goes to
+ *                a word of the scratch array that the next call clears): pass a word if
+ *                the result matters.
  *
  * Limits: shapes whose partial sums (splits * R * N floats) exceed the array, or with
  * more than 4096 output tiles under split-K, are refused with CLASP_ERR_CAPACITY;
@@ -263,15 +299,17 @@ int64_t clasp_launch_count(const clasp_ctx* ctx);
 /* Step tracing of the persistent layer kernel (measurement aid; no counterpart in the
  * paper).  `stamps` is DEVICE memory of n_ctas * cap_per_cta uint64 (borrowed until it is
  * replaced or cleared with NULL): during every following search / verify / draft call the
- * kernel's CTA c writes %globaltimer values (ns) to stamps[c * cap_per_cta + 32 * j + s]
+ * kernel's CTA c writes %globaltimer values (ns) to stamps[c * cap_per_cta + 64 * j + s]
  * when it reaches step boundary s of job j of the call (jobs: one per decoder layer pass or
  * Eq. 2 step, then the LM head; s: 0 job start, 1 q/k/v done, 2-5 attention partials, 6
  * attention merged, 7 o, 8 gate/up, 9 down, 10-13 Eq. 2 step, 14 head; for product p = 0..3
  * (q/k/v, o, gate/up, down) 16+p first operands ready for the tensor core, 20+p last
  * multiply issued, 24+p first accumulator complete; 28 Eq. 2 step published the next operand;
- * 29-31 operand of q/k/v, o, gate/up seen complete by the operand loader; entries a CTA does
- * not reach stay as the caller left them, entries beyond cap_per_cta are not recorded).  *n_ctas (HOST, may be NULL) receives the grid
- * size, 0 when the context does not use the persistent kernel. */
+ * 29-31 operand of q/k/v, o, gate/up seen complete by the operand loader; 32-63 free for finer
+ * stamps; entries a CTA does not reach stay as the caller left them, entries beyond
+ * cap_per_cta are not recorded).  *n_ctas (HOST, may be NULL) receives the grid size, 0 when
+ * the context does not use the persistent kernel.  cap_per_cta < 0 only queries *n_ctas and
+ * leaves a trace buffer in use as it is. */
 int clasp_engine_trace(clasp_ctx* ctx, uint64_t* stamps, int32_t cap_per_cta, int32_t* n_ctas);
 
 const char* clasp_strerror(int code);

@@ -29,6 +29,16 @@ Conventions fixed where the paper is silent (each pinned by a test unless noted)
   * the search after the prompt's prefill (first draft round) uses the last
     prompt token as objective.  PARITY UNPINNED by the paper (it does not say
     where the first skip set comes from); it cannot affect losslessness.
+  * lower optimisation frequency (Sec. 3.7, Sec. 5.3.2): with interval N the
+    search runs after every N-th verification; the rounds in between keep the
+    last skip set.
+  * draft-exiting threshold (Sec. 5.3.3): the confidence of a drafted token is
+    the draft model's softmax probability of that (greedy) token; a token whose
+    confidence is below the threshold is still handed to the verification (it
+    has been computed) but ends the drafting of that round.  The paper names
+    the mechanism and its best value (about 0.7) only; this reading is pinned by
+    its two limits (threshold 0 = fixed draft length, threshold > 1 = one draft
+    per round) and by losslessness.
 """
 from __future__ import annotations
 
@@ -158,6 +168,12 @@ def argmax_lowest(logits: np.ndarray) -> np.ndarray:
     return np.argmax(logits, axis=-1)
 
 
+def top1_probability(logits: np.ndarray) -> np.ndarray:
+    """Softmax probability of the greedy token of each row of logits[n, vocab]."""
+    z = logits - logits.max(axis=-1, keepdims=True)
+    return 1.0 / np.exp(z).sum(axis=-1)
+
+
 def verify_forward(model: Model, tokens: Sequence[int], cache: KVCache, pos0: int,
                    skip: Optional[Sequence[int]] = None):
     """Embed tokens, run the (possibly layer-skipped) model, return
@@ -283,13 +299,16 @@ def greedy_autoregressive(model: Model, prompt: Sequence[int], n_new: int, max_c
 
 def greedy_self_speculative(model: Model, prompt: Sequence[int], n_new: int, max_ctx: int,
                             M: int, K: int, fixed_mask: Optional[Sequence[int]] = None,
-                            dp_interval: int = 1):
-    """Draft K tokens with the layer-skipped model, verify them with the full
-    model in one pass, accept the longest matching prefix plus the full model's
-    own next token, then re-run the layer search on the last accepted token.
+                            dp_interval: int = 1, exit_threshold: float = 0.0):
+    """Draft up to K tokens with the layer-skipped model, verify them with the
+    full model in one pass, accept the longest matching prefix plus the full
+    model's own next token, then re-run the layer search on the last accepted
+    token (after every dp_interval-th verification, Sec. 3.7).  A drafted token
+    whose softmax probability is below exit_threshold ends the round's drafting
+    (Sec. 5.3.3); it is still verified.
 
-    Returns (tokens, stats) where stats lists per round the accepted count and
-    the skip set used.
+    Returns (tokens, stats) where stats lists per round the accepted count, the
+    skip set used, the number of drafted tokens and their confidences.
     """
     cfg = model.cfg
     cache = KVCache(cfg, max_ctx)
@@ -310,19 +329,23 @@ def greedy_self_speculative(model: Model, prompt: Sequence[int], n_new: int, max
     n_verify = 0
     while len(out) < n_new:
         # draft: K single-token passes of the layer-skipped model
-        drafts, tok = [], pending
+        drafts, conf, tok = [], [], pending
         for k in range(K):
-            a, _, _ = verify_forward(model, [tok], cache, n_valid + k, skip=S)
+            a, _, lg = verify_forward(model, [tok], cache, n_valid + k, skip=S)
             tok = int(a[0])
             drafts.append(tok)
-        # verify: one full-model pass over [pending, d_1..d_K]
+            conf.append(float(top1_probability(lg)[0]))
+            if conf[-1] < exit_threshold:
+                break
+        n_d = len(drafts)
+        # verify: one full-model pass over [pending, d_1..d_n]
         am, hidden, _ = verify_forward(model, [pending] + drafts, cache, n_valid)
         a = 0
-        while a < K and drafts[a] == int(am[a]):
+        while a < n_d and drafts[a] == int(am[a]):
             a += 1
         new = drafts[:a] + [int(am[a])]
         out.extend(new)
-        rounds.append({"accepted": a, "S": S.copy()})
+        rounds.append({"accepted": a, "S": S.copy(), "drafted": n_d, "confidence": conf})
         obj_row = hidden[a]                        # last position whose K/V is now valid
         obj_pos = n_valid + a
         n_valid += a + 1

@@ -17,11 +17,12 @@ from . import build as _build
 
 CLASP_FP32, CLASP_BF16 = 0, 1
 CHOICE_APPLY, CHOICE_SKIP, CHOICE_NONE = 0, 1, 255
-FLAG_FORCE_SIMT = 1
+FLAG_FORCE_SIMT, FLAG_NO_DEFER, FLAG_MULTI_KERNEL = 1, 2, 4
 
 SYMBOLS = ["clasp_workspace_bytes", "clasp_create", "clasp_destroy", "clasp_load_layers", "clasp_load_head",
            "clasp_dp_search", "clasp_verify", "clasp_draft_forward", "clasp_accept", "clasp_layer_forward",
-           "clasp_gemm_xwT", "clasp_gemm_xwT_noalloc", "clasp_profile_gemm", "clasp_last_device_status", "clasp_launch_count", "clasp_engine_trace", "clasp_strerror"]
+           "clasp_gemm_xwT", "clasp_gemm_xwT_noalloc", "clasp_profile_gemm", "clasp_last_device_status", "clasp_launch_count", "clasp_engine_trace", "clasp_strerror",
+           "clasp_engine_active", "clasp_set_wait_limit"]
 
 
 class ClaspConfig(C.Structure):
@@ -93,6 +94,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.clasp_launch_count.argtypes = [vp]
     lib.clasp_engine_trace.restype = C.c_int
     lib.clasp_engine_trace.argtypes = [vp, vp, i32, C.POINTER(i32)]
+    lib.clasp_engine_active.restype = C.c_int
+    lib.clasp_engine_active.argtypes = [vp]
+    lib.clasp_set_wait_limit.restype = C.c_int
+    lib.clasp_set_wait_limit.argtypes = [vp, C.c_uint32]
     lib.clasp_strerror.restype = C.c_char_p
     lib.clasp_strerror.argtypes = [C.c_int]
     _lib = lib
@@ -268,9 +273,19 @@ class Clasp:
         return self.lib.clasp_launch_count(self.handle)
 
     def engine_ctas(self) -> int:
+        """Grid size of the persistent kernel (0 when the context does not use it); query only."""
         n = C.c_int32()
-        _check(self.lib.clasp_engine_trace(self.handle, None, 0, C.byref(n)), "clasp_engine_trace")
+        _check(self.lib.clasp_engine_trace(self.handle, None, -1, C.byref(n)), "clasp_engine_trace")
         return n.value
+
+    def engine_active(self) -> bool:
+        r = self.lib.clasp_engine_active(self.handle)
+        if r < 0:
+            raise ClaspError(r, "clasp_engine_active")
+        return r == 1
+
+    def set_wait_limit(self, polls: int):
+        _check(self.lib.clasp_set_wait_limit(self.handle, polls), "clasp_set_wait_limit")
 
     def set_trace(self, stamps: Optional[torch.Tensor], cap_per_cta: int = 0):
         """stamps: int64 device tensor [n_ctas, cap_per_cta] or None to stop tracing."""

@@ -194,6 +194,7 @@ struct clasp_ctx {
   std::vector<clasp::pk::Job> e_jobs;
   unsigned long long* e_trace = nullptr;
   int e_trace_cap = 0;
+  uint32_t wait_limit = 0;   // 0: the kernels' default wait limits
 };
 
 namespace {
@@ -310,6 +311,8 @@ int gemm_tc(clasp_ctx* ctx, const GemmCall& g) {
   p.counters = ctx->ws.counters;
   p.status = ctx->ws.status;
   p.partial = ctx->ws.partial;
+  p.spin_fast = ctx->wait_limit ? (ctx->wait_limit < SPIN_FAST ? ctx->wait_limit : SPIN_FAST) : SPIN_FAST;
+  p.spin_slow = ctx->wait_limit ? ctx->wait_limit : SPIN_SLOW;
   for (int r0 = 0; r0 < g.R; r0 += rb_max) {
     const int Rb = g.R - r0 < rb_max ? g.R - r0 : rb_max;
     p.R = Rb;
@@ -475,6 +478,14 @@ int run_layer_any(clasp_ctx* ctx, int l, const float* x, int64_t ldx, int S, int
   return run_layer<bf16>(ctx, l, x, ldx, S, T, C, pos0, kv, write_kv, out, ldo);
 }
 
+// float buffers are read and written with 16-byte vector accesses, K/V rows with 16-byte pieces
+bool al16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+bool kv_aligned(const clasp_kv_layer* kv, int n) {
+  for (int l = 0; l < n; ++l)
+    if (!al16(kv[l].k) || !al16(kv[l].v)) return false;
+  return true;
+}
+
 bool layers_ready(const clasp_ctx* ctx) {
   for (uint8_t b : ctx->loaded)
     if (!b) return false;
@@ -517,7 +528,7 @@ namespace pk = clasp::pk;
 int engine_setup(clasp_ctx* ctx) {
   const clasp_config& c = ctx->cfg;
   ctx->use_engine = false;
-  if (!ctx->use_tc || getenv("CLASP_NO_ENGINE")) return CLASP_OK;
+  if (!ctx->use_tc || (c.flags & CLASP_FLAG_MULTI_KERNEL)) return CLASP_OK;
   int dev = 0, coop = 0, optin = 0;
   CUDA_TRY(cudaGetDevice(&dev));
   CUDA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
@@ -539,10 +550,6 @@ int engine_setup(clasp_ctx* ctx) {
   for (int k = 0; k < 2; ++k)
     CUDA_TRY(cudaFuncSetAttribute(ctx->e_kernel[k], cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
   int G = ctx->num_sms;
-  if (const char* e = getenv("CLASP_ENGINE_CTAS")) {
-    const int v = atoi(e);
-    if (v >= 1 && v < G) G = v;
-  }
   if (G > ENGINE_MAX_CTAS) G = ENGINE_MAX_CTAS;
   // ---- feature splits and per-CTA tiles.  A CTA's range never straddles two weight matrices:
   // the CTAs of the q/k/v product are dealt to the three matrices in proportion to their rows.
@@ -613,15 +620,11 @@ int engine_setup(clasp_ctx* ctx) {
     ctx->e_wpages[k] = a_pages;   // weight pages of one chunk of the kind's tallest tile
     // ring items of about 32 KB of weights: every item costs the MMA issuers a barrier round trip, so
     // small items waste issue time, while items beyond a sixth of the ring leave too few in flight
-    int kpi_budget = 32, kpi_max = 8;
-    if (const char* e = getenv("CLASP_ENGINE_KPI")) {
-      const int v = atoi(e);
-      if (v >= 4 && v <= 40) { kpi_budget = v; kpi_max = v / 4; }
-    }
+    const int kpi_budget = 32, kpi_max = 8;
     int kpi = kpi_budget / a_pages;
     ctx->e_kpi[k] = kpi < 1 ? 1 : (kpi > kpi_max ? kpi_max : kpi);
     // (the gate/up product interleaves two matrices per chunk, which one box cannot deliver)
-    ctx->e_use3d[k] = (k != pk::G_GU && kind_K[k] % 64 == 0 && ctx->e_kpi[k] > 1 && !getenv("CLASP_ENGINE_NO3D")) ? 1 : 0;
+    ctx->e_use3d[k] = (k != pk::G_GU && kind_K[k] % 64 == 0 && ctx->e_kpi[k] > 1) ? 1 : 0;
   }
   for (int k = 0; k < 5; ++k) {
     ctx->e_tile_idx[k] = (int)tab.size();
@@ -679,11 +682,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   int dev = 0, optin = 0;
   CUDA_TRY(cudaGetDevice(&dev));
   CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-  int ring_pages = (optin - ctx->e_static_smem - 1024 - pk::SCRATCH_BYTES) / pk::PAGE;
-  if (const char* e = getenv("CLASP_ENGINE_PAGES")) {
-    const int v = atoi(e);
-    if (v >= 64 && v < ring_pages && BN <= 32) ring_pages = v;
-  }
+  const int ring_pages = (optin - ctx->e_static_smem - 1024 - pk::SCRATCH_BYTES) / pk::PAGE;
   // an item (gate + up rows and the operand tiles of kpi chunks) must fit the ring twice over
   const int b_pages = BN * pk::BK * 2 / pk::PAGE;
   // chunks per ring item in this launch: the set-up value when two such items fit the ring, else fewer,
@@ -764,6 +763,8 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   P.b.rope = ws.rope;
   P.jobs = ws.jobs; P.n_jobs = (int)ctx->e_jobs.size(); P.wmaps = ws.wmaps; P.tabs = ws.tabs; P.ctl = ws.ctl;
   P.trace = ctx->e_trace; P.trace_cap = ctx->e_trace_cap;
+  P.wait_fast = ctx->wait_limit ? (ctx->wait_limit < pk::WAIT_FAST ? ctx->wait_limit : pk::WAIT_FAST) : pk::WAIT_FAST;
+  P.wait_slow = ctx->wait_limit ? ctx->wait_limit : pk::WAIT_SLOW;
 
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (ctx->profiling) {
@@ -876,11 +877,6 @@ int clasp_create(const clasp_config* cfg, void* workspace, size_t workspace_byte
       return CLASP_ERR_CUDA;
     }
     ctx->cta_cap = 2 * ctx->num_sms;
-    if (const char* e = getenv("CLASP_GEMM_CTA_CAP")) ctx->cta_cap = atoi(e) > 0 ? atoi(e) : ctx->cta_cap;
-    if (const char* e = getenv("CLASP_GEMM_SMEM_KB")) {
-      const int kb = atoi(e);
-      if (kb >= 40 && kb <= 216) ctx->smem_budget = kb * 1024;
-    }
   }
   if (cudaMemsetAsync(ws.status, 0, 256, ctx->stream) != cudaSuccess ||
       cudaMemsetAsync(ws.counters, 0, MAX_COUNTERS * sizeof(int), ctx->stream) != cudaSuccess) {
@@ -959,6 +955,8 @@ int clasp_layer_forward(clasp_ctx* ctx, int32_t layer, const float* x_in, int64_
   if (layer < 0 || layer >= ctx->cfg.L || S < 1 || T < 1 || ctx_len < 0 || pos0 < 0) return CLASP_ERR_INVALID_ARG;
   if (write_kv && S != 1) return CLASP_ERR_INVALID_ARG;
   if (in_stride < ctx->cfg.d_model || out_stride < ctx->cfg.d_model) return CLASP_ERR_INVALID_ARG;
+  if (!al16(x_in) || !al16(x_out) || (in_stride & 3) || (out_stride & 3) || !kv_aligned(kv_layer, 1))
+    return CLASP_ERR_INVALID_ARG;
   if ((int64_t)S * T > ctx->cfg.max_rows || ctx_len > ctx->cfg.max_ctx || pos0 + T > ctx->cfg.max_ctx)
     return CLASP_ERR_CAPACITY;
   if (!ctx->loaded[layer]) return CLASP_ERR_NOT_LOADED;
@@ -988,6 +986,8 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
     return CLASP_ERR_CAPACITY;
   for (int l = 0; l < L; ++l)
     if (!kv[l].k || !kv[l].v) return CLASP_ERR_INVALID_ARG;
+  if (!al16(hidden_states) || (layer_stride & 3) || (token_stride & 3) || !al16(g_final) || !kv_aligned(kv, L))
+    return CLASP_ERR_INVALID_ARG;
   if (M > 0 && !layers_ready(ctx)) return CLASP_ERR_NOT_LOADED;
   Workspace& ws = ctx->ws;
   const int ncell = (L + 1) * (M + 1);
@@ -1029,7 +1029,7 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
     // a layer job followed by another layer job hands over both candidates of every state instead of
     // making the next layer wait for the Eq. 2 decision (needs 2 BN operand rows and accumulator columns)
     const int BNs = M * T <= 16 ? 16 : (M * T + 15) / 16 * 16;
-    if (2 * BNs <= c.max_rows && 2 * BNs <= 128 && !getenv("CLASP_ENGINE_NODEFER"))
+    if (2 * BNs <= c.max_rows && 2 * BNs <= 128 && !(c.flags & CLASP_FLAG_NO_DEFER))
       for (size_t k = 0; k + 1 < ctx->e_jobs.size(); ++k)
         if (ctx->e_jobs[k].type == pk::JOB_LAYER && ctx->e_jobs[k + 1].type == pk::JOB_LAYER) {
           ctx->e_jobs[k].defer = 1;
@@ -1092,6 +1092,7 @@ int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0,
   if (n > c.max_rows || (int64_t)pos0 + n > c.max_ctx || n_head_rows > c.max_head_rows) return CLASP_ERR_CAPACITY;
   for (int l = 0; l < c.L; ++l)
     if (!kv[l].k || !kv[l].v) return CLASP_ERR_INVALID_ARG;
+  if (!al16(hidden_out) || !kv_aligned(kv, c.L)) return CLASP_ERR_INVALID_ARG;
   if (!layers_ready(ctx) || !ctx->embed) return CLASP_ERR_NOT_LOADED;
   const int d = c.d_model, L = c.L;
   int rc;
@@ -1160,6 +1161,8 @@ int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int
   const clasp_config& c = ctx->cfg;
   if ((int64_t)pos + 1 > c.max_ctx) return CLASP_ERR_CAPACITY;
   if (!layers_ready(ctx) || !ctx->embed) return CLASP_ERR_NOT_LOADED;
+  for (int l = 0; l < c.L; ++l)
+    if (!skip_mask_host[l] && (!kv[l].k || !kv[l].v || !kv_aligned(kv + l, 1))) return CLASP_ERR_INVALID_ARG;
   const int d = c.d_model;
   int rc;
   if ((rc = rope_table(ctx, 1, pos))) return rc;
@@ -1319,6 +1322,7 @@ int clasp_gemm_xwT_noalloc(const void* x, const void* w, int32_t R, int32_t N, i
   p.counters = (int*)(nd->scratch + NOALLOC_PARTIAL_BYTES);
   int* scratch_status = (int*)(nd->scratch + NOALLOC_PARTIAL_BYTES + NOALLOC_COUNTERS * sizeof(int));
   p.status = status_out ? status_out : scratch_status;
+  p.spin_fast = SPIN_FAST; p.spin_slow = SPIN_SLOW;
   const int stage_bytes = A_TILE_BYTES + p.BN * BK * 2;
   int stages = 110 * 1024 / stage_bytes;
   if (stages > 8) stages = 8;
@@ -1389,10 +1393,22 @@ int clasp_profile_gemm(clasp_ctx* ctx, int32_t enable, int64_t* n_launches, doub
 int64_t clasp_launch_count(const clasp_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 int clasp_engine_trace(clasp_ctx* ctx, uint64_t* stamps, int32_t cap_per_cta, int32_t* n_ctas) {
-  if (!ctx || cap_per_cta < 0) return CLASP_ERR_INVALID_ARG;
+  if (!ctx) return CLASP_ERR_INVALID_ARG;
   if (n_ctas) *n_ctas = ctx->use_engine ? ctx->e_G : 0;
+  if (cap_per_cta < 0) return CLASP_OK;   // query only: the trace buffer in use stays
   ctx->e_trace = (unsigned long long*)stamps;
   ctx->e_trace_cap = stamps ? cap_per_cta : 0;
+  return CLASP_OK;
+}
+
+int clasp_engine_active(const clasp_ctx* ctx) {
+  if (!ctx) return CLASP_ERR_INVALID_ARG;
+  return ctx->use_engine ? 1 : 0;
+}
+
+int clasp_set_wait_limit(clasp_ctx* ctx, uint32_t polls) {
+  if (!ctx) return CLASP_ERR_INVALID_ARG;
+  ctx->wait_limit = polls;
   return CLASP_OK;
 }
 

@@ -60,10 +60,7 @@ constexpr int MAX_ROWS = 128;         // rows one launch may push through a laye
 // blocks.  4 or 8: with 4 the unrolled per-row code is half as long and 5 to 8 rows already keep both groups
 // busy (measured against 8: 8B search -0.5 %, forward passes -1.7 %, 8192-key contexts -3 %; launches with
 // many rows make more passes: 70B search with 32 rows +0.6 %, 128-row prefill +3 %).
-#ifndef CLASP_RB
-#define CLASP_RB 4
-#endif
-constexpr int RB = CLASP_RB;
+constexpr int RB = 4;
 constexpr int N_HEIGHTS = 4;          // distinct tile heights (TMA box heights) per weight matrix
 constexpr int MAX_CTAS = 192;
 
@@ -81,8 +78,10 @@ enum { T_START = 0, T_QKV, T_ATT_READY, T_ATT_Q, T_ATT_TILES, T_ATT_PUB, T_MERGE
        T_MMA_FIRST = 16, T_MMA_LAST = 20, T_ACC = 24,
        // the Eq. 2 step has published the next layer's operand; the operand producer has seen the operands
        // of the q/k/v, o and gate/up products complete
-       T_SEL_PUB = 28, T_B_READY = 29 };
-constexpr int TRACE_SLOTS = 32;  // time stamps per job
+       T_SEL_PUB = 28, T_B_READY = 29,
+       // finer stamps inside a step while looking for a delay (workers): T_FINE + n, n < 32
+       T_FINE = 32 };
+constexpr int TRACE_SLOTS = 64;  // time stamps per job
 
 struct TileDesc {      // one accumulator's worth of a CTA's feature range: rows y0.. of one weight matrix
   int f0;              // first feature in the product's feature space
@@ -188,6 +187,8 @@ struct Params {
   Ctl* ctl;
   unsigned long long* trace;  // optional [G, trace_cap] time stamps (ns)
   int trace_cap;
+  uint32_t wait_fast;         // polls of a wait before it starts to sleep between polls
+  uint32_t wait_slow;         // further polls (about 100 ns apart) before the wait gives up
 };
 
 // ------------------------------------------------------------------ small PTX helpers
@@ -323,6 +324,7 @@ struct Shared {
   uint64_t acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   volatile int abort;
+  uint32_t wait_fast, wait_slow;   // the launch's wait limits
   volatile int a_issued;    // ring items whose weight loads have been issued (warp 0 -> warp 1)
   int flag;                 // broadcast of a one-thread decision to the workers
   float rs[MAX_ROWS];       // per-row norm factors of the current product
@@ -342,7 +344,8 @@ struct RedTables {
 static_assert(sizeof(RedTables) <= SCRATCH_BYTES, "reduction tables must fit the scratch area");
 
 constexpr uint32_t WAIT_FAST = 1u << 12;
-constexpr uint32_t WAIT_SLOW = 1u << 22;  // x ~100 ns: gives up after roughly half a second
+constexpr uint32_t WAIT_SLOW = 1u << 22;  // x ~100 ns: gives up after roughly half a second (the defaults of
+                                          // Params::wait_fast / wait_slow)
 
 __device__ __forceinline__ void raise_abort(Ctl* ctl, Shared* sh, bool timed_out) {
   if (timed_out && !ld_volatile_i32(&ctl->abort)) atomicExch(&ctl->status, 1);
@@ -358,9 +361,10 @@ __device__ __forceinline__ bool aborted(Ctl* ctl, Shared* sh) {
 // Bounded mbarrier wait that also ends when any CTA raised the abort flag.
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctl* ctl, Shared* sh) {
   const uint32_t b = tc::smem_u32(bar);
-  for (uint32_t it = 0; it < WAIT_FAST; ++it)
+  const uint32_t n_fast = sh->wait_fast, n_slow = sh->wait_slow;
+  for (uint32_t it = 0; it < n_fast; ++it)
     if (tc::mbar_test(b, parity)) return true;
-  for (uint32_t it = 0; it < WAIT_SLOW; ++it) {
+  for (uint32_t it = 0; it < n_slow; ++it) {
     if (tc::mbar_test(b, parity)) return true;
     if (aborted(ctl, sh)) return false;
     __nanosleep(100);
@@ -371,7 +375,8 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Ctl* ct
 
 // Bounded wait until flag >= epoch.
 __device__ __forceinline__ bool wait_flag(const int* flag, int epoch, Ctl* ctl, Shared* sh) {
-  for (uint32_t it = 0; it < (1u << 23); ++it) {
+  const uint32_t n = 2u * sh->wait_slow;
+  for (uint32_t it = 0; it < n; ++it) {
     if (ld_acquire_i32(flag) >= epoch) return true;
     if ((it & 15u) == 15u) {
       if (aborted(ctl, sh)) return false;
@@ -605,9 +610,10 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
           const int at = rp.place(pages, c.ring_pages, fp);
           // the weight producer has made room for this item
           bool ok = false;
-          for (uint32_t w = 0; w < WAIT_SLOW; ++w) {
+          const uint32_t n_fast = sh->wait_fast, n_slow = sh->wait_slow;
+          for (uint32_t w = 0; w < n_slow; ++w) {
             if ((uint32_t)sh->a_issued > it) { ok = true; break; }
-            if (w > WAIT_FAST) {
+            if (w > n_fast) {
               if (aborted(p.ctl, sh)) break;
               __nanosleep(100);
             }
@@ -1738,10 +1744,7 @@ struct Worker {
 };
 
 // ------------------------------------------------------------------ the kernel
-#ifndef CLASP_REGS_SPECIAL
-#define CLASP_REGS_SPECIAL 72
-#endif
-constexpr int REGS_SPECIAL = CLASP_REGS_SPECIAL;
+constexpr int REGS_SPECIAL = 72;
 constexpr int REGS_WORKER = (THREADS * 168 - 128 * REGS_SPECIAL) / 256 / 8 * 8;
 static_assert(THREADS == 384 && WORKER_T0 == 128, "register split assumes one special and two worker warp groups");
 static_assert(128 * REGS_SPECIAL + 256 * REGS_WORKER <= THREADS * 168, "register pool of the CTA");
@@ -1772,6 +1775,8 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
       tc::mbar_init(tc::smem_u32(&sh.acc_empty[b]), 1);
     }
     sh.abort = 0;
+    sh.wait_fast = p.wait_fast;
+    sh.wait_slow = p.wait_slow;
     sh.a_issued = 0;
     sh.flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

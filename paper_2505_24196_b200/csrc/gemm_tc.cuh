@@ -58,6 +58,7 @@ struct Params {
   float* partial;  // [splits][dual+1][R][n_total]
   int* counters;   // one per tile, zero on entry, zero again on exit
   int* status;     // set to 1 when a bounded wait gives up
+  uint32_t spin_fast, spin_slow;  // polls without / with a ~128 ns sleep before a wait gives up
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -81,10 +82,11 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false (and *status = 1) if the phase never completes.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
-  for (uint32_t it = 0; it < SPIN_FAST; ++it)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, uint32_t n_fast = SPIN_FAST,
+                                          uint32_t n_slow = SPIN_SLOW) {
+  for (uint32_t it = 0; it < n_fast; ++it)
     if (mbar_test(bar, parity)) return true;
-  for (uint32_t it = 0; it < SPIN_SLOW; ++it) {
+  for (uint32_t it = 0; it < n_slow; ++it) {
     if (mbar_test(bar, parity)) return true;
     __nanosleep(128);
   }
@@ -191,7 +193,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
       for (int it = 0; it < n_iter; ++it) {
         const int s = it % p.stages;
         const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
-        if (!mbar_wait(smem_u32(&bar_empty[s]), phase ^ 1u, p.status)) { s_abort = 1; break; }
+        if (!mbar_wait(smem_u32(&bar_empty[s]), phase ^ 1u, p.status, p.spin_fast, p.spin_slow)) { s_abort = 1; break; }
         const uint32_t full = smem_u32(&bar_full[s]);
         const uint32_t sa = smem_base + s * stage_bytes;
         const int kx = (kc_begin + it) * BK;
@@ -213,7 +215,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
       for (int it = 0; it < n_iter && ok; ++it) {
         const int s = it % p.stages;
         const uint32_t phase = (uint32_t)(it / p.stages) & 1u;
-        if (!mbar_wait(smem_u32(&bar_full[s]), phase, p.status)) { s_abort = 1; ok = false; break; }
+        if (!mbar_wait(smem_u32(&bar_full[s]), phase, p.status, p.spin_fast, p.spin_slow)) { s_abort = 1; ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t sa = smem_base + s * stage_bytes;
         const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + a_bytes);
@@ -238,7 +240,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     const int col = p.col_off[mat] + n_local;
     const bool have_acc = n_iter > 0;
     bool ok = true;
-    if (have_acc) ok = mbar_wait(smem_u32(&bar_accum), 0, p.status);
+    if (have_acc) ok = mbar_wait(smem_u32(&bar_accum), 0, p.status, p.spin_fast, p.spin_slow);
     ok = __all_sync(0xffffffffu, ok);  // tcgen05.ld below needs the whole warp
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);

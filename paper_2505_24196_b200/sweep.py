@@ -29,7 +29,7 @@ import datagen  # noqa: E402
 import paper_2505_24196_b200 as clasp  # noqa: E402
 from paper_2505_24196_b200.decode import greedy_autoregressive  # noqa: E402
 
-TRACE_SLOTS = 32
+TRACE_SLOTS = 64
 SLOT = {"start": 0, "qkv": 1, "att_ready": 2, "att_pub": 5, "merge": 6, "o": 7, "gu": 8, "down": 9, "dp_done": 13,
         "mma_first_qkv": 16, "mma_first_o": 17, "mma_first_gu": 18, "mma_first_down": 19,
         "mma_last_qkv": 20, "mma_last_o": 21, "mma_last_gu": 22, "mma_last_down": 23}
@@ -129,7 +129,8 @@ STAMP_NAMES = (["job_start", "qkv_epilogue_done", "attention_ready", "attention_
                 "down_epilogue_done", "eq2_sums_published", "eq2_sums_complete", "eq2_decided", "eq2_step_done",
                 "head_done", "-"]
                + [f"{a}_{b}" for a in ("mma_first", "mma_last", "accumulator_ready") for b in ("qkv", "o", "gate_up", "down")]
-               + ["eq2_next_operand_point", "operand_ready_qkv", "operand_ready_o", "operand_ready_gate_up"])
+               + ["eq2_next_operand_point", "operand_ready_qkv", "operand_ready_o", "operand_ready_gate_up"]
+               + [f"fine_{n:02d}" for n in range(32)])
 
 
 def cmd_trace(args):

@@ -367,3 +367,97 @@ def test_full_mask_draft_accepts_everything():
     sd, rounds = orc.greedy_self_speculative(model, prompt, 12, 64, M=0, K=3, fixed_mask=[0] * 8)
     assert all(r["accepted"] == 3 for r in rounds)
     assert sd == orc.greedy_autoregressive(model, prompt, 12, 64)
+
+
+def test_argmax_takes_the_lowest_index_on_an_exact_tie():
+    """Greedy accept rule: ties between logits go to the lowest token id."""
+    lg = np.array([[0.0, 3.0, 3.0, 1.0], [2.0, 2.0, 2.0, 2.0], [-1.0, -5.0, -1.0, -1.0]])
+    np.testing.assert_array_equal(orc.argmax_lowest(lg), [1, 0, 0])
+
+
+def test_top1_probability_closed_forms():
+    # uniform logits: 1 / vocab; one logit ahead by ln(3) among 4: 3 / (3 + 3) = 1/2
+    np.testing.assert_allclose(orc.top1_probability(np.zeros((1, 8))), [0.125], rtol=1e-15)
+    np.testing.assert_allclose(orc.top1_probability(np.array([[math.log(3.0), 0.0, 0.0, 0.0]])), [0.5], rtol=1e-15)
+    # invariant under a shift of all logits, also a large one
+    np.testing.assert_allclose(orc.top1_probability(np.array([[1000.0 + math.log(3.0), 1000.0, 1000.0, 1000.0]])),
+                               [0.5], rtol=1e-12)
+
+
+# ---------------- lower optimisation frequency (Sec. 3.7) ----------------
+
+@pytest.mark.parametrize("N", [2, 3])
+def test_optimisation_interval_keeps_the_skip_set_between_searches(N):
+    """With interval N the skip set changes only after every N-th verification; the output
+    stays lossless, and the searches that do run see the same inputs as in the interval-1
+    loop as long as the committed tokens agree (they do: both are lossless)."""
+    model = from_torch.model_from_datagen(TINY)
+    prompt = datagen.token_ids(TINY, 24).numpy()
+    n_new = 18
+    ar = orc.greedy_autoregressive(model, prompt, n_new, 96)
+    sd, rounds = orc.greedy_self_speculative(model, prompt, n_new, 96, M=2, K=3, dp_interval=N)
+    assert sd == ar
+    assert len(rounds) >= 2 * N
+    for k in range(len(rounds)):
+        first_of_block = (k // N) * N
+        np.testing.assert_array_equal(rounds[k]["S"], rounds[first_of_block]["S"])
+    assert all(int(r["S"].sum()) == 2 for r in rounds)
+
+
+def test_an_interval_beyond_the_run_is_the_fixed_first_skip_set():
+    """Limit of Sec. 3.7: if the search never runs again, every round drafts with the set found
+    after the prefill -- the loop with that set given as a fixed mask, round for round."""
+    model = from_torch.model_from_datagen(TINY)
+    prompt = datagen.token_ids(TINY, 24).numpy()
+    n_new = 14
+    sd, rounds = orc.greedy_self_speculative(model, prompt, n_new, 96, M=2, K=3, dp_interval=10 ** 6)
+    S0 = rounds[0]["S"]
+    sd_f, rounds_f = orc.greedy_self_speculative(model, prompt, n_new, 96, M=2, K=3, fixed_mask=S0)
+    assert sd == sd_f
+    assert [r["accepted"] for r in rounds] == [r["accepted"] for r in rounds_f]
+    assert all(np.array_equal(r["S"], S0) for r in rounds)
+    # and the first set is the search on the last prompt token (reading 12)
+    cache = orc.KVCache(TINY, 96)
+    _, hid, _ = orc.verify_forward(model, prompt, cache, 0)
+    ref = orc.dp_search(model, hid[len(prompt) - 1][:, None, :], cache, len(prompt) - 1, len(prompt) - 1, 2)
+    np.testing.assert_array_equal(S0, ref["S"])
+
+
+# ---------------- draft-exiting threshold (Sec. 5.3.3) ----------------
+
+def test_exit_threshold_limits():
+    """Threshold 0 never stops a round early (the fixed-length loop, round for round); a threshold
+    above 1 stops every round after its first draft (the K = 1 loop, round for round)."""
+    model = from_torch.model_from_datagen(TINY)
+    prompt = datagen.token_ids(TINY, 24).numpy()
+    n_new = 14
+    base, r_base = orc.greedy_self_speculative(model, prompt, n_new, 96, M=2, K=3)
+    zero, r_zero = orc.greedy_self_speculative(model, prompt, n_new, 96, M=2, K=3, exit_threshold=0.0)
+    assert zero == base and [r["drafted"] for r in r_zero] == [3] * len(r_base)
+    one, r_one = orc.greedy_self_speculative(model, prompt, n_new, 96, M=2, K=3, exit_threshold=1.5)
+    k1, r_k1 = orc.greedy_self_speculative(model, prompt, n_new, 96, M=2, K=1)
+    assert one == k1
+    assert [r["drafted"] for r in r_one] == [1] * len(r_k1)
+    assert [r["accepted"] for r in r_one] == [r["accepted"] for r in r_k1]
+
+
+def test_exit_threshold_stops_at_the_first_low_confidence_draft_and_stays_lossless():
+    model = from_torch.model_from_datagen(TINY)
+    prompt = datagen.token_ids(TINY, 24).numpy()
+    n_new = 16
+    ar = orc.greedy_autoregressive(model, prompt, n_new, 96)
+    _, r0 = orc.greedy_self_speculative(model, prompt, n_new, 96, M=2, K=4)
+    # (a random-init model is least sure of a round's first draft: put the threshold among those, so
+    # that some rounds stop after one draft and the others run to the cap)
+    first = sorted(r["confidence"][0] for r in r0)
+    thr = first[len(first) // 2]
+    sd, rounds = orc.greedy_self_speculative(model, prompt, n_new, 96, M=2, K=4, exit_threshold=thr)
+    assert sd == ar
+    assert any(r["drafted"] < 4 for r in rounds) and any(r["drafted"] > 1 for r in rounds)
+    for r in rounds:
+        c = r["confidence"]
+        assert len(c) == r["drafted"] and 0 <= r["accepted"] <= r["drafted"]
+        assert all(x >= thr for x in c[:-1])        # every draft before the last was confident
+        assert c[-1] < thr or r["drafted"] == 4     # the last one was not, or the cap ended the round
+        # the confidence is the softmax probability of the greedy token: between 1/vocab and 1
+        assert all(1.0 / TINY.vocab <= x <= 1.0 for x in c)

@@ -15,15 +15,19 @@ from .binding import Clasp, KVCache
 class SelfSpeculativeDecoder:
     """Greedy self-speculative decoding with the skip set re-optimised after verification.
 
-    M: layers the draft model skips; K: draft length; dp_interval: run the layer
+    M: layers the draft model skips; K: most drafts per round; dp_interval: run the layer
     search every that many verifications (1 = after each, the paper's default
-    before its lower-frequency optimisation of Sec. 3.7).
+    before its lower-frequency optimisation of Sec. 3.7); exit_threshold: a drafted token
+    whose softmax probability (returned by the draft call) is below it ends the round's
+    drafting (Sec. 5.3.3; 0 = always draft K tokens).  The comparison is the only step taken
+    here, on one float per draft read back from the device.
     """
 
     def __init__(self, engine: Clasp, kv: KVCache, M: int, K: int, dp_interval: int = 1, T: int = 1,
-                 time_stages: bool = False):
+                 time_stages: bool = False, exit_threshold: float = 0.0):
         self.e, self.kv, self.M, self.K, self.T = engine, kv, M, K, T
         self.dp_interval = dp_interval
+        self.exit_threshold = float(exit_threshold)
         self.time_stages = time_stages
         dev = engine.device
         L, d = engine.cfg.L, engine.cfg.d_model
@@ -32,6 +36,8 @@ class SelfSpeculativeDecoder:
         self.hidden = torch.empty((K + 1, L + 1, d), dtype=torch.float32, device=dev)
         self.pinned_in = torch.zeros(K + 1, dtype=torch.int32).pin_memory()
         self.pinned_out = torch.zeros(2 * (K + 1), dtype=torch.int32).pin_memory()
+        self.conf = torch.zeros(K, dtype=torch.float32, device=dev)          # confidence of d_1..d_K
+        self.pinned_conf = torch.zeros(K, dtype=torch.float32).pin_memory()
         self.mask_host = bytes(L)
         self.stage_ms = {"dp": 0.0, "draft": 0.0, "verify": 0.0}
         self.rounds: List[Dict] = []
@@ -83,22 +89,32 @@ class SelfSpeculativeDecoder:
         self.pinned_in[0] = self.pending
         self.draft_tok[:1].copy_(self.pinned_in[:1], non_blocking=True)
 
+        thr = self.exit_threshold
+        conf: List[float] = []
+
         def draft():
             for k in range(K):
                 e.draft_forward(self.mask_host, self.draft_tok[k:k + 1], self.n_valid + k, self.kv,
-                                self.draft_tok[k + 1:k + 2])
-        self._timed("draft", draft)
-        self._timed("verify", lambda: e.verify(self.draft_tok, self.n_valid, self.kv, K + 1,
+                                self.draft_tok[k + 1:k + 2], self.conf[k:k + 1] if thr > 0.0 else None)
+                if thr > 0.0:
+                    self.pinned_conf[k:k + 1].copy_(self.conf[k:k + 1], non_blocking=True)
+                    e.stream.synchronize()
+                    conf.append(float(self.pinned_conf[k]))
+                    if conf[-1] < thr:
+                        return k + 1
+            return K
+        n_d = self._timed("draft", draft)
+        self._timed("verify", lambda: e.verify(self.draft_tok[:n_d + 1], self.n_valid, self.kv, n_d + 1,
                                                hidden_out=self.hidden, argmax_out=self.argmax))
         self.pinned_out[:K + 1].copy_(self.draft_tok, non_blocking=True)
         self.pinned_out[K + 1:].copy_(self.argmax, non_blocking=True)
         e.stream.synchronize()
         host = self.pinned_out.tolist()
-        a, committed = e.accept(host[1:K + 1], host[K + 1:])
+        a, committed = e.accept(host[1:n_d + 1], host[K + 1:K + 2 + n_d])
         obj_pos = self.n_valid + a
         self.n_valid += a + 1
         self.pending = committed[-1]
-        self.rounds.append({"accepted": a, "S": self.mask_host})
+        self.rounds.append({"accepted": a, "S": self.mask_host, "drafted": n_d, "confidence": conf})
         if len(self.rounds) % self.dp_interval == 0:
             self._timed("dp", lambda: self._search(self.hidden[a], obj_pos))
         return committed

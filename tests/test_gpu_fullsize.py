@@ -24,6 +24,7 @@ pytestmark = pytest.mark.gpu
 C0 = 512          # visible cache positions
 M = 12
 SAMPLED_LAYER = 1  # the layer whose weights the oracle also holds
+MID_LAYER = 19     # a second one, in the middle of the table, for the 12-row step i = 20
 
 
 class Full8B:
@@ -51,6 +52,11 @@ class Full8B:
         self.kv.v[SAMPLED_LAYER].copy_(cv)
         self.ck64, self.cv64 = ck.double().numpy(), cv.double().numpy()
         self.w64 = {k: from_torch.to_f64(v) for k, v in self.layers[SAMPLED_LAYER].items()}
+        ck2 = datagen.normal_rows(51, 2, shp).to(cfg.torch_dtype)
+        cv2 = datagen.normal_rows(51, 3, shp).to(cfg.torch_dtype)
+        self.kv.k[MID_LAYER].copy_(ck2)
+        self.kv.v[MID_LAYER].copy_(cv2)
+        self.ck64_mid, self.cv64_mid = ck2.double().numpy(), cv2.double().numpy()
         # objective states x_0..x_L: a seeded random walk (consecutive states are close, as in a
         # residual stream)
         steps = datagen.normal_rows(52, 0, (cfg.L + 1, cfg.d_model))
@@ -125,6 +131,37 @@ def test_search_properties_and_sampled_cells(full):
     assert torch.equal(res2["S"], res["S"])
     assert torch.equal(res2["D"].nan_to_num(7.0), res["D"].nan_to_num(7.0))
     assert torch.equal(res2["g_final"], res["g_final"])
+
+
+def test_mid_table_step_with_twelve_rows_against_oracle(full):
+    """Step i = 20 of the full-size search pushes twelve candidate states through layer 19 in one batch.
+    With SKIP forced at every cell, state j of that step is g[19][j] = x_{19-j} and its skip candidate
+    g[19][j-1] = x_{20-j}, both known without running the layers below; the margins the device
+    reports for row 20 (computed whatever is forced) are then
+        cos(x_20, f_19(x_{19-j})) - cos(x_20, x_{20-j}),   j = 1..12,
+    one oracle layer application each: every row of a twelve-row step, in the launch configuration
+    the benchmark times, against the oracle."""
+    cfg, eng = full.cfg, full.engine
+    L, d = cfg.L, cfg.d_model
+    xs = full.x.double().numpy()
+    forced = np.full((L + 1, M + 1), 255, dtype=np.uint8)
+    forced[:, 1:] = orc.SKIP
+    res = eng.dp_search(full.x.cuda(), d, 0, full.kv, C0, C0, 1, M, forced_choice=torch.from_numpy(forced).cuda())
+    torch.cuda.synchronize()
+    assert eng.device_status() == 0
+    margin = res["margin"].cpu().numpy()
+    D = res["D"].cpu().numpy()
+    w64 = {k: from_torch.to_f64(v) for k, v in full.layers[MID_LAYER].items()}
+    i = MID_LAYER + 1
+    for j in range(1, M + 1):
+        G, _, _ = orc.decoder_layer(xs[i - 1 - j:i - j], w64, full.ck64_mid, full.cv64_mid, C0, C0, cfg)
+        s_app, s_skip = _cos(xs[i], G), _cos(xs[i], xs[i - j])
+        assert abs(margin[i, j] - (s_app - s_skip)) < 2e-3, j
+        assert abs(D[i, j] - s_skip) < 1e-3, j            # the forced branch's score
+    # every skip forced: the last M layers are the skip set and g[L][M] = x_{L-M}
+    S = res["S"].cpu().numpy()
+    assert S[:L - M].sum() == 0 and S[L - M:].sum() == M
+    assert np.array_equal(res["g_final"].cpu().numpy()[0], full.x[L - M].numpy())
 
 
 def test_round_is_lossless_at_full_size(full):

@@ -38,6 +38,32 @@ def test_noalloc_gemm_matches_context_gemm_twice_in_a_row():
     eng.close()
 
 
+@pytest.mark.parametrize("R,N,K", [(200, 256, 512), (256, 130, 72), (33, 128, 64), (16, 384, 4096)])
+def test_noalloc_gemm_wide_ragged_and_unsplit_shapes(R, N, K):
+    """The entry point's whole range: up to 256 rows (256 accumulator columns, 48 KB stages), a row
+    count that is not a multiple of 16, a ragged N and K, a single-split product that uses no scratch;
+    with and without a status word (without one a wait that gave up would go unreported, the product
+    itself is the same)."""
+    import paper_2505_24196_b200 as clasp
+    cfg = datagen.CONFIGS["small"]
+    eng = clasp.Clasp(clasp.make_config(cfg, max_ctx=64, max_rows=64, max_M=1))
+    x = datagen.normal_rows(73, R + N, (R, K)).to(torch.bfloat16).cuda()
+    w = datagen.normal_rows(74, N + K, (N, K), 0.05).to(torch.bfloat16).cuda()
+    ref = eng.gemm_xwT(x, w)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y1 = torch.full((R, N), float("nan"), dtype=torch.float32, device="cuda")
+    y2 = torch.full((R, N), float("nan"), dtype=torch.float32, device="cuda")
+    clasp.gemm_xwT_noalloc(x, w, y1, status_out=status)
+    clasp.gemm_xwT_noalloc(x, w, y2)                       # status_out == NULL
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    assert torch.equal(y1, ref) and torch.equal(y2, ref)
+    exact = x.double() @ w.double().T
+    assert float(torch.linalg.norm(y1.double() - exact) / torch.linalg.norm(exact)) < 2e-6
+    assert eng.device_status() == 0
+    eng.close()
+
+
 def test_noalloc_gemm_refuses_what_does_not_fit():
     import paper_2505_24196_b200 as clasp
     x = torch.zeros((257, 64), dtype=torch.bfloat16, device="cuda")

@@ -9,16 +9,21 @@ the search's latency per verification, measured with CUDA events inside the time
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-N > 1 (under torchrun) runs N independent replicas, one per GPU: the path is a single
-sequence and does not shard, so there is no collective on the data path.
+N > 1 runs N independent replicas, one per GPU: the path is a single sequence and does not
+shard, so there is no collective on the data path.  Under torchrun the ranks are the
+replicas; a plain `python bench.py --gpus N` starts the N ranks itself (one torchrun-style
+launch on 127.0.0.1).
 --impl reference times the CPU oracle (a deliberately plain program) on a bounded
 sample of the same workload.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import re
+import socket
 import subprocess
 import sys
 import threading
@@ -98,6 +103,44 @@ class ClockSampler:
         sm.sort()
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def workload_config(name: str, world: int) -> dict:
+    """The `config` object of the JSON line: the same for the CUDA arm and the oracle arm."""
+    wl = WORKLOADS[name]
+    cfg = datagen.CONFIGS[wl["model"]]
+    return {"workload": name, "model_shape": cfg.name, "L": cfg.L, "M": wl["M"], "T": wl["T"],
+            "draft_len": wl["K"], "ctx_len": wl["ctx"], "replicas": world,
+            "l2": "inputs larger than L2 (every layer's matrices are streamed once per search)"}
+
+
+KERNEL_SOURCES = ["engine2.cuh", "gemm_tc.cuh", "kernels.cuh", "clasp_api.cu"]
+
+
+def kernel_sources_digest() -> str:
+    """Digest of the CUDA sources: ties a stored profiler figure to the kernel it was taken from."""
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2505_24196_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload: str):
+    """DRAM bytes (read + write) of one launch of the dominant kernel from the committed ncu summary of
+    this workload -- or None when the CUDA sources have changed since that capture (the summary names
+    the digest of the sources it was taken from)."""
+    path = os.path.join(ROOT, "profiles", "engine_kernel_8b_l6_c512_M3_ncu.md")
+    if workload != "8b-c512-M12" or not os.path.exists(path):
+        return None, "no capture for this workload"
+    text = open(path).read()
+    m = re.search(r"traffic_bytes_per_search_launch:\s*(\d+)", text)
+    g = re.search(r"kernel_sources_digest:\s*([0-9a-f]+)", text)
+    if not m or not g:
+        return None, "summary holds no machine-readable figure"
+    if g.group(1) != kernel_sources_digest():
+        return None, "kernel sources changed since the capture in profiles/engine_kernel_8b_l6_c512_M3_ncu.md"
+    return int(m.group(1)), "profiles/engine_kernel_8b_l6_c512_M3_ncu.md (6-layer capture x 31 / 5 applied layers)"
 
 
 def dp_algorithmic_bytes(cfg, ctx_len: int) -> int:
@@ -200,8 +243,8 @@ def run_ours(args, rank, world):
     roof = None
     if hasattr(eng.lib, "clasp_profile_gemm"):
         roof = gemm_roofline(eng, dec, kv, hid_dev, obj, T, M, d)
-        roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.workload)
-        roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum, scaled from a 6-layer capture)"
+        roof["traffic"], roof["traffic_source"] = ncu_traffic(args.workload)
+        roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)"
     peak, which = measured_peaks()
     alg_bytes = dp_algorithmic_bytes(cfg, obj)
     dp_gbs = alg_bytes / (dp_ms * 1e-3) / 1e9
@@ -218,9 +261,8 @@ def run_ours(args, rank, world):
         "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": round(total_ms / steps, 4),
         "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
         "data": "synthetic (seeded random-init weights, uniform random token ids)",
-        "config": {"workload": args.workload, "model_shape": cfg.name, "L": cfg.L, "M": M, "T": T,
-                   "draft_len": K, "ctx_len": obj, "replicas": world,
-                   "l2": "inputs larger than L2 (13.5 GB of weights streamed per search)"},
+        "config": workload_config(args.workload, world),
+        "run": {"ctx_len_after_timed_rounds": ctx_now, "kernel_sources_digest": kernel_sources_digest()},
         "stage_ms": {k: round(v, 4) for k, v in stage.items()},
         "decode_tokens_per_s": round(tok_s, 2),
         "mean_accepted": round(sum(accepted) / max(len(accepted), 1), 3),
@@ -277,12 +319,6 @@ def dp_only(args, eng, dec, kv, cfg, wl):
     print(json.dumps({"mode": "dp-only", "workload": args.workload, "dp_ms": round(ms, 4),
                       "gbs": round(byts / ms / 1e6, 1), "launches_per_search": (eng.launch_count() - n0) // args.steps,
                       "device_status": eng.device_status()}), flush=True)
-
-
-# DRAM bytes (read + write) of one search launch of the persistent kernel, from the ncu capture summarised in
-# profiles/engine_kernel_8b_l6_c512_M3_ncu.md: taken on a 6-layer model of the same layer shape and scaled by
-# 31 / 5 applied layers.  Set to None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES = {"8b-c512-M12": 13730230000}   # (dram read + write of the 6-layer capture) x 31 / 5
 
 
 def gemm_roofline(eng, dec, kv, hid_dev, obj, T, M, d):
@@ -351,7 +387,7 @@ def layer_row_applications(L, M, n_steps=None):
 
 
 def cpu_baseline(cfg, wl, layers=None, head=None):
-    n_steps = min(5, cfg.L)
+    n_steps = min(8, cfg.L)
     times, t_prefill, _ = oracle_sample(cfg, wl, layers, head, n_steps)
     t_dp = times[0]
     full, part = layer_row_applications(cfg.L, wl["M"]), layer_row_applications(cfg.L, wl["M"], n_steps)
@@ -370,25 +406,49 @@ def run_reference(args, rank, world):
     cfg = datagen.CONFIGS[wl["model"]]
     n_steps = min(4, cfg.L)
     steps, warmup = args.steps, args.warmup
-    n_warm = min(warmup, 1)
-    times, _, _ = oracle_sample(cfg, wl, n_steps=n_steps, repeats=n_warm + min(steps, 3))
-    times = times[n_warm:]
+    times, _, _ = oracle_sample(cfg, wl, n_steps=n_steps, repeats=warmup + steps)
+    times = times[warmup:]
     full, part = layer_row_applications(cfg.L, wl["M"]), layer_row_applications(cfg.L, wl["M"], n_steps)
     scale = full / part
     val = sum(times) / len(times) * 1e3 * scale
-    sample = (f"oracle DP steps i=1..{n_steps} of {cfg.L} per step ({part} of the search's {full} layer passes "
-              f"over one state), scaled by {full}/{part}; {len(times)} timed steps (capped at 3 to bound the run)")
+    sample = (f"per step: oracle DP steps i=1..{n_steps} of {cfg.L} ({part} of the search's {full} layer passes "
+              f"over one state), scaled by {full}/{part}")
     out = {"impl": "reference", "metric": "dp_search_ms_per_verify", "value": round(val, 1), "unit": "ms",
-           "n_gpus": world, "steps": len(times), "warmup": min(warmup, 1), "ms_per_step": round(val, 1),
+           "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": round(val, 1),
            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
            "data": "synthetic (seeded random-init weights, uniform random token ids)",
-           "config": {"workload": args.workload, "model_shape": cfg.name, "M": wl["M"], "T": wl["T"],
-                      "ctx_len": wl["ctx"] - 1},
+           "config": workload_config(args.workload, world),
            "cpu_baseline": {"value": round(val, 1), "unit": "ms", "cores": torch.get_num_threads(),
                             "kind": "oracle", "sample": sample},
            "e2e": {"value": round(val, 1), "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out), flush=True)
+
+
+# --------------------------------------------------------------------------- replicas
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_replicas(n: int, argv) -> int:
+    """`python bench.py --gpus N` outside torchrun: start the N ranks (one replica per GPU) the way
+    torchrun would, on 127.0.0.1, and pass their output through (rank 0 prints the JSON line)."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def combine_check(rank, world):
+    """Replica plumbing without a GPU: every rank contributes made-up measurements, rank 0 prints what
+    the benchmark would report for them (slowest time, summed throughput, n_gpus = ranks)."""
+    total_ms, dp_ms, e2e_ms, tok_s = combine_replicas(10.0 + rank, 4.0 + 0.5 * rank, 5.0 - rank, 100.0 * (rank + 1),
+                                                      world, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"mode": "combine-check", "n_gpus": world, "ms_per_step": total_ms, "value": dp_ms,
+                          "e2e": e2e_ms, "decode_tokens_per_s": tok_s}), flush=True)
 
 
 def main():
@@ -399,13 +459,25 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b-c512-M12", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--mode", default="round", choices=["round", "dp-only"],
-                    help="dp-only: profiling aid, runs just the layer search inside a profiler range")
+    ap.add_argument("--mode", default="round", choices=["round", "dp-only", "combine-check"],
+                    help="dp-only: profiling aid, runs just the layer search inside a profiler range; "
+                         "combine-check: the replicas' cross-rank step on made-up numbers over gloo (no GPU)")
     args = ap.parse_args()
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and args.impl == "ours":
+        sys.exit(launch_replicas(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.mode == "combine-check":
+        if world > 1:
+            torch.distributed.init_process_group("gloo")
+        try:
+            combine_check(rank, world)
+        finally:
+            if world > 1:
+                torch.distributed.destroy_process_group()
         return
     if world > 1:
         torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", 0)))

@@ -44,3 +44,19 @@ def test_two_replicas_report_the_slowest_time_and_the_summed_throughput(tmp_path
 def test_single_replica_is_passed_through():
     import bench
     assert bench.combine_replicas(1.0, 2.0, 3.0, 4.0, 1, torch.device("cpu")) == (1.0, 2.0, 3.0, 4.0)
+
+
+def test_plain_invocation_with_gpus_2_starts_two_ranks_itself():
+    """`python bench.py --gpus 2` without torchrun launches the two ranks on 127.0.0.1 and reports
+    n_gpus = 2 (checked with the GPU-free combine-check mode: gloo, made-up measurements)."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--mode", "combine-check"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                       # rank 0 alone prints
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2
+    assert (out["ms_per_step"], out["value"], out["e2e"], out["decode_tokens_per_s"]) == (11.0, 4.5, 5.0, 300.0)

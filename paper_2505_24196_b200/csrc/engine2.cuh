@@ -332,7 +332,8 @@ struct Shared {
   int choice[MAX_ROWS + 2];   // Eq. 2 decision per state (1: the layer output was taken)
   int choice_row[MAX_ROWS + 16];  // the same per candidate row
   int foot[NB];             // warp 0: ring pages each item in flight gives back when it retires
-  int job_words[(sizeof(Job) + 3) / 4];  // the workers' copy of the current job descriptor
+  alignas(16) int job_words[(sizeof(Job) + 3) / 4];  // the workers' copy of the current job descriptor (read back as a
+                                                     // Job: its pointer fields need 8-byte alignment)
 };
 // The workers' scratch area holds either the attention K/V tiles or, during epilogues and the
 // Eq. 2 step, the cross-warp reduction tables below (the two uses never overlap in time).
@@ -343,6 +344,8 @@ struct RedTables {
 };
 static_assert(sizeof(RedTables) <= SCRATCH_BYTES, "reduction tables must fit the scratch area");
 
+constexpr uint32_t POLL_NS = 100;      // pause between two polls of a flag or counter in global memory: the line is polled
+                                       // by every CTA while the last ones still add to it (no pause: +0.7 % on the 8B search)
 constexpr uint32_t WAIT_FAST = 1u << 12;
 constexpr uint32_t WAIT_SLOW = 1u << 22;  // x ~100 ns: gives up after roughly half a second (the defaults of
                                           // Params::wait_fast / wait_slow)
@@ -378,9 +381,9 @@ __device__ __forceinline__ bool wait_flag(const int* flag, int epoch, Ctl* ctl, 
   const uint32_t n = 2u * sh->wait_slow;
   for (uint32_t it = 0; it < n; ++it) {
     if (ld_acquire_i32(flag) >= epoch) return true;
+    __nanosleep(POLL_NS);
     if ((it & 15u) == 15u) {
       if (aborted(ctl, sh)) return false;
-      if (it > 2048u) __nanosleep(64);
     }
   }
   raise_abort(ctl, sh, true);
@@ -901,15 +904,17 @@ struct Worker {
         }
       }
     }
-    // residual rows of the first block are fetched before the accumulator is ready
-    float res[RB];
+    // residual rows of this thread's first two blocks are fetched before the accumulator is ready (a load
+    // from L2 costs 1 - 2 us here; with twelve rows no block is left that would wait for one)
+    float res[RB], res_n[RB];
 #pragma unroll
-    for (int k = 0; k < RB; ++k) res[k] = 0.f;
-    if (resid && fv && group < ncb) {
+    for (int k = 0; k < RB; ++k) { res[k] = 0.f; res_n[k] = 0.f; }
+    if (resid && fv) {
 #pragma unroll
       for (int k = 0; k < RB; ++k) {
-        const int r = group * RB + k;
+        const int r = group * RB + k, r2 = r + 2 * RB;
         if (r < J.R) res[k] = P.kind == G_O ? __ldcg(J.x_in + r * J.ldx + f) : __ldcg(p.b.x1 + (long long)r * c.d + f);
+        if (r2 < J.R) res_n[k] = P.kind == G_O ? __ldcg(J.x_in + r2 * J.ldx + f) : __ldcg(p.b.x1 + (long long)r2 * c.d + f);
       }
     }
     float wn = 0.f;
@@ -947,7 +952,10 @@ struct Worker {
           if (r < J.R && !sh->choice_row[r]) v[k] = u[k];
         }
       }
-      if (cb != group && resid && fv) {
+      if (cb == group + 2) {
+#pragma unroll
+        for (int k = 0; k < RB; ++k) res[k] = res_n[k];
+      } else if (cb != group && resid && fv) {
 #pragma unroll
         for (int k = 0; k < RB; ++k) {
           const int r = cb * RB + k;

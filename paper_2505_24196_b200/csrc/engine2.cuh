@@ -234,13 +234,10 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, u
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                : "r"(addr));
 }
-// x = hi + lo with hi, lo bf16: two values packed per register (first value in the low half)
-__device__ __forceinline__ void split2(float x, float y, uint32_t& hi, uint32_t& lo) {
+// two values rounded to bf16, packed into one register (first value in the low half)
+__device__ __forceinline__ uint32_t pack2(float x, float y) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
-  const float2 hf = __bfloat1622float2(h);
-  const __nv_bfloat162 l = __floats2bfloat162_rn(x - hf.x, y - hf.y);
-  hi = *reinterpret_cast<const uint32_t*>(&h);
-  lo = *reinterpret_cast<const uint32_t*>(&l);
+  return *reinterpret_cast<const uint32_t*>(&h);
 }
 __device__ __forceinline__ uint2 pack4(float a, float b, float c2, float d2) {
   __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c2, d2);
@@ -1356,7 +1353,7 @@ struct Worker {
       }
       // q fragments, rotated.  Element i of the first half pairs with element i + HD/2: one load
       // of each gives the rotated values of both, i.e. the fragments of k-steps ks and ks + KS/2.
-      uint32_t qh[KS][4], ql[KS][4];
+      uint32_t qh[KS][4];
       {
         // all loads first (one trip to L2), then the rotation
         float2 raw_lo[KS / 2][4], raw_hi[KS / 2][4];
@@ -1388,8 +1385,8 @@ struct Worker {
               const float4 cs = *reinterpret_cast<const float4*>(p.b.rope + (long long)tq[h] * HALF + i);
               const float2 v0 = make_float2((lo2.x * cs.x - hi2.x * cs.y) * qscale, (lo2.y * cs.z - hi2.y * cs.w) * qscale);
               const float2 v1 = make_float2((hi2.x * cs.x + lo2.x * cs.y) * qscale, (hi2.y * cs.z + lo2.y * cs.w) * qscale);
-              split2(v0.x, v0.y, qh[ks][h + kh * 2], ql[ks][h + kh * 2]);
-              split2(v1.x, v1.y, qh[ks + KS / 2][h + kh * 2], ql[ks + KS / 2][h + kh * 2]);
+              qh[ks][h + kh * 2] = pack2(v0.x, v0.y);
+              qh[ks + KS / 2][h + kh * 2] = pack2(v1.x, v1.y);
             }
           }
         }
@@ -1479,7 +1476,6 @@ struct Worker {
             const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kr + ks * 16);
             const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kr + ks * 16 + 8);
             mma_16816(s[nb], qh[ks], b0, b1);
-            mma_16816(s[nb], ql[ks], b0, b1);
           }
         }
         float mx[2] = {-INFINITY, -INFINITY};
@@ -1529,11 +1525,11 @@ struct Worker {
         }
 #pragma unroll
         for (int k2 = 0; k2 < 2; ++k2) {
-          uint32_t ph[4], pl[4];
-          split2(s[2 * k2][0], s[2 * k2][1], ph[0], pl[0]);
-          split2(s[2 * k2][2], s[2 * k2][3], ph[1], pl[1]);
-          split2(s[2 * k2 + 1][0], s[2 * k2 + 1][1], ph[2], pl[2]);
-          split2(s[2 * k2 + 1][2], s[2 * k2 + 1][3], ph[3], pl[3]);
+          uint32_t ph[4];
+          ph[0] = pack2(s[2 * k2][0], s[2 * k2][1]);
+          ph[1] = pack2(s[2 * k2][2], s[2 * k2][3]);
+          ph[2] = pack2(s[2 * k2 + 1][0], s[2 * k2 + 1][1]);
+          ph[3] = pack2(s[2 * k2 + 1][2], s[2 * k2 + 1][3]);
           const int mrow = k2 * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
           const int mcol = (lane >> 4) * 8;
 #pragma unroll
@@ -1541,9 +1537,7 @@ struct Worker {
             uint32_t b0, b1, b2, b3;
             ldmatrix_x4_trans(tc::smem_u32(v_s + mrow * LD + nb * 8 + mcol), b0, b1, b2, b3);
             mma_16816(o[nb], ph, b0, b1);
-            mma_16816(o[nb], pl, b0, b1);
             mma_16816(o[nb + 1], ph, b2, b3);
-            mma_16816(o[nb + 1], pl, b2, b3);
           }
         }
       }

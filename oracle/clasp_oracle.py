@@ -198,8 +198,14 @@ def cosine_score(x: np.ndarray, y: np.ndarray) -> float:
 APPLY, SKIP = 0, 1
 
 
+def reachable(i: int, j: int, L: int, M: int) -> bool:
+    """Can the backtrack from (L, M) pass through cell (i, j)?  Each remaining step removes at most
+    one skip, so it needs j >= M - (L - i) (and j <= min(i, M) for the cell to exist)."""
+    return M - (L - i) <= j <= min(i, M)
+
+
 def dp_search(model: Model, x: np.ndarray, cache: KVCache, C: int, pos0: int, M: int,
-              forced_choice: Optional[np.ndarray] = None):
+              forced_choice: Optional[np.ndarray] = None, prune: bool = False):
     """Algorithm 1.  x[L+1, T, d] are the full model's states of the T objective
     rows; the search reads cache positions [0, C) and never writes the cache.
 
@@ -209,6 +215,9 @@ def dp_search(model: Model, x: np.ndarray, cache: KVCache, C: int, pos0: int, M:
       margin [L+1, M+1]        score(apply) - score(skip) where both exist, else NaN
       choice [L+1, M+1] uint8  SKIP (1) / APPLY (0) taken at (i, j); 255 where undefined
       S      [L] uint8         backtracked skip set, 1 = skipped
+    prune=True leaves out the states from which (L, M) cannot be reached (the paper's Algorithm 1
+    computes them; they can never influence S): their cells stay NaN / 255 and `applied` counts the
+    decoder-layer applications that were made.
     """
     cfg = model.cfg
     L = cfg.L
@@ -220,6 +229,7 @@ def dp_search(model: Model, x: np.ndarray, cache: KVCache, C: int, pos0: int, M:
     choice = np.full((L + 1, M + 1), 255, dtype=np.uint8)
     g[0, 0] = x[0]
     D[0, 0] = 1.0
+    applied = 0
     for i in range(1, L + 1):
         g[i, 0] = x[i]                      # column 0: nothing skipped = the full model
         D[i, 0] = 1.0
@@ -227,7 +237,10 @@ def dp_search(model: Model, x: np.ndarray, cache: KVCache, C: int, pos0: int, M:
         ell = min(i - 1, M)
         w = model.layer(i - 1) if ell > 0 else None
         for j in range(1, ell + 1):
+            if prune and not reachable(i, j, L, M):
+                continue
             G, _, _ = decoder_layer(g[i - 1, j], w, cache.k[i - 1], cache.v[i - 1], C, pos0, cfg)
+            applied += 1
             s_app = cosine_score(x[i], G)
             s_skip = cosine_score(x[i], g[i - 1, j - 1])
             margin[i, j] = s_app - s_skip
@@ -238,11 +251,11 @@ def dp_search(model: Model, x: np.ndarray, cache: KVCache, C: int, pos0: int, M:
                 g[i, j], D[i, j], choice[i, j] = G, s_app, APPLY
             else:
                 g[i, j], D[i, j], choice[i, j] = g[i - 1, j - 1], s_skip, SKIP
-        if i <= M:                          # diagonal: every one of the first i layers skipped
+        if i <= M and not (prune and not reachable(i, i, L, M)):   # diagonal: the first i layers all skipped
             g[i, i] = g[i - 1, i - 1]
             D[i, i] = cosine_score(x[i], g[i, i])
             choice[i, i] = SKIP
-    return {"g": g, "D": D, "margin": margin, "choice": choice, "S": backtrack(choice, L, M)}
+    return {"g": g, "D": D, "margin": margin, "choice": choice, "S": backtrack(choice, L, M), "applied": applied}
 
 
 def backtrack(choice: np.ndarray, L: int, M: int) -> np.ndarray:

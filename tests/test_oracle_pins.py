@@ -461,3 +461,58 @@ def test_exit_threshold_stops_at_the_first_low_confidence_draft_and_stays_lossle
         assert c[-1] < thr or r["drafted"] == 4     # the last one was not, or the cap ended the round
         # the confidence is the softmax probability of the greedy token: between 1/vocab and 1
         assert all(1.0 / TINY.vocab <= x <= 1.0 for x in c)
+
+
+# ---------------- reachability pruning (result-neutral) ----------------
+
+@pytest.mark.parametrize("M", [1, 2, 3, 5, 8])
+def test_pruning_unreachable_states_changes_nothing_reachable(tiny, M):
+    """States with j < M - (L - i) cannot lie on a path to (L, M).  Leaving them out must not change
+    the skip set, any reachable score, margin, decision or state; the cells left out are exactly
+    those, and the number of layer applications drops by the count of the pruned apply-cells."""
+    model, toks, cache, am, hid, logits = tiny
+    L = TINY.L
+    p = 40
+    x = hid[p][:, None, :]
+    full = orc.dp_search(model, x, cache, p, p, M)
+    pr = orc.dp_search(model, x, cache, p, p, M, prune=True)
+    np.testing.assert_array_equal(pr["S"], full["S"])
+    n_pruned_apply = 0
+    for i in range(L + 1):
+        for j in range(M + 1):
+            exists = j <= min(i, M)
+            reach = exists and j >= M - (L - i)
+            if j == 0:
+                assert pr["D"][i, 0] == 1.0          # column 0 is the given full-model state: always there
+                continue
+            if reach:
+                assert pr["D"][i, j] == full["D"][i, j] and pr["choice"][i, j] == full["choice"][i, j]
+                np.testing.assert_array_equal(pr["g"][i, j], full["g"][i, j])
+                if not np.isnan(full["margin"][i, j]):
+                    assert pr["margin"][i, j] == full["margin"][i, j]
+            else:
+                assert np.isnan(pr["D"][i, j]) and pr["choice"][i, j] == 255
+                if exists and j <= i - 1:
+                    n_pruned_apply += 1
+    assert full["applied"] - pr["applied"] == n_pruned_apply
+    # every cell the backtrack visits is reachable (so pruning can never be seen by it)
+    i, j = L, M
+    while i > 0 and j > 0:
+        assert orc.reachable(i, j, L, M)
+        if full["choice"][i, j] == orc.SKIP:
+            j -= 1
+        i -= 1
+
+
+def test_reachability_by_brute_force():
+    """reachable(i, j) against its definition: some sequence of L - i further steps, each keeping j
+    or raising it by one (a skip), ends at M."""
+    L, M = 7, 3
+    for i in range(L + 1):
+        for j in range(M + 1):
+            if j > min(i, M):
+                continue
+            ends = {j}
+            for _ in range(L - i):
+                ends = ends | {e + 1 for e in ends}
+            assert orc.reachable(i, j, L, M) == (M in ends), (i, j)

@@ -86,6 +86,10 @@ typedef struct clasp_config {
                                    both candidates of a state through the layer's q/k/v
                                    product and keeping the chosen one.  Same operand bytes
                                    either way, so the results agree. */
+#define CLASP_FLAG_PRUNE 8      /* the search leaves out the states from which (L, M) can no longer be
+                                   reached, j < M - (L - i): Algorithm 1 computes them, but the backtrack
+                                   can never visit them.  Skip mask, g[L][M] and every reachable cell are
+                                   unchanged; the cells left out read NaN in `scores` and `margins`. */
 #define CLASP_FLAG_MULTI_KERNEL 4 /* diagnostics, bf16 model: one kernel per step (tcgen05
                                    GEMM, attention, norm, Eq. 2 select ...) instead of the
                                    persistent kernel that runs a whole call in one launch */

@@ -996,31 +996,43 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
   if (rc) return rc;
   if ((rc = rope_table(ctx, T, pos0))) return rc;
   const int64_t Td = (int64_t)T * d;
+  const bool prune = (c.flags & CLASP_FLAG_PRUNE) != 0;
   if (ctx->use_engine && M > 0 && M * T <= pk::MAX_ROWS) {
     // one cooperative launch for the whole search: step i = (layer i-1 over the candidate
     // states) + (Eq. 2 select); row 0 of the g table is x_i itself and is never stored
     clasp::dp_origin_kernel<<<1, 32, 0, ctx->stream>>>(scores, ws.choice);
     if ((rc = launch_check(ctx))) return rc;
     ctx->e_jobs.clear();
-    int cur = 0;
+    int cur = 0, prev_lo = 1;
     for (int i = 1; i <= L; ++i) {
       const int ell = (i - 1 < M) ? i - 1 : M;
+      // states the step carries: j_lo..ell (plus the diagonal state i while i <= M).  With pruning the
+      // states from which (L, M) cannot be reached any more, j < M - (L - i), are left out; the job
+      // sees its states as 1..n through pointers offset by j_lo - 1 states.
+      const int j_lo = (prune && M - (L - i) > 1) ? M - (L - i) : 1;
+      const int n = ell - j_lo + 1 > 0 ? ell - j_lo + 1 : 0;
+      const int64_t sh = j_lo - 1;
       pk::Job J{};
-      if (ell > 0) {
-        J = layer_job(ctx, i - 1, ell, T, ctx_len, false, kv[i - 1]);
-        J.x_in = ws.grow[cur] + Td; J.ldx = d; J.dp = 1;
+      if (n > 0) {
+        J = layer_job(ctx, i - 1, n, T, ctx_len, false, kv[i - 1]);
+        J.x_in = ws.grow[cur] + j_lo * Td; J.ldx = d; J.dp = 1;
       } else {
         J.type = pk::JOB_SELECT; J.T = T;
       }
-      J.i = i; J.ell = ell; J.diag = i <= M ? 1 : 0; J.M = M;
+      J.i = i; J.ell = n; J.diag = i <= M ? 1 : 0; J.M = M - (int)sh;
       J.x_i = hidden_states + (int64_t)i * layer_stride;
-      J.x_im1 = hidden_states + (int64_t)(i - 1) * layer_stride;
       J.x_tok_stride = token_stride;
-      J.g_prev = ws.grow[cur]; J.g_next = ws.grow[cur ^ 1];
-      J.D = scores + (int64_t)i * (M + 1);
-      J.margin = margins ? margins + (int64_t)i * (M + 1) : nullptr;
-      J.choice = ws.choice + (int64_t)i * (M + 1);
-      J.forced = forced_choice ? forced_choice + (int64_t)i * (M + 1) : nullptr;
+      if (j_lo == 1) { J.x_im1 = hidden_states + (int64_t)(i - 1) * layer_stride; J.x_im1_stride = token_stride; }
+      else { J.x_im1 = ws.grow[cur] + sh * Td; J.x_im1_stride = d; }
+      J.in_shift = (j_lo - prev_lo) * T;
+      prev_lo = j_lo;
+      J.g_prev = ws.grow[cur] + sh * Td; J.g_next = ws.grow[cur ^ 1] + sh * Td;
+      J.D0 = scores + (int64_t)i * (M + 1);
+      J.choice0 = ws.choice + (int64_t)i * (M + 1);
+      J.D = J.D0 + sh;
+      J.margin = margins ? margins + (int64_t)i * (M + 1) + sh : nullptr;
+      J.choice = J.choice0 + sh;
+      J.forced = forced_choice ? forced_choice + (int64_t)i * (M + 1) + sh : nullptr;
       J.norm_next = i < L ? ctx->layers[i].attn_norm : nullptr;
       J.g_final = (i == L) ? g_final : nullptr;
       ctx->e_jobs.push_back(J);
@@ -1044,18 +1056,20 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
     clasp::DpStepArgs a0{};  // g[0][0] = x_0, D[0][0] = 1: the b == 0 path of a step over x_0 itself
     a0.x_i = hidden_states; a0.x_tok_stride = token_stride; a0.G = ws.G; a0.g_prev = ws.grow[0];
     a0.g_next = ws.grow[0]; a0.D = scores; a0.margin = nullptr; a0.choice = ws.choice; a0.forced = nullptr;
-    a0.T = T; a0.d = d; a0.ell = 0; a0.i = 0; a0.M = M;
+    a0.T = T; a0.d = d; a0.ell = 0; a0.i = 0; a0.M = M; a0.j_lo = 1;
     clasp::dp_step_kernel<<<1, 256, 0, ctx->stream>>>(a0);
     if ((rc = launch_check(ctx))) return rc;
   }
   int cur = 0;
   for (int i = 1; i <= L; ++i) {
     const int ell = (i - 1 < M) ? i - 1 : M;
+    const int j_lo = (prune && M - (L - i) > 1) ? M - (L - i) : 1;   // first state the step carries
+    const int n = ell - j_lo + 1 > 0 ? ell - j_lo + 1 : 0;
     float* g_prev = ws.grow[cur];
     float* g_next = ws.grow[cur ^ 1];
-    if (ell > 0) {
-      // all candidate states j = 1..ell through layer i-1 in one batch (Sec. 3.6)
-      rc = run_layer_any(ctx, i - 1, g_prev + Td, d, ell, T, ctx_len, pos0, kv[i - 1], false, ws.G, d);
+    if (n > 0) {
+      // the candidate states j = j_lo..ell through layer i-1 in one batch (Sec. 3.6)
+      rc = run_layer_any(ctx, i - 1, g_prev + j_lo * Td, d, n, T, ctx_len, pos0, kv[i - 1], false, ws.G, d);
       if (rc) return rc;
     }
     clasp::DpStepArgs a{};
@@ -1068,8 +1082,8 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
     a.margin = margins ? margins + (int64_t)i * (M + 1) : nullptr;
     a.choice = ws.choice + (int64_t)i * (M + 1);
     a.forced = forced_choice ? forced_choice + (int64_t)i * (M + 1) : nullptr;
-    a.T = T; a.d = d; a.ell = ell; a.i = i; a.M = M;
-    const int blocks = 1 + ell + (i <= M ? 1 : 0);
+    a.T = T; a.d = d; a.ell = n; a.i = i; a.M = M; a.j_lo = j_lo;
+    const int blocks = 1 + n + (i <= M ? 1 : 0);
     clasp::dp_step_kernel<<<blocks, 256, 0, ctx->stream>>>(a);
     if ((rc = launch_check(ctx))) return rc;
     cur ^= 1;

@@ -148,6 +148,8 @@ struct Job {
                  // down epilogue), rows [BN, 2 BN) the skip candidates -- and its epilogue keeps the chosen one
   int dual_src;  // 1: this job's q/k/v operand has those two row blocks (the previous job has `defer`)
   int row_off;   // JOB_HEAD: first row (of the previous job's rows) that goes through the head
+  int in_shift;  // first row of the previous job's operand rows / decisions that is this job's row 0 (a search that
+                 // leaves out unreachable states drops leading states from one step to the next)
   int src_flag;  // step kind that publishes this job's first operand (F_PREP / F_DOWN / F_SELECT)
   int src_tgt;   // how often every CTA has published that step once the operand is complete
   int tgt[N_FLAGS];  // how often every CTA has published each step kind when this job's step is done
@@ -165,11 +167,14 @@ struct Job {
   const float* x_i;
   const float* x_im1;
   long long x_tok_stride;
+  long long x_im1_stride;  // row stride of x_im1 (the objective rows' stride, or d_model when x_im1 points into g)
   const float* g_prev;
   float* g_next;
-  float* D;
+  float* D;        // D, margin, choice, forced: row i of the tables, offset so that local state 1 is entry [1]
   float* margin;
   uint8_t* choice;
+  float* D0;       // entry (i, 0) of the score table and of the choice table
+  uint8_t* choice0;
   const uint8_t* forced;
   float* g_final;  // written with g_next[M] when not null
   // head
@@ -586,6 +591,7 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
       if (P.n_tiles == 0) continue;
       // the operand exists once every CTA has published the step that writes it
       int fkind, tgt, bmap;
+      const int row0 = P.kind == G_QKV ? J.in_shift : 0;   // first operand row of this job in the rows' buffer
       if (P.kind == G_QKV) { fkind = J.src_flag; tgt = J.src_tgt; bmap = J.dual_src ? 5 : 0; }
       else if (P.kind == G_O) { fkind = F_MERGE; tgt = J.tgt[F_MERGE]; bmap = 1; }
       else if (P.kind == G_GU) { fkind = F_O; tgt = J.tgt[F_O]; bmap = 2; }
@@ -626,12 +632,12 @@ __device__ void producer_b(const Params& p, Shared* sh, uint32_t ring_base, cons
           if (d3) {
             if (lane == 0) {
               tc::mbar_expect_tx(full, (uint32_t)P.kpi * pb_bytes);
-              tma_load_3d(dst, bmaps3[bmap], full, 0, 0, k0, pol);
+              tma_load_3d(dst, bmaps3[bmap], full, 0, row0, k0, pol);
             }
           } else {
             if (lane == 0) tc::mbar_expect_tx(full, (uint32_t)nk * pb_bytes);
             __syncwarp();
-            if (lane < nk) tc::tma_load_2d(dst + (uint32_t)lane * pb_bytes, bmaps[bmap], full, (k0 + lane) * BK, 0, pol);
+            if (lane < nk) tc::tma_load_2d(dst + (uint32_t)lane * pb_bytes, bmaps[bmap], full, (k0 + lane) * BK, row0, pol);
           }
           __syncwarp();
         }
@@ -929,7 +935,7 @@ struct Worker {
     if (tile_no == 0 && P.kind < 4) mark(T_ACC + P.kind);
     if (P.kind == G_QKV && tile_no == 0 && (J.src_flag == F_SELECT || J.dual_src)) {
       // the rows come from an Eq. 2 step: it left their factors in shared memory
-      for (int r = wtid; r < J.R; r += WORKERS) sh->rs[r] = sh->rs_next[r];
+      for (int r = wtid; r < J.R; r += WORKERS) sh->rs[r] = sh->rs_next[r + J.in_shift];
       worker_sync();
     } else if ((P.kind == G_QKV || P.kind == G_GU || P.kind == G_HEAD) && tile_no == 0) {
       // the reduction consumed every operand column, so every CTA's sums of squares are published
@@ -946,7 +952,7 @@ struct Worker {
 #pragma unroll
         for (int k = 0; k < RB; ++k) {
           const int r = cb * RB + k;
-          if (r < J.R && !sh->choice_row[r]) v[k] = u[k];
+          if (r < J.R && !sh->choice_row[r + J.in_shift]) v[k] = u[k];
         }
       }
       if (cb == group + 2) {
@@ -1097,10 +1103,10 @@ struct Worker {
   // the same by row r = (j - 1) T + t of the step: state 1's candidates are the objective rows of the step
   // before, the others row r - T ... of g, i.e. row r of the array that starts at g[i-1][0]
   __device__ __forceinline__ const float* skip_row(const Job& J, int r) const {
-    return r < J.T ? J.x_im1 + r * J.x_tok_stride : J.g_prev + (long long)r * p.c.d;
+    return r < J.T ? J.x_im1 + r * J.x_im1_stride : J.g_prev + (long long)r * p.c.d;
   }
   __device__ __forceinline__ const float* skip_src(const Job& J, int j, int t) const {
-    return j == 1 ? J.x_im1 + t * J.x_tok_stride : J.g_prev + ((long long)(j - 1) * J.T + t) * p.c.d;
+    return j == 1 ? J.x_im1 + t * J.x_im1_stride : J.g_prev + ((long long)(j - 1) * J.T + t) * p.c.d;
   }
 
   static constexpr double COS_FIX = 268435456.0;  // 2^28: sums up to 3e10 with 4e-9 resolution
@@ -1114,7 +1120,7 @@ struct Worker {
   // row and s the skip candidate of state j: x_old[t] for j = 1, else g[j - 1][t].  They are added
   // to the job's accumulators as soon as the candidates exist, off the step's critical path.
   __device__ void pre_sums(int tgt, int rows, int Tn, const float* x_new, const float* x_old, long long xs,
-                           const float* g, bool fv, int f) {
+                           long long xs_old, const float* g, bool fv, int f) {
     const Cfg& c = p.c;
     RedTables* T = tables();
     const int quarter = ww & 3, group = ww >> 2;
@@ -1129,7 +1135,7 @@ struct Worker {
         if (fv && r < rows) {
           const int j = rd.div(r) + 1, t = rd.mod(r);
           xv = __ldg(x_new + t * xs + f);
-          sv = __ldcg((j == 1 ? x_old + t * xs : g + ((long long)(j - 1) * Tn + t) * c.d) + f);
+          sv = __ldcg((j == 1 ? x_old + t * xs_old : g + ((long long)(j - 1) * Tn + t) * c.d) + f);
         }
         pa[k] = xv * sv;
         pa[RB + k] = sv * sv;
@@ -1180,7 +1186,7 @@ struct Worker {
     const RowDiv rd(J.T);
     const float wn = (fv && J.norm_next) ? __ldg(J.norm_next + f) : 0.f;   // needed right after the decision
     // (a layer job adds its sums over the skip candidates while it waits for its o product)
-    if (J.type == JOB_SELECT) pre_sums(jb, rows, J.T, J.x_i, J.x_im1, J.x_tok_stride, J.g_prev, fv, f);
+    if (J.type == JOB_SELECT) pre_sums(jb, rows, J.T, J.x_i, J.x_im1, J.x_tok_stride, J.x_im1_stride, J.g_prev, fv, f);
     if (!from_epilogue) {
       // no layer ran for this CTA's features: only skip candidates exist
 #pragma unroll
@@ -1232,8 +1238,8 @@ struct Worker {
       }
     }
     if (blockIdx.x == 0 && wtid == 0) {
-      J.D[0] = 1.0f;
-      J.choice[0] = 0;
+      J.D0[0] = 1.0f;
+      J.choice0[0] = 0;
     }
     worker_sync();
     mark(T_DP_DECIDED);
@@ -1716,7 +1722,8 @@ struct Worker {
           // Eq. 2 step over the skip candidates, which the previous step left in g
           const int f_lo = __ldg(split_lo(S_D) + blockIdx.x), f_hi = __ldg(split_lo(S_D) + blockIdx.x + 1);
           const int fl = feat_local(f_hi - f_lo, ww & 3, lane);
-          pre_sums(jb, (J.ell + (J.diag ? 1 : 0)) * J.T, J.T, J.x_i, J.x_im1, J.x_tok_stride, J.g_prev, fl >= 0, f_lo + fl);
+          pre_sums(jb, (J.ell + (J.diag ? 1 : 0)) * J.T, J.T, J.x_i, J.x_im1, J.x_tok_stride, J.x_im1_stride, J.g_prev, fl >= 0,
+                   f_lo + fl);
         }
         for (int t = 0; t < P.n_tiles; ++t)
           if (!epilogue(J, jb, P, tiles[P.tile0 + t], t, keep_y, keep_s)) return false;

@@ -393,7 +393,7 @@ __global__ void attn_merge_kernel(const float* __restrict__ part_acc, const floa
 struct DpStepArgs {
   const float* x_i;       // row t at x_i + t * x_tok_stride
   int64_t x_tok_stride;
-  const float* G;         // [ell*T, d] layer outputs for j = 1..ell
+  const float* G;         // [ell*T, d] layer outputs of the ell states j = j_lo .. j_lo + ell - 1
   const float* g_prev;    // [(M+1)*T, d]
   float* g_next;          // [(M+1)*T, d]
   float* D;               // row i of the tables: [M+1]
@@ -401,6 +401,7 @@ struct DpStepArgs {
   uint8_t* choice;        // row i of the choice table (always present: workspace)
   const uint8_t* forced;  // row i or null
   int T, d, ell, i, M;
+  int j_lo;               // first state the step carries (1, or later when unreachable states are left out)
 };
 
 __device__ __forceinline__ void block_sum3(double (&v)[3], double* sh) {
@@ -456,7 +457,7 @@ __global__ void dp_step_kernel(DpStepArgs a) {
     }
     return;
   }
-  if (b == a.ell + 1) {  // diagonal j = i: all of the first i layers skipped
+  if (b == a.ell + 1) {  // (only launched while i <= M) diagonal j = i: all of the first i layers skipped
     const int j = a.i;
     const float* src = a.g_prev + (int64_t)(j - 1) * Td;
     const float sc = mean_cosine(a, src, sh);
@@ -468,8 +469,8 @@ __global__ void dp_step_kernel(DpStepArgs a) {
     }
     return;
   }
-  const int j = b;
-  const float* app = a.G + (int64_t)(j - 1) * Td;
+  const int j = a.j_lo + b - 1;
+  const float* app = a.G + (int64_t)(b - 1) * Td;
   const float* skp = a.g_prev + (int64_t)(j - 1) * Td;
   const float s_app = mean_cosine(a, app, sh);
   const float s_skip = mean_cosine(a, skp, sh);

@@ -35,11 +35,11 @@ SLOT = {"start": 0, "qkv": 1, "att_ready": 2, "att_pub": 5, "merge": 6, "o": 7, 
         "mma_last_qkv": 20, "mma_last_o": 21, "mma_last_gu": 22, "mma_last_down": 23}
 
 
-def build_engine(name, max_ctx, max_M, max_T, max_head_rows=8):
+def build_engine(name, max_ctx, max_M, max_T, max_head_rows=8, flags=0):
     cfg = datagen.CONFIGS[name]
     dev = torch.device("cuda", 0)
     ccfg = clasp.make_config(cfg, max_ctx=max_ctx, max_rows=128, max_M=max_M, max_T=max_T,
-                             max_head_rows=max_head_rows)
+                             max_head_rows=max_head_rows, flags=flags)
     eng = clasp.Clasp(ccfg, device=dev)
     layers = [datagen.layer_weights(cfg, l, dev) for l in range(cfg.L)]
     head = datagen.head_weights(cfg, dev)
@@ -90,7 +90,7 @@ def layer_split(eng, run, n_jobs):
 def cmd_dp(args):
     cfg0 = datagen.CONFIGS[args.model]
     max_ctx = max(args.ctx) + 64
-    cfg, ccfg, eng, keep = build_engine(args.model, max_ctx, max(args.M), max(args.T))
+    cfg, ccfg, eng, keep = build_engine(args.model, max_ctx, max(args.M), max(args.T), flags=args.flags)
     kv = clasp.KVCache(ccfg, device=eng.device)
     toks = datagen.token_ids(cfg, max(args.ctx)).to(eng.device)
     d, L = cfg.d_model, cfg.L
@@ -116,7 +116,8 @@ def cmd_dp(args):
                 torch.cuda.synchronize()
                 ms = a.elapsed_time(b) / args.reps
                 byts = (L - 1) * (cfg.layer_matrix_bytes() + 2 * p0 * cfg.n_kv_heads * cfg.head_dim * esz)
-                out = {"what": "dp_search", "model": cfg.name, "ctx": C, "M": M, "T": T, "dp_ms": round(ms, 4),
+                out = {"what": "dp_search", "model": cfg.name, "flags": args.flags, "ctx": C, "M": M, "T": T,
+                       "dp_ms": round(ms, 4),
                        "algorithmic_gb": round(byts / 1e9, 3), "gbs": round(byts / ms / 1e6, 1),
                        "skipped": int(r["S"].sum()), "device_status": eng.device_status()}
                 out.update(layer_split(eng, run, L))
@@ -231,6 +232,7 @@ def main():
     p.add_argument("--M", type=int, nargs="+", default=[12])
     p.add_argument("--T", type=int, nargs="+", default=[1])
     p.add_argument("--reps", type=int, default=10)
+    p.add_argument("--flags", type=int, default=0, help="library flags (8: leave out unreachable states)")
     p = sub.add_parser("trace")
     p.add_argument("--model", default="8b")
     p.add_argument("--ctx", type=int, nargs="+", default=[512])

@@ -14,7 +14,7 @@ from tests.util import Pair, check_search_against_oracle, close_hidden, kv_to_or
 
 pytestmark = pytest.mark.gpu
 
-FLAG_FORCE_SIMT, FLAG_NO_DEFER, FLAG_MULTI_KERNEL = 1, 2, 4
+FLAG_FORCE_SIMT, FLAG_NO_DEFER, FLAG_MULTI_KERNEL, FLAG_PRUNE = 1, 2, 4, 8
 # (config name, library flags): the fp32 model runs the CUDA-core GEMM; the bf16 models run
 # the tcgen05 GEMM, and once more with the CUDA-core GEMM as a cross-check of the rest.
 ENGINES = [("tiny", 0), ("small", 0), ("mini8b", 0), ("small", FLAG_FORCE_SIMT)]
@@ -202,6 +202,50 @@ def test_search_with_and_without_deferred_decision(pair):
         Dc = c["D"].cpu().numpy()
         np.testing.assert_allclose(Dc[~np.isnan(Dc)], ref["D"][~np.isnan(Dc)], atol=1e-3)
         assert close_hidden(c["g_final"].cpu().numpy(), ref["g"][L, M], tol_hidden(cfg))
+        assert eng2.device_status() == 0
+    finally:
+        eng2.close()
+
+
+@pytest.mark.parametrize("M,T,extra", [(2, 1, 0), (3, 1, 0), (3, 2, 0), (4, 1, 0), (3, 1, FLAG_NO_DEFER)])
+def test_search_without_the_unreachable_states(pair, M, T, extra):
+    """CLASP_FLAG_PRUNE leaves out the states from which (L, M) cannot be reached (j < M - (L - i)).
+    Result-neutral: the skip set, g[L][M] and every reachable cell equal the unpruned search's (a row's
+    arithmetic does not depend on which other rows share its launch); the cells left out read NaN,
+    exactly where the oracle's pruned table has none either."""
+    cfg = pair.cfg
+    L, d = cfg.L, cfg.d_model
+    M = min(M, L)
+    n = 40
+    toks, ocache, am_o, hid_o, _, kv, am_g, hid_g = _prefill_both(pair, n)
+    p0 = n - T
+    full = pair.engine.dp_search(hid_g[p0], d, (L + 1) * d, kv, p0, p0, T, M)
+    eng2 = pair.engine_with_flags(pair.ccfg.flags | FLAG_PRUNE | extra)
+    try:
+        pr = eng2.dp_search(hid_g[p0], d, (L + 1) * d, kv, p0, p0, T, M)
+        torch.cuda.synchronize()
+        assert eng2.device_status() == 0 and pair.engine.device_status() == 0
+        Df, Dp = full["D"].cpu().numpy(), pr["D"].cpu().numpy()
+        mf, mp = full["margin"].cpu().numpy(), pr["margin"].cpu().numpy()
+        x_o = np.transpose(hid_o[p0:n], (1, 0, 2))
+        ref = orc.dp_search(pair.oracle, x_o, ocache, p0, p0, M, prune=True)
+        assert np.array_equal(np.isnan(Dp), np.isnan(ref["D"]))
+        assert np.array_equal(np.isnan(mp), np.isnan(ref["margin"]))
+        keep = ~np.isnan(Dp)
+        assert np.isnan(Dp).sum() > np.isnan(Df).sum() or M == 1      # something was left out
+        np.testing.assert_allclose(Dp[keep], Df[keep], rtol=0, atol=1e-6)
+        km = ~np.isnan(mp)
+        np.testing.assert_allclose(mp[km], mf[km], rtol=0, atol=2e-6)
+        assert torch.equal(pr["S"], full["S"])
+        assert rel_l2(pr["g_final"].cpu().numpy(), full["g_final"].cpu().numpy()) < 1e-6
+        # and against the oracle's pruned search with its decisions forced
+        forced = torch.from_numpy(ref["choice"].copy()).cuda()
+        pf = eng2.dp_search(hid_g[p0], d, (L + 1) * d, kv, p0, p0, T, M, forced_choice=forced)
+        Dq = pf["D"].cpu().numpy()
+        assert np.array_equal(np.isnan(Dq), np.isnan(ref["D"]))
+        np.testing.assert_allclose(Dq[keep], ref["D"][keep], atol=1e-3)
+        np.testing.assert_array_equal(pf["S"].cpu().numpy(), ref["S"])
+        assert close_hidden(pf["g_final"].cpu().numpy(), ref["g"][L, M], tol_hidden(cfg))
         assert eng2.device_status() == 0
     finally:
         eng2.close()

@@ -367,3 +367,136 @@ def greedy_self_speculative(model: Model, prompt: Sequence[int], n_new: int, max
         if n_verify % dp_interval == 0:
             S = search(obj_row, obj_pos)
     return out[:n_new], rounds
+
+
+# --------------------------------------------------------------------------
+# non-greedy decoding: speculative sampling (Sec. 4, Table 1 "Temperature = 1";
+# the accept / resample rule is the one of Leviathan et al. 2023, which the
+# paper cites for losslessness)
+# --------------------------------------------------------------------------
+# Random numbers come from one counter-based generator, Philox4x32-10 (Salmon
+# et al., "Parallel random numbers: as easy as 1, 2, 3", SC'11), keyed by the
+# seed and counted by (index, position, purpose, round), so that every draw is
+# a pure function of where it is used.  The CUDA side implements the same
+# published definition on its own.
+
+PHILOX_M0, PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+PHILOX_W0, PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+DRAW_DRAFT, DRAW_ACCEPT, DRAW_RESIDUAL, DRAW_TARGET = 0, 1, 2, 3
+
+
+def philox4x32_10(c0, c1, c2, c3, k0: int, k1: int):
+    """Ten rounds of Philox-4x32 on uint32 arrays c0..c3 (broadcast together) with key (k0, k1)."""
+    c0, c1, c2, c3 = np.broadcast_arrays(*[np.asarray(c, dtype=np.uint64) for c in (c0, c1, c2, c3)])
+    mask = np.uint64(0xFFFFFFFF)
+    for r in range(10):
+        p0 = np.uint64(PHILOX_M0) * c0                      # 64-bit products of 32-bit factors
+        p1 = np.uint64(PHILOX_M1) * c2
+        hi0, lo0 = p0 >> np.uint64(32), p0 & mask
+        hi1, lo1 = p1 >> np.uint64(32), p1 & mask
+        c0, c1, c2, c3 = hi1 ^ c1 ^ np.uint64(k0), lo1, hi0 ^ c3 ^ np.uint64(k1), lo0
+        k0 = (k0 + PHILOX_W0) & 0xFFFFFFFF
+        k1 = (k1 + PHILOX_W1) & 0xFFFFFFFF
+    return [c.astype(np.uint32) for c in (c0, c1, c2, c3)]
+
+
+def uniform_draws(seed: int, index, position: int, purpose: int, rnd: int) -> np.ndarray:
+    """Uniforms in (0, 1) on a 2^-24 grid (exact in float and double): ((x >> 8) + 0.5) / 2^24 of
+    the first Philox word for counter (index, position, purpose, round) and key = the 64-bit seed."""
+    x = philox4x32_10(index, position, purpose, rnd, seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)[0]
+    return ((x >> np.uint32(8)).astype(np.float64) + 0.5) * (1.0 / 16777216.0)
+
+
+def gumbel_max_sample(logits: np.ndarray, temperature: float, seed: int, position: int, purpose: int,
+                      rnd: int) -> int:
+    """A sample of softmax(logits / temperature): argmax of logits / temperature + Gumbel noise
+    (noise of entry v from draw v); entries at -inf can never win; lowest index on exact ties."""
+    u = uniform_draws(seed, np.arange(logits.shape[0]), position, purpose, rnd)
+    return int(np.argmax(logits / temperature - np.log(-np.log(u))))
+
+
+def log_softmax(z: np.ndarray) -> np.ndarray:
+    z = z - z.max()
+    return z - np.log(np.exp(z).sum())
+
+
+def speculative_accept(p_logits: np.ndarray, q_logits: np.ndarray, drafts: Sequence[int], temperature: float,
+                       seed: int, pos0: int, rnd: int):
+    """The accept / resample rule.  drafts[k] was sampled from q_k = softmax(q_logits[k] / T) and
+    would sit at position pos0 + k; p_k = softmax(p_logits[k] / T) is the full model's distribution
+    there (p_logits has one more row: the position after the last draft).  Draft k is accepted with
+    probability min(1, p_k(x) / q_k(x)); the first rejected position gets a sample of
+    norm(max(0, p_k - q_k)) instead and ends the round; if every draft is accepted the next position
+    gets a sample of p_K.  Returns (accepted, committed tokens) -- accepted + 1 tokens."""
+    K = len(drafts)
+    out = []
+    for k in range(K):
+        lp, lq = log_softmax(p_logits[k] / temperature), log_softmax(q_logits[k] / temperature)
+        x = int(drafts[k])
+        u = float(uniform_draws(seed, 0, pos0 + k, DRAW_ACCEPT, rnd))
+        if u < np.exp(min(0.0, lp[x] - lq[x])):
+            out.append(x)
+            continue
+        resid = np.maximum(np.exp(lp) - np.exp(lq), 0.0)
+        with np.errstate(divide="ignore"):
+            lr = np.log(resid)                              # -inf where p <= q
+        out.append(gumbel_max_sample(lr, 1.0, seed, pos0 + k, DRAW_RESIDUAL, rnd))
+        return k, out
+    out.append(gumbel_max_sample(p_logits[K], temperature, seed, pos0 + K, DRAW_TARGET, rnd))
+    return K, out
+
+
+def sampling_autoregressive(model: Model, prompt: Sequence[int], n_new: int, max_ctx: int, temperature: float,
+                            seed: int) -> List[int]:
+    """Plain ancestral sampling of the full model (the distribution speculative sampling preserves)."""
+    cache = KVCache(model.cfg, max_ctx)
+    _, _, lg = verify_forward(model, prompt, cache, 0)
+    pos = len(prompt)
+    out = [gumbel_max_sample(lg[-1], temperature, seed, pos, DRAW_TARGET, 0)]
+    while len(out) < n_new:
+        _, _, lg = verify_forward(model, [out[-1]], cache, pos)
+        pos += 1
+        out.append(gumbel_max_sample(lg[0], temperature, seed, pos, DRAW_TARGET, 0))
+    return out
+
+
+def sampling_self_speculative(model: Model, prompt: Sequence[int], n_new: int, max_ctx: int, M: int, K: int,
+                              temperature: float, seed: int, fixed_mask: Optional[Sequence[int]] = None,
+                              dp_interval: int = 1):
+    """The three-stage loop of Sec. 3.1 with sampling instead of arg-max: drafts are samples of the
+    layer-skipped model, the verification applies the accept / resample rule, the layer search runs on
+    the last accepted position as in the greedy loop.  Returns (tokens, per-round stats)."""
+    cfg = model.cfg
+    cache = KVCache(cfg, max_ctx)
+    P = len(prompt)
+    _, hidden, lg = verify_forward(model, prompt, cache, 0)
+    out = [gumbel_max_sample(lg[-1], temperature, seed, P, DRAW_TARGET, 0)]
+    pending, n_valid = out[0], P
+
+    def search(hid_row, obj_pos):
+        if fixed_mask is not None:
+            return np.asarray(fixed_mask, dtype=np.uint8)
+        return dp_search(model, hid_row[:, None, :], cache, obj_pos, obj_pos, M)["S"]
+
+    S = search(hidden[P - 1], P - 1)
+    rounds = []
+    rnd = 0
+    while len(out) < n_new:
+        rnd += 1
+        drafts, q_rows, tok = [], [], pending
+        for k in range(K):
+            _, _, lq = verify_forward(model, [tok], cache, n_valid + k, skip=S)
+            # draft k is the token that would sit at position n_valid + k + 1
+            tok = gumbel_max_sample(lq[0], temperature, seed, n_valid + k + 1, DRAW_DRAFT, rnd)
+            drafts.append(tok)
+            q_rows.append(lq[0])
+        _, hidden, lp = verify_forward(model, [pending] + drafts, cache, n_valid)
+        a, new = speculative_accept(lp, np.stack(q_rows), drafts, temperature, seed, n_valid + 1, rnd)
+        out.extend(new)
+        rounds.append({"accepted": a, "S": S.copy(), "drafts": drafts, "committed": new})
+        obj_row, obj_pos = hidden[a], n_valid + a
+        n_valid += a + 1
+        pending = new[-1]
+        if rnd % dp_interval == 0:
+            S = search(obj_row, obj_pos)
+    return out[:n_new], rounds

@@ -215,6 +215,38 @@ int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int
                         int32_t pos, const clasp_kv_layer* kv, int32_t* token_out,
                         float* top1_prob_out);
 
+/* Non-greedy decoding (Sec. 4 and Table 1, "Temperature = 1"; the accept / resample rule is the one of
+ * speculative sampling, which the paper cites for losslessness).  Random numbers are Philox4x32-10
+ * draws keyed by `seed` and counted by (index, position, purpose, round): a call is a pure function of
+ * its arguments, there is no generator state.
+ *
+ * clasp_draft_sample: one token through the layer-skipped model as clasp_draft_forward, but the next
+ * token is a draw of softmax(logits / temperature) (arg-max of logits / T + Gumbel noise, lowest index
+ * on ties) instead of the arg-max.
+ *   logits_out   device, float[vocab], 16-byte aligned, out: the draft model's logits for the drafted
+ *                position (the verification needs them)
+ *   round        >= 0: distinguishes the draws of different rounds at the same position
+ * clasp_verify_sample: full-model forward over n tokens at pos0.. as clasp_verify; the last
+ * n_drafts tokens are drafts (tokens[n - n_drafts + k] sampled from draft_logits[k]).  Draft k is
+ * accepted with probability min(1, p_k(x) / q_k(x)); the first rejected position gets a draw of
+ * norm(max(0, p_k - q_k)) and ends the walk; if all are accepted the position after the last draft gets
+ * a draw of the full model's distribution.  n_drafts == 0 just samples the token after the n rows
+ * (prompt prefill, plain ancestral sampling).
+ *   draft_logits   device, float[n_drafts * vocab] (may be NULL when n_drafts == 0)
+ *   logits_ws      device, float[(n_drafts + 1) * vocab], 16-byte aligned: receives the full model's
+ *                  logits of the head rows (caller-owned scratch, readable afterwards)
+ *   n_accepted_out device, int32[1]; committed_out device, int32[n_drafts + 1]: the accepted drafts
+ *                  followed by the sampled token; must not overlap `tokens`
+ * Errors: INVALID_ARG (temperature <= 0, null or misaligned buffers, n_drafts >= n), CAPACITY
+ * (n_drafts > 63 or as clasp_verify with n_head_rows = n_drafts + 1). */
+int clasp_draft_sample(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int32_t* token_in,
+                       int32_t pos, const clasp_kv_layer* kv, float temperature, uint64_t seed,
+                       int32_t round, int32_t* token_out, float* logits_out);
+int clasp_verify_sample(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0,
+                        const clasp_kv_layer* kv, int32_t n_drafts, const float* draft_logits,
+                        float temperature, uint64_t seed, int32_t round, float* logits_ws,
+                        int32_t* n_accepted_out, int32_t* committed_out, float* hidden_out);
+
 /* Greedy acceptance (Sec. 3.1, verification stage).  HOST pointers, no GPU
  * work: draft[K] are the drafted tokens, full_argmax[K+1] the full model's
  * greedy tokens for the rows [pending, draft_1..draft_K].  Writes the number a

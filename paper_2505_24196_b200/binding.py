@@ -22,7 +22,7 @@ FLAG_FORCE_SIMT, FLAG_NO_DEFER, FLAG_MULTI_KERNEL, FLAG_PRUNE = 1, 2, 4, 8
 SYMBOLS = ["clasp_workspace_bytes", "clasp_create", "clasp_destroy", "clasp_load_layers", "clasp_load_head",
            "clasp_dp_search", "clasp_verify", "clasp_draft_forward", "clasp_accept", "clasp_layer_forward",
            "clasp_gemm_xwT", "clasp_gemm_xwT_noalloc", "clasp_profile_gemm", "clasp_last_device_status", "clasp_launch_count", "clasp_engine_trace", "clasp_strerror",
-           "clasp_engine_active", "clasp_set_wait_limit"]
+           "clasp_engine_active", "clasp_set_wait_limit", "clasp_draft_sample", "clasp_verify_sample"]
 
 
 class ClaspConfig(C.Structure):
@@ -78,6 +78,11 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.clasp_verify.argtypes = [vp, vp, i32, i32, C.POINTER(ClaspKvLayer), i32, vp, vp]
     lib.clasp_draft_forward.restype = C.c_int
     lib.clasp_draft_forward.argtypes = [vp, C.c_char_p, vp, i32, C.POINTER(ClaspKvLayer), vp, vp]
+    lib.clasp_draft_sample.restype = C.c_int
+    lib.clasp_draft_sample.argtypes = [vp, C.c_char_p, vp, i32, C.POINTER(ClaspKvLayer), C.c_float, C.c_uint64, i32, vp, vp]
+    lib.clasp_verify_sample.restype = C.c_int
+    lib.clasp_verify_sample.argtypes = [vp, vp, i32, i32, C.POINTER(ClaspKvLayer), i32, vp, C.c_float, C.c_uint64, i32,
+                                        vp, vp, vp, vp]
     lib.clasp_accept.restype = C.c_int
     lib.clasp_accept.argtypes = [C.POINTER(i32), C.POINTER(i32), i32, C.POINTER(i32), C.POINTER(i32)]
     lib.clasp_layer_forward.restype = C.c_int
@@ -238,6 +243,20 @@ class Clasp:
                       token_out: torch.Tensor, top1_prob_out: Optional[torch.Tensor] = None):
         _check(self.lib.clasp_draft_forward(self.handle, skip_mask_host, token_in.data_ptr(), pos, kv.array,
                                             token_out.data_ptr(), _ptr(top1_prob_out)), "clasp_draft_forward")
+
+    def draft_sample(self, skip_mask_host: bytes, token_in: torch.Tensor, pos: int, kv: KVCache, temperature: float,
+                     seed: int, rnd: int, token_out: torch.Tensor, logits_out: torch.Tensor):
+        _check(self.lib.clasp_draft_sample(self.handle, skip_mask_host, token_in.data_ptr(), pos, kv.array, temperature,
+                                           seed, rnd, token_out.data_ptr(), logits_out.data_ptr()), "clasp_draft_sample")
+
+    def verify_sample(self, tokens: torch.Tensor, pos0: int, kv: KVCache, n_drafts: int,
+                      draft_logits: Optional[torch.Tensor], temperature: float, seed: int, rnd: int,
+                      logits_ws: torch.Tensor, n_accepted_out: torch.Tensor, committed_out: torch.Tensor,
+                      hidden_out: Optional[torch.Tensor] = None):
+        _check(self.lib.clasp_verify_sample(self.handle, tokens.data_ptr(), tokens.numel(), pos0, kv.array, n_drafts,
+                                            _ptr(draft_logits), temperature, seed, rnd, logits_ws.data_ptr(),
+                                            n_accepted_out.data_ptr(), committed_out.data_ptr(), _ptr(hidden_out)),
+               "clasp_verify_sample")
 
     def accept(self, draft: Sequence[int], full_argmax: Sequence[int]):
         K = len(draft)

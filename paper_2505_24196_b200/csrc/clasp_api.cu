@@ -19,6 +19,7 @@
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
 #include "engine2.cuh"
+#include "sampling.cuh"
 
 namespace {
 
@@ -70,6 +71,7 @@ struct Workspace {
   CUtensorMap* wmaps;
   clasp::pk::Job* jobs;
   int* tabs;
+  clasp::smp::AcceptScratch* spec;
   int e_chunk_cap;
   int e_run_len;
   int e_rcap;
@@ -126,6 +128,7 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
   w.att_ml = (float2*)take(R * c.n_q_heads * att_chunks * sizeof(float2));
   w.logits = (float*)take((size_t)c.max_head_rows * c.vocab * 4);
   w.partial = (float*)take(PARTIAL_FLOATS * 4);
+  w.spec = (clasp::smp::AcceptScratch*)take(sizeof(clasp::smp::AcceptScratch));
   if (c.dtype == CLASP_BF16) {
     // buffers of the persistent layer engine (per-CTA tables sized for ENGINE_MAX_CTAS)
     namespace pk = clasp::pk;
@@ -493,7 +496,8 @@ bool layers_ready(const clasp_ctx* ctx) {
 }
 
 // final norm + LM head + argmax over `rows` rows of x (float, stride ldx)
-int run_head(clasp_ctx* ctx, const float* x, int64_t ldx, int rows, int32_t* argmax_out, float* top1) {
+int run_head(clasp_ctx* ctx, const float* x, int64_t ldx, int rows, int32_t* argmax_out, float* top1,
+             float* logits_out = nullptr) {
   const clasp_config& c = ctx->cfg;
   int rc;
   if (c.dtype == CLASP_FP32) rc = rmsnorm<float>(ctx, x, ldx, ctx->final_norm, rows, ctx->ws.xn);
@@ -505,7 +509,11 @@ int run_head(clasp_ctx* ctx, const float* x, int64_t ldx, int rows, int32_t* arg
   g.yf = ctx->ws.logits; g.ldy = c.vocab;
   if ((rc = gemm(ctx, g))) return rc;
   clasp::argmax_kernel<<<rows, 1024, 0, ctx->stream>>>(ctx->ws.logits, c.vocab, argmax_out, top1);
-  return launch_check(ctx);
+  if ((rc = launch_check(ctx))) return rc;
+  if (logits_out)
+    CUDA_TRY(cudaMemcpyAsync(logits_out, ctx->ws.logits, (size_t)rows * c.vocab * sizeof(float), cudaMemcpyDeviceToDevice,
+                             ctx->stream));
+  return CLASP_OK;
 }
 
 int embed_rows(clasp_ctx* ctx, const int32_t* tokens, int n, float* out, int64_t ldo) {
@@ -1097,8 +1105,11 @@ int clasp_dp_search(clasp_ctx* ctx, const float* hidden_states, int64_t layer_st
   return CLASP_OK;
 }
 
-int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0, const clasp_kv_layer* kv,
-                 int32_t n_head_rows, int32_t* argmax_out, float* hidden_out) {
+}  // extern "C"
+
+namespace {
+int verify_impl(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0, const clasp_kv_layer* kv,
+                int32_t n_head_rows, int32_t* argmax_out, float* hidden_out, float* logits_out) {
   if (!ctx || !tokens || !kv || n < 1 || pos0 < 0 || n_head_rows < 0 || n_head_rows > n)
     return CLASP_ERR_INVALID_ARG;
   if (n_head_rows > 0 && !argmax_out) return CLASP_ERR_INVALID_ARG;
@@ -1135,7 +1146,7 @@ int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0,
     if (n_head_rows > 0) {
       pk::Job H{};
       H.type = pk::JOB_HEAD; H.R = n_head_rows; H.T = 1; H.row_off = n - n_head_rows;
-      H.argmax_out = argmax_out;
+      H.argmax_out = argmax_out; H.logits_out = logits_out;
       ctx->e_jobs.push_back(H);
     }
     link_jobs(ctx->e_jobs);
@@ -1165,12 +1176,12 @@ int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0,
     ldx = d;
   }
   if (n_head_rows > 0)
-    return run_head(ctx, x + (int64_t)(n - n_head_rows) * ldx, ldx, n_head_rows, argmax_out, nullptr);
+    return run_head(ctx, x + (int64_t)(n - n_head_rows) * ldx, ldx, n_head_rows, argmax_out, nullptr, logits_out);
   return CLASP_OK;
 }
 
-int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int32_t* token_in, int32_t pos,
-                        const clasp_kv_layer* kv, int32_t* token_out, float* top1_prob_out) {
+int draft_impl(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int32_t* token_in, int32_t pos,
+               const clasp_kv_layer* kv, int32_t* token_out, float* top1_prob_out, float* logits_out) {
   if (!ctx || !skip_mask_host || !token_in || !kv || !token_out || pos < 0) return CLASP_ERR_INVALID_ARG;
   const clasp_config& c = ctx->cfg;
   if ((int64_t)pos + 1 > c.max_ctx) return CLASP_ERR_CAPACITY;
@@ -1201,6 +1212,7 @@ int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int
     ctx->e_jobs.back().norm_next = ctx->final_norm;
     pk::Job H{};
     H.type = pk::JOB_HEAD; H.R = 1; H.T = 1; H.row_off = 0; H.argmax_out = token_out; H.top1_out = top1_prob_out;
+    H.logits_out = logits_out;
     ctx->e_jobs.push_back(H);
     link_jobs(ctx->e_jobs);
     return engine_launch(ctx, 1, 0);
@@ -1211,7 +1223,54 @@ int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int
     if ((rc = run_layer_any(ctx, l, a, d, 1, 1, pos, pos, kv[l], true, b, d))) return rc;
     float* t = a; a = b; b = t;
   }
-  return run_head(ctx, a, d, 1, token_out, top1_prob_out);
+  return run_head(ctx, a, d, 1, token_out, top1_prob_out, logits_out);
+}
+}  // namespace
+
+extern "C" {
+
+int clasp_verify(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0, const clasp_kv_layer* kv,
+                 int32_t n_head_rows, int32_t* argmax_out, float* hidden_out) {
+  return verify_impl(ctx, tokens, n, pos0, kv, n_head_rows, argmax_out, hidden_out, nullptr);
+}
+
+int clasp_draft_forward(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int32_t* token_in, int32_t pos,
+                        const clasp_kv_layer* kv, int32_t* token_out, float* top1_prob_out) {
+  return draft_impl(ctx, skip_mask_host, token_in, pos, kv, token_out, top1_prob_out, nullptr);
+}
+
+int clasp_draft_sample(clasp_ctx* ctx, const uint8_t* skip_mask_host, const int32_t* token_in, int32_t pos,
+                       const clasp_kv_layer* kv, float temperature, uint64_t seed, int32_t round, int32_t* token_out,
+                       float* logits_out) {
+  if (!logits_out || !(temperature > 0.f) || round < 0 || !al16(logits_out)) return CLASP_ERR_INVALID_ARG;
+  int rc = draft_impl(ctx, skip_mask_host, token_in, pos, kv, token_out, nullptr, logits_out);
+  if (rc) return rc;
+  // the drafted token will sit at position pos + 1
+  clasp::smp::gumbel_argmax_kernel<<<1, clasp::smp::THREADS, 0, ctx->stream>>>(
+      logits_out, ctx->cfg.vocab, 1.0f / temperature, (unsigned long long)seed, pos + 1, clasp::smp::DRAW_DRAFT, round,
+      token_out);
+  return launch_check(ctx);
+}
+
+int clasp_verify_sample(clasp_ctx* ctx, const int32_t* tokens, int32_t n, int32_t pos0, const clasp_kv_layer* kv,
+                        int32_t n_drafts, const float* draft_logits, float temperature, uint64_t seed, int32_t round,
+                        float* logits_ws, int32_t* n_accepted_out, int32_t* committed_out, float* hidden_out) {
+  if (!ctx || !logits_ws || !n_accepted_out || !committed_out || n_drafts < 0 || n_drafts >= n || round < 0 ||
+      !(temperature > 0.f) || (n_drafts > 0 && !draft_logits) || !al16(logits_ws))
+    return CLASP_ERR_INVALID_ARG;
+  if (n_drafts > clasp::smp::MAX_DRAFTS) return CLASP_ERR_CAPACITY;
+  // the last n_drafts + 1 rows go through the head; their logits land in logits_ws
+  int rc = verify_impl(ctx, tokens, n, pos0, kv, n_drafts + 1, committed_out, hidden_out, logits_ws);
+  if (rc) return rc;
+  const int first = pos0 + n - n_drafts;   // position of the first draft (of the sampled token when there is none)
+  clasp::smp::spec_rows_kernel<<<n_drafts + 1, clasp::smp::THREADS, 0, ctx->stream>>>(
+      logits_ws, draft_logits, tokens + (n - n_drafts), n_drafts, ctx->cfg.vocab, 1.0f / temperature,
+      (unsigned long long)seed, first, round, ctx->ws.spec);
+  if ((rc = launch_check(ctx))) return rc;
+  clasp::smp::spec_commit_kernel<<<1, 32, 0, ctx->stream>>>(ctx->ws.spec, tokens + (n - n_drafts), n_drafts,
+                                                            (unsigned long long)seed, first, round, n_accepted_out,
+                                                            committed_out);
+  return launch_check(ctx);
 }
 
 int clasp_accept(const int32_t* draft, const int32_t* full_argmax, int32_t K, int32_t* n_accepted,

@@ -180,6 +180,7 @@ struct Job {
   // head
   int32_t* argmax_out;
   float* top1_out;
+  float* logits_out;  // optional [R, vocab]: the head rows' logits (for sampling instead of arg-max)
 };
 
 struct Params {
@@ -1044,6 +1045,7 @@ struct Worker {
           const int r = cb * RB + k;
           if (r >= J.R) break;
           const float mine = fv ? v[k] * sh->rs[r] : -INFINITY;
+          if (J.logits_out && fv) __stcg(J.logits_out + (long long)r * c.vocab + f, mine);
           float best = mine;
           int bi = fv ? f : 0x7fffffff;
 #pragma unroll

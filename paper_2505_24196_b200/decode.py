@@ -145,3 +145,76 @@ def greedy_autoregressive(engine: Clasp, kv: KVCache, prompt: Sequence[int], n_n
         out.append(int(cur.cpu()[0]))
         pos += 1
     return out
+
+
+class SpeculativeSampler:
+    """Non-greedy self-speculative decoding (Table 1, temperature 1): drafts are draws of the
+    layer-skipped model, the verification accepts or replaces them by the rule of speculative
+    sampling (inside the library), the layer search runs on the last accepted position as in the
+    greedy loop.  Control flow only; all arithmetic and every random draw happen in libclasp.so."""
+
+    def __init__(self, engine: Clasp, kv: KVCache, M: int, K: int, temperature: float, seed: int, dp_interval: int = 1,
+                 fixed_mask: Optional[bytes] = None):
+        self.e, self.kv, self.M, self.K = engine, kv, M, K
+        self.temperature, self.seed, self.dp_interval, self.fixed_mask = float(temperature), int(seed), dp_interval, fixed_mask
+        dev = engine.device
+        L, d, V = engine.cfg.L, engine.cfg.d_model, engine.cfg.vocab
+        self.tok = torch.zeros(K + 1, dtype=torch.int32, device=dev)        # [pending, d_1..d_K]
+        self.q_logits = torch.empty((K, V), dtype=torch.float32, device=dev)
+        self.p_logits = torch.empty((K + 1, V), dtype=torch.float32, device=dev)
+        self.n_acc = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.committed = torch.zeros(K + 1, dtype=torch.int32, device=dev)
+        self.hidden = torch.empty((K + 1, L + 1, d), dtype=torch.float32, device=dev)
+        self.mask_host = bytes(L) if fixed_mask is None else bytes(fixed_mask)
+        self.rounds: List[Dict] = []
+        self.n_valid, self.pending, self.rnd = 0, None, 0
+
+    def _search(self, hidden_row: torch.Tensor, obj_pos: int):
+        if self.fixed_mask is not None or self.M == 0:
+            return
+        r = self.e.dp_search(hidden_row, self.e.cfg.d_model, 0, self.kv, obj_pos, obj_pos, 1, self.M,
+                             want_margins=False, want_g=False)
+        self.mask_host = bytes(r["S"].cpu().tolist())
+
+    def prefill(self, prompt: Sequence[int]) -> int:
+        e = self.e
+        toks = torch.as_tensor(list(prompt), dtype=torch.int32).to(e.device)
+        P, step = toks.numel(), e.cfg.max_rows
+        hid = None
+        for s in range(0, P, step):
+            chunk = toks[s:s + step]
+            if s + step >= P:
+                hid = torch.empty((chunk.numel(), e.cfg.L + 1, e.cfg.d_model), dtype=torch.float32, device=e.device)
+                e.verify_sample(chunk, s, self.kv, 0, None, self.temperature, self.seed, 0, self.p_logits, self.n_acc,
+                                self.committed, hid)
+            else:
+                e.verify(chunk, s, self.kv, 0, want_hidden=False)
+        first = int(self.committed.cpu()[0])
+        self.n_valid, self.pending = P, first
+        self._search(hid[-1], P - 1)
+        return first
+
+    def round(self) -> List[int]:
+        e, K = self.e, self.K
+        self.rnd += 1
+        self.tok[:1] = self.pending
+        for k in range(K):
+            e.draft_sample(self.mask_host, self.tok[k:k + 1], self.n_valid + k, self.kv, self.temperature, self.seed,
+                           self.rnd, self.tok[k + 1:k + 2], self.q_logits[k])
+        e.verify_sample(self.tok, self.n_valid, self.kv, K, self.q_logits, self.temperature, self.seed, self.rnd,
+                        self.p_logits, self.n_acc, self.committed, self.hidden)
+        a = int(self.n_acc.cpu()[0])
+        new = self.committed[:a + 1].cpu().tolist()
+        self.rounds.append({"accepted": a, "S": self.mask_host, "drafts": self.tok[1:].cpu().tolist(), "committed": new})
+        obj_pos = self.n_valid + a
+        self.n_valid += a + 1
+        self.pending = new[-1]
+        if self.rnd % self.dp_interval == 0:
+            self._search(self.hidden[a], obj_pos)
+        return new
+
+    def generate(self, prompt: Sequence[int], n_new: int) -> List[int]:
+        out = [self.prefill(prompt)]
+        while len(out) < n_new:
+            out.extend(self.round())
+        return out[:n_new]

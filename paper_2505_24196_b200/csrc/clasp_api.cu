@@ -58,8 +58,9 @@ struct Workspace {
   float* partial;
   // persistent layer engine
   void* xn_m;
-  float* e_att_acc;
-  float2* e_att_ml;
+  uint2* e_att_acc;
+  uint4* e_att_ml;
+  size_t e_att_bytes;
   long long* ss_a;
   long long* ss_m;
   size_t acc_bytes;
@@ -139,8 +140,11 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
     w.xn_m = take(R * d * 2);
     w.e_run_len = pk::ATT_KEYS * ((c.max_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32));
     w.e_chunk_cap = 32 + (int)((rcap + pk::ATT_KEYS - 1) / pk::ATT_KEYS);   // at most 32 runs of cache keys + own rows
-    w.e_att_acc = (float*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * c.head_dim * 4);
-    w.e_att_ml = (float2*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * sizeof(float2));
+    // partial attention outputs (two bf16 values + tag per 8 bytes) and their (maximum, tag, sum, tag): contiguous
+    w.e_att_acc = (uint2*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * c.head_dim * 4);
+    w.e_att_ml = (uint4*)take(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * sizeof(uint4));
+    w.e_att_bytes = (size_t)((uint8_t*)w.e_att_ml - (uint8_t*)w.e_att_acc) +
+                    align_up(rcap * c.n_q_heads * (size_t)w.e_chunk_cap * sizeof(uint4), 256);
     // fixed-point accumulators, zeroed before every launch: ss_a, ss_m, cosacc are contiguous
     const size_t ss_bytes = align_up(((size_t)c.L + 5) * rcap * sizeof(long long), 256);
     w.ss_a = (long long*)take(ss_bytes);
@@ -198,6 +202,7 @@ struct clasp_ctx {
   unsigned long long* e_trace = nullptr;
   int e_trace_cap = 0;
   uint32_t wait_limit = 0;   // 0: the kernels' default wait limits
+  uint32_t launch_seq = 0;   // launches of the persistent kernel so far (tags of the attention's partial results)
 };
 
 namespace {
@@ -683,7 +688,8 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   const clasp_config& c = ctx->cfg;
   Workspace& ws = ctx->ws;
   if (ctx->e_jobs.empty()) return CLASP_OK;
-  if (Rmax > pk::MAX_ROWS || (int)ctx->e_jobs.size() > c.L + 4) return CLASP_ERR_CAPACITY;
+  // (the job number is also the low 7 bits of the tags of the attention's partial results)
+  if (Rmax > pk::MAX_ROWS || (int)ctx->e_jobs.size() > c.L + 4 || ctx->e_jobs.size() > 127) return CLASP_ERR_CAPACITY;
   const int d = c.d_model, qd = c.n_q_heads * c.head_dim;
   const int rows_cap = c.max_rows;
   const int BN = Rmax <= 16 ? 16 : (Rmax + 15) / 16 * 16;
@@ -771,6 +777,12 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   P.b.rope = ws.rope;
   P.jobs = ws.jobs; P.n_jobs = (int)ctx->e_jobs.size(); P.wmaps = ws.wmaps; P.tabs = ws.tabs; P.ctl = ws.ctl;
   P.trace = ctx->e_trace; P.trace_cap = ctx->e_trace_cap;
+  ctx->launch_seq = (ctx->launch_seq + 1) & 0x1ffffffu;
+  if (ctx->launch_seq == 0) {   // the tags start over: no old tag may survive in the buffers
+    CUDA_TRY(cudaMemsetAsync(ws.e_att_acc, 0, ws.e_att_bytes, ctx->stream));
+    ctx->launch_seq = 1;
+  }
+  P.launch_tag = ctx->launch_seq << 7;
   P.wait_fast = ctx->wait_limit ? (ctx->wait_limit < pk::WAIT_FAST ? ctx->wait_limit : pk::WAIT_FAST) : pk::WAIT_FAST;
   P.wait_slow = ctx->wait_limit ? ctx->wait_limit : pk::WAIT_SLOW;
 
@@ -892,7 +904,8 @@ int clasp_create(const clasp_config* cfg, void* workspace, size_t workspace_byte
     return CLASP_ERR_CUDA;
   }
   if (ctx->use_tc) {
-    if (engine_setup(ctx) != CLASP_OK || cudaMemsetAsync(ws.ctl, 0, 256, ctx->stream) != cudaSuccess) {
+    if (engine_setup(ctx) != CLASP_OK || cudaMemsetAsync(ws.ctl, 0, 256, ctx->stream) != cudaSuccess ||
+        cudaMemsetAsync(ws.e_att_acc, 0, ws.e_att_bytes, ctx->stream) != cudaSuccess) {
       delete ctx;
       return CLASP_ERR_CUDA;
     }

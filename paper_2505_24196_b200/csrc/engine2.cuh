@@ -117,8 +117,8 @@ struct Bufs {
   float* qkv;      // [rows, qd + 2 kvd] projections (norm factor applied, not rotated)
   float* x1;       // [rows, d]    residual stream after attention
   float* Gbuf;     // [rows, d]    layer outputs of the candidate states (Eq. 2)
-  float* att_acc;  // [rows*nq, chunk_cap, hd]
-  float2* att_ml;  // [rows*nq, chunk_cap]
+  uint2* att_acc;  // [rows*nq, chunk_cap, hd / 2] partial attention outputs: (two bf16 values, tag) per 8 bytes
+  uint4* att_ml;   // [rows*nq, chunk_cap] (running maximum, tag, sum, tag)
   long long* ss_a; // [jobs, Rcap] row sums of squares of the operand of job j's first product (attention
                    // norm / head norm), summed over the CTAs in fixed point; zero at launch
   long long* ss_m; // [jobs, Rcap] same for the operand of job j's gate/up product (MLP norm)
@@ -193,6 +193,8 @@ struct Params {
   Ctl* ctl;
   unsigned long long* trace;  // optional [G, trace_cap] time stamps (ns)
   int trace_cap;
+  uint32_t launch_tag;        // (launch number << 7): with the job number, the tag that marks a partial attention result
+                              // as written by this job of this launch (never repeated over a context's life)
   uint32_t wait_fast;         // polls of a wait before it starts to sleep between polls
   uint32_t wait_slow;         // further polls (about 100 ns apart) before the wait gives up
 };
@@ -1313,6 +1315,7 @@ struct Worker {
     const int qkvd = c.qd + 2 * c.kvd;
     const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;
     const RowDiv rdT(J.T);
+    const uint32_t tag = p.launch_tag | (uint32_t)(jb + 1);
     // The cache does not depend on this layer's projections: the first K/V tile of this CTA's first
     // item is on its way from HBM while the CTA waits for them.
     constexpr int FILL = ATT_KEYS * (HD / 8) / WORKERS;   // 16-byte pieces of a tile per thread
@@ -1554,92 +1557,90 @@ struct Worker {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           if (!pv[h]) continue;
+          // Every 8-byte store carries its own tag, so the merge needs no flag and no fence: it reads the
+          // partial results themselves until every piece shows this job's tag (8-byte accesses are single
+          // copies).  Values as bf16: the merged row is rounded to bf16 for the o product anyway.
           const long long idx = ((long long)rr[h] * c.nq + hq[h]) * c.chunk_cap + chunk;
-          float* pa = p.b.att_acc + idx * HD + c4 * 2;
+          uint2* pa = p.b.att_acc + idx * (HD / 2) + c4;
 #pragma unroll
-          for (int nb = 0; nb < NBLK; ++nb)
-            __stcg(reinterpret_cast<float2*>(pa + nb * 8), make_float2(o[nb][2 * h], o[nb][2 * h + 1]));
-          if (c4 == 0) __stcg(p.b.att_ml + idx, make_float2(m[h], l[h]));
+          for (int nb = 0; nb < NBLK; ++nb) __stcg(pa + nb * 4, make_uint2(pack2(o[nb][2 * h], o[nb][2 * h + 1]), tag));
+          if (c4 == 0) __stcg(p.b.att_ml + idx, make_uint4(__float_as_uint(m[h]), tag, __float_as_uint(l[h]), tag));
         }
       }
     }
-    publish(F_ATTN, jb + 1);
     return true;
   }
 
-  // all chunks of query head h merged, one warp per row; head h is merged by CTA h % G
+  // All chunks of a (row, query head) pair merged by one warp; the pairs are dealt out to all CTAs and,
+  // inside a CTA, to its warps.  There is no flag to wait for: the warp reads the partial results until
+  // every piece carries this job's tag (see attention_partials), one trip to L2 when they are there.
   __device__ bool attention_merge(const Job& J, int jb) {
-    constexpr int DPL = HD / 32;   // head dimensions per lane
+    constexpr int LANES = HD / 4;    // lanes that hold four head dimensions each
+    constexpr int MB = 17;           // partials fetched per trip to L2 (a 512-key context has 17)
     const Cfg& c = p.c;
-    const int Gq = c.nq / c.nkv;
-    const int n_pbg = (J.R * Gq + 127) / 128;
     const int k_tot = J.uniform ? J.C + J.T : J.C;
     const int n_runs = (k_tot + c.run_len - 1) / c.run_len;
     const int n_chunks = n_runs + (J.uniform ? 0 : (J.R + ATT_KEYS - 1) / ATT_KEYS);
-    // One warp per (row, head) pair; the pairs are dealt out to all CTAs and, inside a CTA, to its warps.
+    const uint32_t tag = p.launch_tag | (uint32_t)(jb + 1);
+    const uint32_t n_poll = 2u * sh->wait_slow;
     bool all_ok = true;
     for (int u = (int)blockIdx.x + c.G * ww; u < J.R * c.nq; u += c.G * 8) {
-      const int r = u / c.nq, hq = u - r * c.nq;
-      {
-        // the items of this head's kv head ran on CTAs (item index) % G
-        const int kvh = hq / Gq;
-        const int it0 = kvh * n_chunks * n_pbg, n_it = n_chunks * n_pbg;
+      const long long pr = u;        // = row * nq + query head
+      const uint4* ml = p.b.att_ml + pr * c.chunk_cap;
+      const uint4* acc = reinterpret_cast<const uint4*>(p.b.att_acc + pr * c.chunk_cap * (HD / 2)) + lane;
+      uint4 v0, v1, a[MB];
+      // one trip: maxima / sums of all chunks and the first MB partial outputs; repeated until all are tagged
+      auto load_trip = [&](int ch0, bool with_ml) -> bool {
         bool ok = true;
-        for (int k = lane; k < min(n_it, c.G); k += 32)
-          ok = wait_flag(p.b.flags + F_ATTN * c.G + (it0 + k) % c.G, jb + 1, p.ctl, sh) && ok;
-        if (!__all_sync(0xffffffffu, ok)) { all_ok = false; break; }
-        const long long pr = (long long)r * c.nq + hq;
-        const float2* ml = p.b.att_ml + pr * c.chunk_cap;
-        float2 v0 = make_float2(-INFINITY, 0.f), v1 = v0;
-        if (lane < n_chunks) v0 = __ldcg(ml + lane);
-        if (lane + 32 < n_chunks) v1 = __ldcg(ml + lane + 32);
-        constexpr int MB = 17;   // partials fetched per trip to L2 (a 512-key context has 17)
-        const float* acc = p.b.att_acc + pr * c.chunk_cap * HD + lane * DPL;
-        float a[MB][DPL];
-        auto load_trip = [&](int ch0) {
-#pragma unroll
-          for (int e = 0; e < MB; ++e) {
-#pragma unroll
-            for (int k = 0; k < DPL; ++k) a[e][k] = 0.f;
-            if (ch0 + e < n_chunks) {
-              if (DPL == 4) {
-                const float4 t = __ldcg(reinterpret_cast<const float4*>(acc + (long long)(ch0 + e) * HD));
-                a[e][0] = t.x; a[e][1] = t.y; a[e][2] = t.z; a[e][3] = t.w;
-              } else {
-                const float2 t = __ldcg(reinterpret_cast<const float2*>(acc + (long long)(ch0 + e) * HD));
-                a[e][0] = t.x; a[e][1] = t.y;
-              }
-            }
-          }
-        };
-        load_trip(0);   // in the same trip to L2 as the maxima and sums: the partials do not depend on them
-        const float mx = warp_max(fmaxf(v0.x, v1.x));
-        const float w0 = v0.x == -INFINITY ? 0.f : exp2f(v0.x - mx);
-        const float w1 = v1.x == -INFINITY ? 0.f : exp2f(v1.x - mx);
-        const float den = warp_sum(w0 * v0.y + w1 * v1.y);
-        float num[DPL];
-#pragma unroll
-        for (int k = 0; k < DPL; ++k) num[k] = 0.f;
-        for (int ch0 = 0; ch0 < n_chunks; ch0 += MB) {
-          if (ch0 > 0) load_trip(ch0);
-#pragma unroll
-          for (int e = 0; e < MB; ++e) {
-            const int ch = ch0 + e;
-            const float wa = __shfl_sync(0xffffffffu, w0, ch & 31), wb = __shfl_sync(0xffffffffu, w1, ch & 31);
-            const float w = ch < 32 ? wa : wb;
-#pragma unroll
-            for (int k = 0; k < DPL; ++k) num[k] = fmaf(w, a[e][k], num[k]);
-          }
+        if (with_ml) {
+          v0 = v1 = make_uint4(0xff800000u, tag, 0u, tag);   // (-inf, 0)
+          if (lane < n_chunks) v0 = __ldcg(ml + lane);
+          if (lane + 32 < n_chunks) v1 = __ldcg(ml + lane + 32);
         }
-        bf16* dst = p.b.attn + pr * HD + lane * DPL;
-        const float inv = 1.0f / den;
-        if (DPL == 4) {
-          *reinterpret_cast<uint2*>(dst) = pack4(num[0] * inv, num[1] * inv, num[2] * inv, num[DPL - 1] * inv);
-        } else {
-          __nv_bfloat162 t = __floats2bfloat162_rn(num[0] * inv, num[1] * inv);
-          *reinterpret_cast<__nv_bfloat162*>(dst) = t;
+#pragma unroll
+        for (int e = 0; e < MB; ++e) {
+          a[e] = make_uint4(0u, tag, 0u, tag);
+          if (ch0 + e < n_chunks && lane < LANES) a[e] = __ldcg(acc + (long long)(ch0 + e) * LANES);
+        }
+        if (with_ml) ok = v0.y == tag && v0.w == tag && v1.y == tag && v1.w == tag;
+#pragma unroll
+        for (int e = 0; e < MB; ++e) ok = ok && a[e].y == tag && a[e].w == tag;
+        return __all_sync(0xffffffffu, ok);
+      };
+      auto poll_trip = [&](int ch0, bool with_ml) -> bool {
+        for (uint32_t it = 0; it < n_poll; ++it) {
+          if (load_trip(ch0, with_ml)) return true;
+          if ((it & 15u) == 15u && aborted(p.ctl, sh)) return false;
+          __nanosleep(POLL_NS);
+        }
+        raise_abort(p.ctl, sh, true);
+        return false;
+      };
+      if (!poll_trip(0, true)) { all_ok = false; break; }
+      const float m0 = __uint_as_float(v0.x), m1 = __uint_as_float(v1.x);
+      const float mx = warp_max(fmaxf(m0, m1));
+      const float w0 = m0 == -INFINITY ? 0.f : exp2f(m0 - mx);
+      const float w1 = m1 == -INFINITY ? 0.f : exp2f(m1 - mx);
+      const float den = warp_sum(w0 * __uint_as_float(v0.z) + w1 * __uint_as_float(v1.z));
+      float num[4] = {0.f, 0.f, 0.f, 0.f};
+      bool ok = true;
+      for (int ch0 = 0; ch0 < n_chunks; ch0 += MB) {
+        if (ch0 > 0 && !poll_trip(ch0, false)) { ok = false; break; }
+#pragma unroll
+        for (int e = 0; e < MB; ++e) {
+          const int ch = ch0 + e;
+          const float wa = __shfl_sync(0xffffffffu, w0, ch & 31), wb = __shfl_sync(0xffffffffu, w1, ch & 31);
+          const float w = ch < 32 ? wa : wb;
+          const float2 d01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a[e].x));
+          const float2 d23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a[e].z));
+          num[0] = fmaf(w, d01.x, num[0]); num[1] = fmaf(w, d01.y, num[1]);
+          num[2] = fmaf(w, d23.x, num[2]); num[3] = fmaf(w, d23.y, num[3]);
         }
       }
+      if (!ok) { all_ok = false; break; }
+      const float inv = 1.0f / den;
+      if (lane < LANES)
+        *reinterpret_cast<uint2*>(p.b.attn + pr * HD + lane * 4) = pack4(num[0] * inv, num[1] * inv, num[2] * inv, num[3] * inv);
     }
     if (!worker_and(all_ok)) return false;
     publish(F_MERGE, jb + 1);

@@ -1477,17 +1477,22 @@ struct Worker {
         if (!own && key0 + ATT_KEYS < key_hi) load_cache_tile(key0 + ATT_KEYS);   // in flight during the tile's math
         worker_sync();
         if (!active) continue;
+        // S = Q K^T.  The multiplies are issued in program order (volatile asm): the k-step is the outer loop,
+        // so that four independent accumulators alternate instead of eight dependent multiplies in a row.
         float s[4][4];
 #pragma unroll
-        for (int nb = 0; nb < 4; ++nb) {
-          s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
-          const bf16* kr = k_s + (nb * 8 + g8) * LD + c4 * 2;
+        for (int nb = 0; nb < 4; ++nb) s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
 #pragma unroll
-          for (int ks = 0; ks < KS; ++ks) {
-            const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kr + ks * 16);
-            const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kr + ks * 16 + 8);
-            mma_16816(s[nb], qh[ks], b0, b1);
+        for (int ks = 0; ks < KS; ++ks) {
+          uint32_t b0[4], b1[4];
+#pragma unroll
+          for (int nb = 0; nb < 4; ++nb) {
+            const bf16* kr = k_s + (nb * 8 + g8) * LD + c4 * 2 + ks * 16;
+            b0[nb] = *reinterpret_cast<const uint32_t*>(kr);
+            b1[nb] = *reinterpret_cast<const uint32_t*>(kr + 8);
           }
+#pragma unroll
+          for (int nb = 0; nb < 4; ++nb) mma_16816(s[nb], qh[ks], b0[nb], b1[nb]);
         }
         float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
@@ -1544,11 +1549,16 @@ struct Worker {
           const int mrow = k2 * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
           const int mcol = (lane >> 4) * 8;
 #pragma unroll
-          for (int nb = 0; nb < NBLK; nb += 2) {
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(tc::smem_u32(v_s + mrow * LD + nb * 8 + mcol), b0, b1, b2, b3);
-            mma_16816(o[nb], ph, b0, b1);
-            mma_16816(o[nb + 1], ph, b2, b3);
+          for (int nb = 0; nb < NBLK; nb += 8) {   // four fragment loads in flight, then their eight multiplies
+            uint32_t vb[4][4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              ldmatrix_x4_trans(tc::smem_u32(v_s + mrow * LD + (nb + 2 * q) * 8 + mcol), vb[q][0], vb[q][1], vb[q][2], vb[q][3]);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              mma_16816(o[nb + 2 * q], ph, vb[q][0], vb[q][1]);
+              mma_16816(o[nb + 2 * q + 1], ph, vb[q][2], vb[q][3]);
+            }
           }
         }
       }

@@ -76,6 +76,7 @@ def test_layer_rows_against_oracle(full):
     """Twelve independent states through one layer over a 512-position cache (what one step of the
     search launches); rows 0, 5 and 11 are recomputed by the oracle."""
     cfg = full.cfg
+    assert full.engine.engine_active()      # this shape runs in the one-launch-per-call kernel, not its fall-back
     x = datagen.normal_rows(53, 0, (12, cfg.d_model)).to(torch.float32)
     out = full.engine.layer_forward(SAMPLED_LAYER, x.cuda(), 12, 1, C0, C0, full.kv).cpu().numpy()
     for r in (0, 5, 11):

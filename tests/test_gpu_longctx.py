@@ -56,6 +56,7 @@ def mlong():
 
 def test_layer_rows_over_a_long_context(mlong):
     cfg = mlong.cfg
+    assert mlong.engine.engine_active()
     x = datagen.normal_rows(72, 0, (12, cfg.d_model)).to(torch.float32)
     out = mlong.engine.layer_forward(1, x.cuda(), 12, 1, C0, C0, mlong.kv).cpu().numpy()
     w = mlong.oracle.layer(1)

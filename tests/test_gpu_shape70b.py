@@ -56,6 +56,7 @@ def m70():
 
 def test_layer_rows_on_the_70b_shape(m70):
     cfg = m70.cfg
+    assert m70.engine.engine_active()      # this shape runs in the one-launch-per-call kernel, not its fall-back
     x = datagen.normal_rows(62, 0, (40, cfg.d_model)).to(torch.float32)
     out = m70.engine.layer_forward(1, x.cuda(), 40, 1, C0, C0, m70.kv).cpu().numpy()
     w = m70.oracle.layer(1)

@@ -17,7 +17,7 @@ from . import build as _build
 
 CLASP_FP32, CLASP_BF16 = 0, 1
 CHOICE_APPLY, CHOICE_SKIP, CHOICE_NONE = 0, 1, 255
-FLAG_FORCE_SIMT, FLAG_NO_DEFER, FLAG_MULTI_KERNEL, FLAG_PRUNE = 1, 2, 4, 8
+FLAG_FORCE_SIMT, FLAG_NO_DEFER, FLAG_MULTI_KERNEL, FLAG_PRUNE, FLAG_NO_ATT_TC = 1, 2, 4, 8, 16
 
 SYMBOLS = ["clasp_workspace_bytes", "clasp_create", "clasp_destroy", "clasp_load_layers", "clasp_load_head",
            "clasp_dp_search", "clasp_verify", "clasp_draft_forward", "clasp_accept", "clasp_layer_forward",

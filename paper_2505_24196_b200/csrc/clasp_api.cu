@@ -70,6 +70,7 @@ struct Workspace {
   int* flags;
   clasp::pk::Ctl* ctl;
   CUtensorMap* wmaps;
+  CUtensorMap* kvmaps;   // tensor-core attention: key and value cache maps of each layer job of the launch
   clasp::pk::Job* jobs;
   int* tabs;
   clasp::smp::AcceptScratch* spec;
@@ -156,6 +157,7 @@ Workspace carve(const clasp_config& c, uint8_t* base) {
     w.flags = (int*)take(pk::N_FLAGS * (G + 32) * sizeof(int));
     w.ctl = (pk::Ctl*)take(256);
     w.wmaps = (CUtensorMap*)take(((size_t)c.L * 7 + 1) * pk::N_HEIGHTS * 2 * sizeof(CUtensorMap));
+    w.kvmaps = (CUtensorMap*)take(((size_t)c.L + 4) * 2 * sizeof(CUtensorMap));
     w.jobs = (pk::Job*)take(((size_t)c.L + 4) * sizeof(pk::Job));
     w.tabs = (int*)take(ENGINE_TAB_INTS * sizeof(int));
   }
@@ -190,11 +192,13 @@ struct clasp_ctx {
   bool use_engine = false;
   int e_G = 0;              // CTAs of the cooperative grid (one per SM)
   int e_static_smem = 0;
-  const void* e_kernel[2] = {nullptr, nullptr};   // the layer kernel for this head dimension: plain, with step stamps
+  const void* e_kernel[4] = {nullptr, nullptr, nullptr, nullptr};   // the layer kernel for this head dimension: plain, with step
+                                                                    // stamps; [2], [3]: the same with the tensor-core attention
   int e_split_lo[clasp::pk::N_SPLITS], e_split_units[clasp::pk::N_SPLITS], e_tile_idx[5], e_tiles_off = 0,
       e_kpi[5], e_use3d[5], e_wpages[5];
   int e_heights[8][clasp::pk::N_HEIGHTS];   // tile heights per matrix slot (wq wk wv wo gate up down head)
   std::vector<CUtensorMap> e_wmaps_host;
+  std::vector<CUtensorMap> e_kvmaps_host;
   bool e_wmaps_dirty = true;
   std::map<int, std::array<CUtensorMap, 10>> e_bmaps;          // by BN: 2-D maps of the four operands, then 3-D, then xn with 2 BN rows (2-D, 3-D)
   std::map<std::pair<int, int>, std::array<CUtensorMap, 2>> e_headmaps;  // by (row offset, BN): 2-D, 3-D
@@ -550,17 +554,20 @@ int engine_setup(clasp_ctx* ctx) {
   const int d = c.d_model, qd = c.n_q_heads * c.head_dim, kvd = c.n_kv_heads * c.head_dim;
   if (d % 8 || c.d_ffn % 8 || c.vocab % 8) return CLASP_OK;
   // the instantiations for this model's head dimension, without and with step stamps
-  ctx->e_kernel[0] = c.head_dim == 128 ? (const void*)pk::engine_kernel<false, 128> : (const void*)pk::engine_kernel<false, 64>;
-  ctx->e_kernel[1] = c.head_dim == 128 ? (const void*)pk::engine_kernel<true, 128> : (const void*)pk::engine_kernel<true, 64>;
+  ctx->e_kernel[0] = c.head_dim == 128 ? (const void*)pk::engine_kernel<false, 128, false> : (const void*)pk::engine_kernel<false, 64, false>;
+  ctx->e_kernel[1] = c.head_dim == 128 ? (const void*)pk::engine_kernel<true, 128, false> : (const void*)pk::engine_kernel<true, 64, false>;
+  ctx->e_kernel[2] = c.head_dim == 128 ? (const void*)pk::engine_kernel<false, 128, true> : nullptr;
+  ctx->e_kernel[3] = c.head_dim == 128 ? (const void*)pk::engine_kernel<true, 128, true> : nullptr;
+  const int n_kern = c.head_dim == 128 ? 4 : 2;
   ctx->e_static_smem = 0;
-  for (int k = 0; k < 2; ++k) {  // one shared-memory budget for both
+  for (int k = 0; k < n_kern; ++k) {  // one shared-memory budget for both
     cudaFuncAttributes fa;
     CUDA_TRY(cudaFuncGetAttributes(&fa, ctx->e_kernel[k]));
     if ((int)fa.sharedSizeBytes > ctx->e_static_smem) ctx->e_static_smem = (int)fa.sharedSizeBytes;
   }
   const int dyn_max = optin - ctx->e_static_smem;
   if (dyn_max < 1024 + 64 * pk::PAGE + pk::SCRATCH_BYTES) return CLASP_OK;
-  for (int k = 0; k < 2; ++k)
+  for (int k = 0; k < n_kern; ++k)
     CUDA_TRY(cudaFuncSetAttribute(ctx->e_kernel[k], cudaFuncAttributeMaxDynamicSharedMemorySize, dyn_max));
   int G = ctx->num_sms;
   if (G > ENGINE_MAX_CTAS) G = ENGINE_MAX_CTAS;
@@ -696,7 +703,17 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   int dev = 0, optin = 0;
   CUDA_TRY(cudaGetDevice(&dev));
   CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-  const int ring_pages = (optin - ctx->e_static_smem - 1024 - pk::SCRATCH_BYTES) / pk::PAGE;
+  // Searches over a long context run the attention over the cache keys on the tensor cores: that needs a
+  // larger scratch area (taken from the weight ring) and runs of whole 64-key tiles.
+  // (measured on the 8B shape: it pays from about 4096 positions on, and from about 2048 when a kv head has 256 or more
+  // (row, query head) pairs; below that the smaller ring costs the products more than the attention gains)
+  const int att_pairs = Rmax * (c.n_q_heads / c.n_kv_heads);
+  const bool att_tc = c.head_dim == 128 && !(c.flags & CLASP_FLAG_NO_ATT_TC) &&
+                      (search_ctx >= pk::TC_MIN_CTX || (search_ctx >= pk::TC_MIN_CTX / 2 && att_pairs >= 256));
+  // (row, query head) pairs of a kv head: up to 64 of them fit an M = 64 accumulator, which leaves the ring 24 KB more
+  const int att_rows = att_pairs <= 64 ? 64 : pk::TC_ROWS;
+  const int scratch_bytes = !att_tc ? pk::SCRATCH_BYTES : (att_rows == 64 ? pk::SCRATCH_TC64_BYTES : pk::SCRATCH_TC_BYTES);
+  const int ring_pages = (optin - ctx->e_static_smem - 1024 - scratch_bytes) / pk::PAGE;
   // an item (gate + up rows and the operand tiles of kpi chunks) must fit the ring twice over
   const int b_pages = BN * pk::BK * 2 / pk::PAGE;
   // chunks per ring item in this launch: the set-up value when two such items fit the ring, else fewer,
@@ -713,7 +730,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
     if (kpi[k] != ctx->e_kpi[k]) use3d[k] = 0;
     if (!use3d[k] && kpi[k] > 16) kpi[k] = 16;   // one lane pair per chunk
   }
-  const size_t dyn = 1024 + (size_t)ring_pages * pk::PAGE + pk::SCRATCH_BYTES;
+  const size_t dyn = 1024 + (size_t)ring_pages * pk::PAGE + scratch_bytes;
 
   const int qdim = qd;
   auto bm = ctx->e_bmaps.find(BN);
@@ -750,6 +767,21 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
                              cudaMemcpyHostToDevice, ctx->stream));
     ctx->e_wmaps_dirty = false;
   }
+  if (att_tc) {
+    // the caches of this launch's layer jobs as 2-D maps {kv width, context rows}: 64 x 64 boxes, 128-byte swizzle,
+    // rows past the context read as zeros
+    ctx->e_kvmaps_host.assign(ctx->e_jobs.size() * 2, CUtensorMap{});
+    for (size_t j = 0; j < ctx->e_jobs.size(); ++j) {
+      pk::Job& J = ctx->e_jobs[j];
+      if (J.type != pk::JOB_LAYER || J.uniform) continue;
+      J.kvmap = (int)(2 * j);
+      if (make_map(ctx, J.ck, J.C, c.n_kv_heads * c.head_dim, 64, &ctx->e_kvmaps_host[2 * j]) ||
+          make_map(ctx, J.cv, J.C, c.n_kv_heads * c.head_dim, 64, &ctx->e_kvmaps_host[2 * j + 1]))
+        return CLASP_ERR_CUDA;
+    }
+    CUDA_TRY(cudaMemcpyAsync(ws.kvmaps, ctx->e_kvmaps_host.data(), ctx->e_kvmaps_host.size() * sizeof(CUtensorMap),
+                             cudaMemcpyHostToDevice, ctx->stream));
+  }
   CUDA_TRY(cudaMemcpyAsync(ws.jobs, ctx->e_jobs.data(), ctx->e_jobs.size() * sizeof(pk::Job),
                            cudaMemcpyHostToDevice, ctx->stream));
   CUDA_TRY(cudaMemsetAsync(ws.ctl, 0, 4, ctx->stream));  // abort flag; the status word is sticky
@@ -766,7 +798,22 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   // the keys it sees into at most 32 runs, which spreads a short context over many more CTAs.
   if (search_ctx >= 0) P.c.run_len = pk::ATT_KEYS * ((search_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32) > 0
                                                        ? (search_ctx + pk::ATT_KEYS * 32 - 1) / (pk::ATT_KEYS * 32) : 1);
-  P.c.BN = BN; P.c.ring_pages = ring_pages;
+  if (att_tc) {
+    // run length: whole 64-key tiles, at most 32 runs; the cut that needs the fewest tile steps when the
+    // (kv head, run, pair block) items are dealt out to the CTAs (one more step per round for its set-up)
+    const int n_pb = (Rmax * (c.n_q_heads / c.n_kv_heads) + att_rows - 1) / att_rows;
+    int best_len = 0;
+    long best_cost = 0;
+    for (int n = 1; n <= 32; ++n) {
+      const int len = 64 * (((search_ctx + n - 1) / n + 63) / 64);
+      const int runs = (search_ctx + len - 1) / len;
+      const long rounds = ((long)c.n_kv_heads * runs * n_pb + ctx->e_G - 1) / ctx->e_G;
+      const long cost = rounds * (len / 64 + 1);
+      if (best_len == 0 || cost < best_cost) { best_len = len; best_cost = cost; }
+    }
+    P.c.run_len = best_len;
+  }
+  P.c.BN = BN; P.c.ring_pages = ring_pages; P.c.att_tc = att_tc ? 1 : 0; P.c.att_rows = att_rows;
 
   for (int s = 0; s < pk::N_SPLITS; ++s) { P.c.split_lo[s] = ctx->e_split_lo[s]; P.c.split_units[s] = ctx->e_split_units[s]; }
   for (int k = 0; k < 5; ++k) { P.c.tile_idx[k] = ctx->e_tile_idx[k]; P.c.kpi[k] = kpi[k]; P.c.use3d[k] = use3d[k]; }
@@ -775,7 +822,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   P.b.qkv = ws.qkv; P.b.x1 = ws.x1; P.b.Gbuf = ws.G; P.b.att_acc = ws.e_att_acc; P.b.att_ml = ws.e_att_ml;
   P.b.ss_a = ws.ss_a; P.b.ss_m = ws.ss_m; P.b.cosacc = ws.cosacc; P.b.head_best = ws.head_best; P.b.flags = ws.flags;
   P.b.rope = ws.rope;
-  P.jobs = ws.jobs; P.n_jobs = (int)ctx->e_jobs.size(); P.wmaps = ws.wmaps; P.tabs = ws.tabs; P.ctl = ws.ctl;
+  P.jobs = ws.jobs; P.n_jobs = (int)ctx->e_jobs.size(); P.wmaps = ws.wmaps; P.kvmaps = ws.kvmaps; P.tabs = ws.tabs; P.ctl = ws.ctl;
   P.trace = ctx->e_trace; P.trace_cap = ctx->e_trace_cap;
   ctx->launch_seq = (ctx->launch_seq + 1) & 0x1ffffffu;
   if (ctx->launch_seq == 0) {   // the tags start over: no old tag may survive in the buffers
@@ -794,7 +841,7 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   void* args[] = {(void*)&bm->second[0], (void*)&bm->second[1], (void*)&bm->second[2], (void*)&bm->second[3],
                   (void*)&hm->second[0], (void*)&bm->second[4], (void*)&bm->second[5], (void*)&bm->second[6],
                   (void*)&bm->second[7], (void*)&hm->second[1], (void*)&bm->second[8], (void*)&bm->second[9], (void*)&P};
-  const void* kern = ctx->e_kernel[ctx->e_trace ? 1 : 0];
+  const void* kern = ctx->e_kernel[(att_tc ? 2 : 0) + (ctx->e_trace ? 1 : 0)];
   cudaError_t err = cudaLaunchCooperativeKernel(kern, dim3(ctx->e_G), dim3(pk::THREADS),
                                                 args, dyn, ctx->stream);
   if (ctx->profiling) {

@@ -55,6 +55,10 @@ constexpr int WORKER_T0 = 128;
 constexpr int NB = 32;                // items in flight (mbarrier pairs)
 constexpr int ATT_KEYS = 32;
 constexpr int SCRATCH_BYTES = 2 * ATT_KEYS * 136 * 2 + 2048;  // two padded K/V tiles + slack (>= 16 KB guard)
+constexpr int TC_MIN_CTX = 4000;              // search contexts from here on take the tensor-core attention (half of it with many rows)
+constexpr int TC_ROWS = 128;                  // (row, query head) pairs of one tensor-core attention item
+constexpr int SCRATCH_TC64_BYTES = 57 * 1024; // the same with 64 rows per item: q tile 16 KB, P tile 8 KB
+constexpr int SCRATCH_TC_BYTES = 81 * 1024;   // q tile 32 KB, K, V and P tiles 16 KB each (1024-aligned), 1 KB of per-row words
 constexpr int MAX_ROWS = 128;         // rows one launch may push through a layer
 // Rows (accumulator columns) a worker group finishes per pass; the two groups of four warps take alternate
 // blocks.  4 or 8: with 4 the unrolled per-row code is half as long and 5 to 8 rows already keep both groups
@@ -98,6 +102,9 @@ struct Cfg {
   int run_len, chunk_cap;
   int BN;              // activation rows padded to a multiple of 16 (MMA N)
   int ring_pages;
+  int att_rows;        // tensor-core attention: (row, query head) pairs per item, 64 or 128
+  int att_tc;          // 1: search jobs run the attention over their cache keys on tcgen05 (kernel instantiation with
+                       // TC set; the launch carries SCRATCH_TC_BYTES of worker scratch instead of SCRATCH_BYTES)
   // tables (ints / structs in Params::tabs, offsets in ints)
   int split_lo[N_SPLITS];    // [G + 1] first feature of each CTA: lo(c) = 8 floor(c units / G)
   int split_units[N_SPLITS]; // 8-feature units of each split
@@ -148,6 +155,7 @@ struct Job {
                  // down epilogue), rows [BN, 2 BN) the skip candidates -- and its epilogue keeps the chosen one
   int dual_src;  // 1: this job's q/k/v operand has those two row blocks (the previous job has `defer`)
   int row_off;   // JOB_HEAD: first row (of the previous job's rows) that goes through the head
+  int kvmap;     // tensor-core attention: index in Params::kvmaps of the tensor map of this layer's key cache (values: + 1)
   int in_shift;  // first row of the previous job's operand rows / decisions that is this job's row 0 (a search that
                  // leaves out unreachable states drops leading states from one step to the next)
   int src_flag;  // step kind that publishes this job's first operand (F_PREP / F_DOWN / F_SELECT)
@@ -189,6 +197,7 @@ struct Params {
   const Job* jobs;
   int n_jobs;
   const CUtensorMap* wmaps;  // [(L*7 + 1) * N_HEIGHTS] 2-D maps, then as many 3-D maps
+  const CUtensorMap* kvmaps; // tensor-core attention: per layer job, 2-D maps {kv width, context rows} of the key and value cache
   const int* tabs;
   Ctl* ctl;
   unsigned long long* trace;  // optional [G, trace_cap] time stamps (ns)
@@ -227,6 +236,18 @@ __device__ __forceinline__ bool worker_and(bool ok) {
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(r)
       : "r"((uint32_t)ok)
+      : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ bool worker_or(bool v) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "barrier.cta.red.or.pred p, 1, 256, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)v)
       : "memory");
   return r != 0;
 }
@@ -327,6 +348,8 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 struct Shared {
   uint64_t full[NB], empty[NB];
   uint64_t acc_full[2], acc_empty[2];
+  uint64_t att_bar;         // completion of the attention's own tcgen05 multiplies
+  uint64_t att_k_bar, att_v_bar;   // arrival of the attention's K / V tile
   uint32_t tmem_base;
   volatile int abort;
   uint32_t wait_fast, wait_slow;   // the launch's wait limits
@@ -729,8 +752,8 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
 // ------------------------------------------------------------------ worker steps
 // TR: the step stamps are compiled in; HD: the model's head dimension (64 or 128).  The kernel is
 // sensitive to its code size, so an instantiation carries neither stamps it does not take nor the
-// attention code of the other head dimension.
-template <bool TR, int HD>
+// attention code of the other head dimension; TC: with the tensor-core attention of long-context searches.
+template <bool TR, int HD, bool TC>
 struct Worker {
   const Params& p;
   Shared* sh;
@@ -739,6 +762,8 @@ struct Worker {
   int wtid, ww, lane;
   uint32_t n_acc;
   int n_mark;
+  uint32_t att_phase = 0;   // parity of att_bar's next completion
+  uint32_t att_kph = 0, att_vph = 0;   // the same for the K / V tile barriers (worker warp 4)
 
   // time stamp of step `slot` (one of the T_* above) of the current job
   __device__ __forceinline__ void mark(int slot) {
@@ -1294,6 +1319,9 @@ struct Worker {
   // ---- attention: partial softmax over one run of cache keys or one chunk of own rows.
   // q, k, v of the rows come from the projection buffer (norm factor applied, not rotated): they
   // are rotated here; new keys / values are rounded to the cache type before use.
+  // OWN_ONLY: the caller has already dealt with the runs of cache keys (attention_tc) and waited for the
+  // projections; only the chunks of the rows' own keys are left, dealt out from the last CTA downwards.
+  template <bool OWN_ONLY = false>
   __device__ bool attention_partials(const Job& J, int jb) {
     const Cfg& c = p.c;
     constexpr int KS = HD / 16;
@@ -1309,7 +1337,8 @@ struct Worker {
     const int n_runs = (k_tot + c.run_len - 1) / c.run_len;
     const int n_own = J.uniform ? 0 : (J.R + ATT_KEYS - 1) / ATT_KEYS;
     const int n_chunks = n_runs + n_own;
-    const int n_items = c.nkv * n_chunks * n_pbg;
+    const int n_ch = OWN_ONLY ? n_own : n_chunks;   // chunks this call deals out
+    const int n_items = c.nkv * n_ch * n_pbg;
     const int g8 = lane >> 2, c4 = lane & 3;
     const long long kvld = c.kvd;
     const int qkvd = c.qd + 2 * c.kvd;
@@ -1322,7 +1351,7 @@ struct Worker {
     static_assert(FILL * WORKERS == ATT_KEYS * (HD / 8), "tile pieces must divide among the workers");
     uint4 pre_k[FILL], pre_v[FILL];
     bool pre_ok = false;
-    if ((int)blockIdx.x < n_items) {
+    if (!OWN_ONLY && (int)blockIdx.x < n_items) {
       const int chunk = ((int)blockIdx.x / n_pbg) % n_chunks;
       const int kvh = (int)blockIdx.x / (n_pbg * n_chunks);
       if (chunk < n_runs) {
@@ -1342,12 +1371,14 @@ struct Worker {
       }
     }
     // every row's q, k, v exist once all CTAs have published their slice of the projections
-    if (!wait_all(F_QKV, J.tgt[F_QKV])) return false;
-    mark(T_ATT_READY);
-    for (int it = blockIdx.x; it < n_items; it += c.G) {
+    if (!OWN_ONLY) {
+      if (!wait_all(F_QKV, J.tgt[F_QKV])) return false;
+      mark(T_ATT_READY);
+    }
+    for (int it = OWN_ONLY ? c.G - 1 - (int)blockIdx.x : (int)blockIdx.x; it < n_items; it += c.G) {
       const int pbg = it % n_pbg;
-      const int chunk = (it / n_pbg) % n_chunks;
-      const int kvh = it / (n_pbg * n_chunks);
+      const int chunk = (OWN_ONLY ? n_runs : 0) + (it / n_pbg) % n_ch;
+      const int kvh = it / (n_pbg * n_ch);
       const bool own = chunk >= n_runs;
       const int p0 = (pbg * 8 + ww) * 16;
       const bool active = p0 < Pn;
@@ -1581,6 +1612,335 @@ struct Worker {
     return true;
   }
 
+  // 16 accumulator columns of this thread's lane: write (the read is tc::tmem_ld16)
+  __device__ __forceinline__ static void tmem_st16(uint32_t taddr, const float (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15]))
+        : "memory");
+  }
+
+  // 32 accumulator columns of this thread's lane
+  __device__ __forceinline__ static void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+  }
+
+  // ---- pieces of the tensor-core attention (plain functions: the tiles' registers must not end up behind
+  // a closure's pointers, in local memory, where every load would be waited for at once)
+  // scratch: Q tile [2 halves][AM rows][128 B], K and V tiles [2 halves][64 keys][128 B], P tile [AM rows][128 B],
+  // then two floats per row (what the halves of a row tell each other); AM = 64 or 128 rows per item
+  static constexpr int TK = 64;
+  static constexpr uint32_t Q_OFF = 0;
+  __device__ __forceinline__ static uint32_t k_off(int AM) { return (uint32_t)AM * 256u; }
+  __device__ __forceinline__ static uint32_t v_off(int AM) { return k_off(AM) + TK * 256; }
+  __device__ __forceinline__ static uint32_t p_off(int AM) { return v_off(AM) + TK * 256; }
+  __device__ __forceinline__ static uint32_t x_off(int AM) { return p_off(AM) + (uint32_t)AM * 128u; }
+  static constexpr uint32_t S_COL = 0, O_COL = 128;
+  // worker warp 4, one lane: the 64-key tile at key0 of one kv head, two 64-dim halves of [64 keys][128 bytes]
+  // as the tensor map's 128-byte swizzle lays them out (rows past the context read as zeros)
+  __device__ __forceinline__ void tc_fetch(const CUtensorMap* map, uint32_t dst, uint64_t* bar, int kvh, int key0,
+                                           uint64_t policy, uint32_t el) const {
+    if (ww != 4 || !el) return;
+    const uint32_t b = tc::smem_u32(bar);
+    tc::mbar_expect_tx(b, (uint32_t)(TK * HD * 2));
+    tc::tma_load_2d(dst, map, b, kvh * HD, key0, policy);
+    tc::tma_load_2d(dst + TK * 128, map, b, kvh * HD + 64, key0, policy);
+  }
+  // worker warp 4: the multiplies of one step, then one commit on the attention's barrier
+  // (it first waits for the tiles the multiplies read; a wait that runs out raises the abort flag, which ends tc_wait)
+  __device__ __forceinline__ void tc_issue(uint32_t s_base, int AM, bool pv, bool pv_acc, bool qk) {
+    if (ww != 4) return;
+    if (pv) {
+      if (!wait_bar(&sh->att_v_bar, att_vph & 1u, p.ctl, sh)) return;
+      att_vph ^= 1u;
+    }
+    if (qk) {
+      if (!wait_bar(&sh->att_k_bar, att_kph & 1u, p.ctl, sh)) return;
+      att_kph ^= 1u;
+    }
+    const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TK >> 3) << 17) | ((uint32_t)(AM >> 4) << 24);
+    const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(AM >> 4) << 24);
+    const uint32_t K_OFF = k_off(AM), V_OFF = v_off(AM), P_OFF = p_off(AM);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t el = elect_one();
+    if (pv) {
+      const uint64_t da = make_desc(s_base + P_OFF);
+      // V: 8-key groups 1024 bytes apart (stride offset), 64-dim halves TK * 128 bytes apart (leading offset)
+      const uint64_t db = ((uint64_t)DESC_HI << 32) | (uint64_t)((((s_base + V_OFF) & 0x3FFFFu) >> 4) | ((uint32_t)(TK * 128 / 16) << 16));
+      if (pv_acc) mma_el<true>(tmem_base + O_COL, da, db, idesc_pv, el);
+      else mma_el<false>(tmem_base + O_COL, da, db, idesc_pv, el);
+#pragma unroll
+      for (int s4 = 1; s4 < TK / 16; ++s4)
+        mma_el<true>(tmem_base + O_COL, da + (uint64_t)(2 * s4), db + (uint64_t)(s4 * (16 * 128 / 16)), idesc_pv, el);
+    }
+    if (qk) {
+#pragma unroll
+      for (int s8 = 0; s8 < HD / 16; ++s8) {
+        const uint64_t da = make_desc(s_base + Q_OFF + (s8 >> 2) * (AM * 128)) + (uint64_t)((s8 & 3) * 2);
+        const uint64_t db = make_desc(s_base + K_OFF + (s8 >> 2) * (TK * 128)) + (uint64_t)((s8 & 3) * 2);
+        if (s8 == 0) mma_el<false>(tmem_base + S_COL, da, db, idesc_qk, el);
+        else mma_el<true>(tmem_base + S_COL, da, db, idesc_qk, el);
+      }
+    }
+    mma_commit_el(tc::smem_u32(&sh->att_bar), el);
+  }
+  // one thread polls the barrier, the others sleep in the hardware barrier behind it (one decision for all)
+  __device__ __forceinline__ bool tc_wait() {
+    bool ok = true;
+    if (wtid == 0) ok = wait_bar(&sh->att_bar, att_phase & 1u, p.ctl, sh);
+    att_phase ^= 1u;
+    ok = worker_and(ok);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    return ok;
+  }
+  // Every thread polls the barrier itself: no CTA barrier behind the wait.  A thread whose wait ran out carries
+  // on (it touches shared and tensor memory only) and reports it at the next reducing barrier, where all decide together.
+  __device__ __forceinline__ bool tc_poll() {
+    const bool ok = wait_bar(&sh->att_bar, att_phase & 1u, p.ctl, sh);
+    att_phase ^= 1u;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    return ok;
+  }
+  // generic-proxy writes of the tiles before the tensor core reads them; tensor-memory accesses before the barrier
+  __device__ __forceinline__ static void tc_fences() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  }
+  __device__ __forceinline__ static float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+  }
+  // weights of 32 columns of a row under the maximum m: bf16 into the row of the P tile (pieces 4 half ..) if `wr`,
+  // their sum back; columns from nv on are not keys of the run and weigh nothing
+  template <bool MASKED>
+  __device__ __forceinline__ static float tc_weights(const float (&s)[32], int nv, float m, uint8_t* p_row, int swz, int half,
+                                                     bool wr) {
+    float r4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float w[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        w[k] = ex2(s[j * 8 + k] - m);
+        if (MASKED && j * 8 + k >= nv) w[k] = 0.f;
+        r4[k & 3] += w[k];
+      }
+      const uint2 p01 = pack4(w[0], w[1], w[2], w[3]), p23 = pack4(w[4], w[5], w[6], w[7]);
+      if (wr) *reinterpret_cast<uint4*>(p_row + (((half * 4 + j) ^ swz) << 4)) = make_uint4(p01.x, p01.y, p23.x, p23.y);
+    }
+    return (r4[0] + r4[1]) + (r4[2] + r4[3]);
+  }
+
+  // ---- attention of a search job over its cache keys on the tensor cores (head dimension 128).
+  // Item = (kv head, run of cache keys, block of TC_ROWS (row, query head) pairs).  Per 64-key tile:
+  //   S = Q K^T   (M = 128 pairs, N = 64 keys, K = 128 dims; Q and K tiles K-major, 128-byte swizzle)
+  //   P = exp2(S - m) as bf16 into shared memory, row sums in registers
+  //   O += P V    (N = 128 dims, K = 64 keys; the V tile stays as the cache has it, key rows of 128 dims,
+  //                i.e. the MN-major form of the B operand)
+  // S and O live in tensor memory, which no product uses while the attention runs (the o projection
+  // waits for the merged rows of every CTA).  A row of S sits in one lane: worker warps w and w + 4 share
+  // lane quarter w & 3 and take 32 of the row's 64 columns each.  The row's maximum m is fixed by the
+  // first tile and only moves when a later tile exceeds it by more than 2^8 (the whole CTA then takes a
+  // slow path that rescales O and the sums), so a tile is normally one trip over S.  K and V tiles come
+  // by TMA through the layer's tensor maps, each as soon as the multiplies that read its predecessor are done.  The partial result of an item has the format of
+  // attention_partials, which still computes the chunks of the rows' own keys.
+  __device__ bool attention_tc(const Job& J, int jb) {
+    if constexpr (HD != 128 || !TC) {
+      return false;
+    } else {
+      const Cfg& c = p.c;
+      static_assert(256 * TC_ROWS + 2 * TK * 256 + 128 * TC_ROWS + 2 * TC_ROWS * 4 <= SCRATCH_TC_BYTES, "attention tiles must fit the scratch area");
+      const int AM = c.att_rows;   // 64: an M = 64 accumulator keeps row r in lane 32 (r / 16) + r % 16; 128: row r in lane r
+      const uint32_t K_OFF = k_off(AM), V_OFF = v_off(AM), P_OFF = p_off(AM);
+      const uint32_t s_base = tc::smem_u32(scratch);
+      float* xch = reinterpret_cast<float*>(scratch + x_off(AM));
+      const int Gq = c.nq / c.nkv;
+      const int Pn = J.R * Gq;
+      const int n_pb = (Pn + AM - 1) / AM;
+      const int n_runs = (J.C + c.run_len - 1) / c.run_len;
+      const int n_items = c.nkv * n_runs * n_pb;
+      const int qkvd = c.qd + 2 * c.kvd;
+      const float qscale = rsqrtf((float)HD) * 1.4426950408889634f;
+      const RowDiv rdT(J.T), rdG(Gq);
+      const uint32_t tag = p.launch_tag | (uint32_t)(jb + 1);
+      const int quarter = ww & 3, half = ww >> 2;
+      const int qrows = AM >> 2;                       // rows of a lane quarter
+      const bool lane_ok = lane < qrows;
+      const int row = quarter * qrows + (lane_ok ? lane : 0);
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      const CUtensorMap* kmap = p.kvmaps + J.kvmap;
+      const CUtensorMap* vmap = kmap + 1;
+      const uint32_t el = elect_one();
+      uint64_t pol;
+      asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+      if (ww == 4 && el) {
+        // the maps were written by a copy on the stream before this launch, at addresses earlier launches also used:
+        // the copies of them this SM may still hold are dropped
+        asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(kmap) : "memory");
+        asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(vmap) : "memory");
+      }
+      int it = blockIdx.x;
+      if (it < n_items) {   // the cache does not depend on this layer's projections
+        const int run = (it / n_pb) % n_runs, kvh = it / (n_pb * n_runs);
+        tc_fetch(kmap, s_base + K_OFF, &sh->att_k_bar, kvh, run * c.run_len, pol, el);
+        tc_fetch(vmap, s_base + V_OFF, &sh->att_v_bar, kvh, run * c.run_len, pol, el);
+      }
+      if (!wait_all(F_QKV, J.tgt[F_QKV])) return false;
+      mark(T_ATT_READY);
+      for (; it < n_items; it += c.G) {
+        const int pb = it % n_pb;
+        const int run = (it / n_pb) % n_runs;
+        const int kvh = it / (n_pb * n_runs);
+        const int key_lo = run * c.run_len, key_hi = min(J.C, key_lo + c.run_len);
+        const int nt = (key_hi - key_lo + TK - 1) / TK;
+        if (it != (int)blockIdx.x) {   // (the last item's multiplies are done: both tiles are free)
+          tc_fetch(kmap, s_base + K_OFF, &sh->att_k_bar, kvh, key_lo, pol, el);
+          tc_fetch(vmap, s_base + V_OFF, &sh->att_v_bar, kvh, key_lo, pol, el);
+        }
+        // Q tile: rows rotated and scaled; dims i and i + 64 of a row share a rotation, so one thread
+        // makes the pieces (row, j) and (row, j + 8) from the same loads
+#pragma unroll 2
+        for (int e = 0; e < AM * 8 / WORKERS; ++e) {   // (two tasks' loads in flight)
+          const int task = wtid + e * WORKERS;
+          const int qrow = task >> 3, j = task & 7;
+          const int pp = pb * AM + qrow;
+          uint4 lo_p = make_uint4(0, 0, 0, 0), hi_p = make_uint4(0, 0, 0, 0);
+          if (pp < Pn) {
+            const int rr = rdG.div(pp);
+            const int hq = kvh * Gq + (pp - rr * Gq);
+            const float* qr = p.b.qkv + (long long)rr * qkvd + hq * HD + j * 8;
+            const float4 a0 = __ldcg(reinterpret_cast<const float4*>(qr)), a1 = __ldcg(reinterpret_cast<const float4*>(qr + 4));
+            const float4 b0 = __ldcg(reinterpret_cast<const float4*>(qr + HD / 2)), b1 = __ldcg(reinterpret_cast<const float4*>(qr + HD / 2 + 4));
+            const float4* cs4 = reinterpret_cast<const float4*>(p.b.rope + (long long)rdT.mod(rr) * (HD / 2) + j * 8);
+            const float lo[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            const float hi[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+            float v0[8], v1[8];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float4 cs = cs4[q];   // (cos, sin) of dims 2q and 2q + 1
+              v0[2 * q] = (lo[2 * q] * cs.x - hi[2 * q] * cs.y) * qscale;
+              v1[2 * q] = (hi[2 * q] * cs.x + lo[2 * q] * cs.y) * qscale;
+              v0[2 * q + 1] = (lo[2 * q + 1] * cs.z - hi[2 * q + 1] * cs.w) * qscale;
+              v1[2 * q + 1] = (hi[2 * q + 1] * cs.z + lo[2 * q + 1] * cs.w) * qscale;
+            }
+            const uint2 l01 = pack4(v0[0], v0[1], v0[2], v0[3]), l23 = pack4(v0[4], v0[5], v0[6], v0[7]);
+            const uint2 h01 = pack4(v1[0], v1[1], v1[2], v1[3]), h23 = pack4(v1[4], v1[5], v1[6], v1[7]);
+            lo_p = make_uint4(l01.x, l01.y, l23.x, l23.y);
+            hi_p = make_uint4(h01.x, h01.y, h23.x, h23.y);
+          }
+          uint8_t* dst = scratch + Q_OFF + qrow * 128 + ((j ^ (qrow & 7)) << 4);
+          *reinterpret_cast<uint4*>(dst) = lo_p;
+          *reinterpret_cast<uint4*>(dst + AM * 128) = hi_p;
+        }
+        mark(T_ATT_Q);
+        tc_fences();
+        worker_sync();
+        tc_issue(s_base, AM, false, false, true);
+        if (!tc_wait()) return false;
+        if (nt > 1) tc_fetch(kmap, s_base + K_OFF, &sh->att_k_bar, kvh, key_lo + TK, pol, el);   // S of tile 0 exists: K is free
+
+        const bool rows_here = pb * AM + quarter * qrows < Pn;
+        float m_used = -INFINITY, l_part = 0.f;
+        bool failed = false;   // this thread's last wait for the multiplies ran out
+        for (int t = 0; t < nt; ++t) {
+          const int nv = key_hi - (key_lo + t * TK) - half * 32;   // columns of this half that are keys of the run
+          float s[32];
+          float mx = -INFINITY;
+          if (rows_here) {
+            tmem_ld32(t_row + S_COL + half * 32, s);
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int k = 0; k < 32; ++k)
+              if (k < nv) m4[k & 3] = fmaxf(m4[k & 3], s[k]);
+            mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+          }
+          if (t == 0) {   // the row's maximum over both halves of the first tile
+            if (lane_ok) xch[half * TC_ROWS + row] = mx;
+            worker_sync();
+            m_used = fmaxf(mx, xch[(half ^ 1) * TC_ROWS + row]);
+          }
+          float rs = 0.f;
+          if (rows_here) {
+            if (nv >= 32) rs = tc_weights<false>(s, nv, m_used, scratch + P_OFF + row * 128, row & 7, half, lane_ok);
+            else rs = tc_weights<true>(s, nv, m_used, scratch + P_OFF + row * 128, row & 7, half, lane_ok);
+          }
+          tc_fences();
+          if (worker_or(failed || (rows_here && lane_ok && t > 0 && mx > m_used + 8.f))) {
+            if (!worker_and(!failed)) return false;
+            // some row of this CTA outgrew its maximum: every row looks at both halves again
+            if (lane_ok) xch[half * TC_ROWS + row] = mx;
+            worker_sync();
+            const float m_new = fmaxf(m_used, fmaxf(mx, xch[(half ^ 1) * TC_ROWS + row]));
+            const bool moved = m_new > m_used + 8.f;   // the same answer in both halves of the row
+            if (rows_here && __any_sync(0xffffffffu, moved)) {
+              const float corr = moved ? exp2f(m_used - m_new) : 1.f;
+              if (moved) { l_part *= corr; m_used = m_new; }
+#pragma unroll
+              for (int q = 0; q < HD / 32; ++q) {   // this half's 64 columns of O
+                float o[16];
+                tc::tmem_ld16(t_row + O_COL + half * (HD / 2) + q * 16, o);
+#pragma unroll
+                for (int k = 0; k < 16; ++k) o[k] *= corr;
+                tmem_st16(t_row + O_COL + half * (HD / 2) + q * 16, o);
+              }
+              asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+              rs = tc_weights<true>(s, nv, m_used, scratch + P_OFF + row * 128, row & 7, half, lane_ok);
+            }
+            tc_fences();
+            worker_sync();
+          }
+          l_part += rs;
+          tc_issue(s_base, AM, true, t > 0, t + 1 < nt);
+          failed = !tc_poll();
+          // the multiplies just waited for were the last readers of V (t) and K (t + 1)
+          if (t + 1 < nt) tc_fetch(vmap, s_base + V_OFF, &sh->att_v_bar, kvh, key_lo + (t + 1) * TK, pol, el);
+          if (t + 2 < nt) tc_fetch(kmap, s_base + K_OFF, &sh->att_k_bar, kvh, key_lo + (t + 2) * TK, pol, el);
+        }
+        mark(T_ATT_TILES);
+        if (lane_ok) xch[half * TC_ROWS + row] = l_part;
+        if (!worker_and(!failed)) return false;
+        if (rows_here) {
+          const float l_sum = l_part + xch[(half ^ 1) * TC_ROWS + row];
+          const int pp = pb * AM + row;
+          const int rr = rdG.div(min(pp, Pn - 1));
+          const int hq = kvh * Gq + (min(pp, Pn - 1) - rr * Gq);
+          const long long idx = ((long long)rr * c.nq + hq) * c.chunk_cap + run;
+          uint4* pa = reinterpret_cast<uint4*>(p.b.att_acc + idx * (HD / 2)) + half * (HD / 8);
+#pragma unroll
+          for (int q = 0; q < HD / 32; ++q) {
+            float o[16];
+            tc::tmem_ld16(t_row + O_COL + half * (HD / 2) + q * 16, o);
+            if (pp < Pn && lane_ok) {
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                __stcg(pa + q * 4 + k, make_uint4(pack2(o[4 * k], o[4 * k + 1]), tag, pack2(o[4 * k + 2], o[4 * k + 3]), tag));
+            }
+          }
+          if (pp < Pn && lane_ok && half == 0) __stcg(p.b.att_ml + idx, make_uint4(__float_as_uint(m_used), tag, __float_as_uint(l_sum), tag));
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      worker_sync();
+      return true;
+    }
+  }
+
   // All chunks of a (row, query head) pair merged by one warp; the pairs are dealt out to all CTAs and,
   // inside a CTA, to its warps.  There is no flag to wait for: the warp reads the partial results until
   // every piece carries this job's tag (see attention_partials), one trip to L2 when they are there.
@@ -1743,7 +2103,12 @@ struct Worker {
         mark(ph == G_QKV ? T_QKV : (ph == G_O ? T_O : (ph == G_GU ? T_GU : T_DOWN)));
         if (ph == G_QKV) {
           publish(F_QKV, jb + 1);
-          if (!attention_partials(J, jb)) return false;
+          if (TC && c.att_tc && !J.uniform) {
+            if (!attention_tc(J, jb)) return false;
+            if (!attention_partials<true>(J, jb)) return false;
+          } else if (!attention_partials(J, jb)) {
+            return false;
+          }
           mark(T_ATT_PUB);
           if (!attention_merge(J, jb)) return false;
           mark(T_MERGE);
@@ -1771,7 +2136,7 @@ constexpr int REGS_WORKER = (THREADS * 168 - 128 * REGS_SPECIAL) / 256 / 8 * 8;
 static_assert(THREADS == 384 && WORKER_T0 == 128, "register split assumes one special and two worker warp groups");
 static_assert(128 * REGS_SPECIAL + 256 * REGS_WORKER <= THREADS * 168, "register pool of the CTA");
 
-template <bool TR, int HD>
+template <bool TR, int HD, bool TC>
 __global__ void __launch_bounds__(THREADS, 1)
 engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constant__ CUtensorMap map_attn,
               const __grid_constant__ CUtensorMap map_xn_m, const __grid_constant__ CUtensorMap map_act,
@@ -1796,6 +2161,9 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
       tc::mbar_init(tc::smem_u32(&sh.acc_full[b]), 1);
       tc::mbar_init(tc::smem_u32(&sh.acc_empty[b]), 1);
     }
+    tc::mbar_init(tc::smem_u32(&sh.att_bar), 1);
+    tc::mbar_init(tc::smem_u32(&sh.att_k_bar), 1);
+    tc::mbar_init(tc::smem_u32(&sh.att_v_bar), 1);
     sh.abort = 0;
     sh.wait_fast = p.wait_fast;
     sh.wait_slow = p.wait_slow;
@@ -1831,7 +2199,7 @@ engine_kernel(const __grid_constant__ CUtensorMap map_xn_a, const __grid_constan
     }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_WORKER));
-    Worker<TR, HD> w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0};
+    Worker<TR, HD, TC> w{p, &sh, scratch, tmem_base, (int)threadIdx.x - WORKER_T0, warp - 4, lane, 0u, 0};
     w.run();
   }
 

@@ -139,7 +139,7 @@ def cmd_trace(args):
     microseconds after the job's first stamp."""
     import numpy as np
     C, M, T = args.ctx[0], args.M[0], args.T[0]
-    cfg, ccfg, eng, keep = build_engine(args.model, C + 64, M, T)
+    cfg, ccfg, eng, keep = build_engine(args.model, C + 64, M, T, flags=args.flags)
     kv = clasp.KVCache(ccfg, device=eng.device)
     toks = datagen.token_ids(cfg, C).to(eng.device)
     hid = prefill_to(eng, kv, toks, 0, C, T)[-T:].contiguous()
@@ -239,6 +239,7 @@ def main():
     p.add_argument("--M", type=int, nargs="+", default=[12])
     p.add_argument("--T", type=int, nargs="+", default=[1])
     p.add_argument("--job", type=int, default=20)
+    p.add_argument("--flags", type=int, default=0, help="library flags (16: no tensor-core attention)")
     p = sub.add_parser("decode")
     p.add_argument("--model", default="8b")
     p.add_argument("--prompt", type=int, default=512)

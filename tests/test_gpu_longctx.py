@@ -1,11 +1,15 @@
 """Parity at a long context: the LLaMA3-8B layer shape (d = 4096, 32 / 8 heads of 128, FFN 14336, bf16)
-over an 8192-position cache (every run of cache keys spans several 32-key tiles, 32 runs per kv head), on a
-two-layer model so that the oracle can hold a layer in float64: sampled rows of one decoder layer, and one
-search with T = 4 objective rows per state (M = 2) compared cell by cell.
+over an 8192-position cache (every run of cache keys spans several tiles), on a two-layer model so that
+the oracle can hold a layer in float64: sampled rows of one decoder layer, one search with T = 4
+objective rows per state (M = 2) compared cell by cell, and searches built so that the chosen state is
+a layer output the search itself computed (M = 1): its rows are compared with the oracle's, for row
+counts that take the 64-row and the 128-row shape of the tensor-core attention, two blocks of
+(row, head) pairs, and keys that grow along the context so that the running maximum moves late.
 
 Inputs are seeded and synthetic, the same bytes on both sides (weights created on the device and copied
 to the host for the oracle; cache contents and states from seeded normal streams).  Tolerances: hidden
 states relative L2 <= 2e-2 (bf16 model), scores 1e-3."""
+import contextlib
 import dataclasses
 
 import numpy as np
@@ -27,7 +31,7 @@ class LongContext8B:
         import paper_2505_24196_b200 as clasp
         self.cfg = cfg = dataclasses.replace(datagen.CONFIGS["8b"], name="8b-l2", L=2, vocab=8192)
         dev = torch.device("cuda", 0)
-        self.ccfg = clasp.make_config(cfg, max_ctx=C0 + 64, max_rows=128, max_M=2, max_T=4, max_head_rows=8)
+        self.ccfg = clasp.make_config(cfg, max_ctx=C0 + 64, max_rows=128, max_M=2, max_T=40, max_head_rows=8)
         self.engine = clasp.Clasp(self.ccfg, device=dev)
         self.layers = [datagen.layer_weights(cfg, l, dev) for l in range(cfg.L)]
         self.head = datagen.head_weights(cfg, dev)
@@ -88,3 +92,62 @@ def test_search_over_a_long_context(mlong):
         np.testing.assert_array_equal(res["S"].cpu().numpy(), ref["S"])
         assert rel_l2(res["g_final"].cpu().numpy(), ref["g"][L, M]) < 2e-2
     assert int(res["S"].sum()) == M
+
+
+def _search_that_applies_layer_1(mlong, T, seed):
+    """Hidden states x[0..2] such that the best state with one skipped layer is f_1(x_0): the search
+    must compute it (rows attend to the cache and to the rows before them) and return it as g[L][M]."""
+    cfg, eng = mlong.cfg, mlong.engine
+    L, d, M = cfg.L, cfg.d_model, 1
+    p0 = C0 - T
+    x0 = datagen.normal_rows(seed, 0, (T, d)).to(torch.float32)
+    w = mlong.oracle.layer(1)
+    f1, _, _ = orc.decoder_layer(x0.double().numpy(), w, mlong.ocache.k[1], mlong.ocache.v[1], p0, p0, cfg)
+    x1 = x0 + datagen.normal_rows(seed, 1, (T, d)).to(torch.float32)          # far from everything
+    x2 = torch.from_numpy(f1).to(torch.float32)
+    x = torch.stack([x0, x1, x2])
+    ref = orc.dp_search(mlong.oracle, x.double().numpy(), mlong.ocache, p0, p0, M)
+    assert list(ref["S"]) == [1, 0]                # layer 0 skipped, layer 1 applied by the search
+    res = eng.dp_search(x.cuda(), T * d, d, mlong.kv, p0, p0, T, M)
+    torch.cuda.synchronize()
+    assert eng.device_status() == 0
+    np.testing.assert_array_equal(res["S"].cpu().numpy(), ref["S"])
+    got = res["g_final"].cpu().numpy().reshape(T, d)
+    for r in range(T):                             # row by row: a wrong row must not hide among good ones
+        assert rel_l2(got[r:r + 1], f1[r:r + 1]) < 2e-2, r
+    D = res["D"].cpu().numpy()
+    np.testing.assert_allclose(D[~np.isnan(D)], ref["D"][~np.isnan(D)], atol=1e-3)
+
+
+@contextlib.contextmanager
+def scaled_keys(mlong, first, factor):
+    """Layer 1's cached keys from position `first` on times a power of two (exact in bf16 and float64), on
+    both sides.  With unit-variance keys a row's weights spread evenly over 8192 positions and the attention
+    output nearly vanishes in the layer output; larger keys concentrate them on a few positions, so that a
+    mistake in any tile of keys or values moves some row by far more than the tolerance."""
+    mlong.kv.k[1, first:] *= factor
+    mlong.ocache.k[1][first:] *= float(factor)
+    try:
+        yield
+    finally:
+        mlong.kv.k[1, first:] /= factor
+        mlong.ocache.k[1][first:] /= float(factor)
+
+
+@pytest.mark.parametrize("T", [12, 40])
+def test_search_returns_the_layer_output_it_computed(mlong, T):
+    """T = 12: 48 (row, head) pairs per kv head, one 64-row item; T = 40: 160 pairs, a full 128-row
+    block and a second one with 32 rows."""
+    with scaled_keys(mlong, 0, 4):
+        _search_that_applies_layer_1(mlong, T, 74 + T)
+
+
+@pytest.mark.parametrize("lo_scale", [1, 2])
+def test_search_with_keys_that_grow_along_the_context(mlong, lo_scale):
+    """Keys from the middle of the cache on 4 times those before: the scores of the later tiles
+    exceed the maximum the first tile fixed by more than 2^8, so the rows' running maxima move
+    and the accumulated output is rescaled.  (Much larger keys would test bf16's rounding of q instead:
+    a score of several hundred carries an absolute error near 1.)"""
+    # (the step sits inside a run of keys, past its first 64-key tile: a run is one item's share of the context)
+    with scaled_keys(mlong, 0, lo_scale), scaled_keys(mlong, C0 // 2 + 100, 4):
+        _search_that_applies_layer_1(mlong, 12, 91)

@@ -1640,8 +1640,7 @@ struct Worker {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
   }
 
-  // ---- pieces of the tensor-core attention (plain functions: the tiles' registers must not end up behind
-  // a closure's pointers, in local memory, where every load would be waited for at once)
+  // ---- pieces of the tensor-core attention
   // scratch: Q tile [2 halves][AM rows][128 B], K and V tiles [2 halves][64 keys][128 B], P tile [AM rows][128 B],
   // then two floats per row (what the halves of a row tell each other); AM = 64 or 128 rows per item
   static constexpr int TK = 64;
@@ -1748,8 +1747,8 @@ struct Worker {
   }
 
   // ---- attention of a search job over its cache keys on the tensor cores (head dimension 128).
-  // Item = (kv head, run of cache keys, block of TC_ROWS (row, query head) pairs).  Per 64-key tile:
-  //   S = Q K^T   (M = 128 pairs, N = 64 keys, K = 128 dims; Q and K tiles K-major, 128-byte swizzle)
+  // Item = (kv head, run of cache keys, block of 64 or 128 (row, query head) pairs).  Per 64-key tile:
+  //   S = Q K^T   (M = the block's pairs, N = 64 keys, K = 128 dims; Q and K tiles K-major, 128-byte swizzle)
   //   P = exp2(S - m) as bf16 into shared memory, row sums in registers
   //   O += P V    (N = 128 dims, K = 64 keys; the V tile stays as the cache has it, key rows of 128 dims,
   //                i.e. the MN-major form of the B operand)

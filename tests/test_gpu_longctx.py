@@ -9,7 +9,6 @@ counts that take the 64-row and the 128-row shape of the tensor-core attention, 
 Inputs are seeded and synthetic, the same bytes on both sides (weights created on the device and copied
 to the host for the oracle; cache contents and states from seeded normal streams).  Tolerances: hidden
 states relative L2 <= 2e-2 (bf16 model), scores 1e-3."""
-import contextlib
 import dataclasses
 
 import numpy as np
@@ -19,7 +18,7 @@ import torch
 import datagen
 from oracle import clasp_oracle as orc
 from oracle import from_torch
-from tests.util import rel_l2
+from tests.util import rel_l2, scaled_keys, search_that_applies_layer_1
 
 pytestmark = pytest.mark.gpu
 
@@ -94,52 +93,12 @@ def test_search_over_a_long_context(mlong):
     assert int(res["S"].sum()) == M
 
 
-def _search_that_applies_layer_1(mlong, T, seed):
-    """Hidden states x[0..2] such that the best state with one skipped layer is f_1(x_0): the search
-    must compute it (rows attend to the cache and to the rows before them) and return it as g[L][M]."""
-    cfg, eng = mlong.cfg, mlong.engine
-    L, d, M = cfg.L, cfg.d_model, 1
-    p0 = C0 - T
-    x0 = datagen.normal_rows(seed, 0, (T, d)).to(torch.float32)
-    w = mlong.oracle.layer(1)
-    f1, _, _ = orc.decoder_layer(x0.double().numpy(), w, mlong.ocache.k[1], mlong.ocache.v[1], p0, p0, cfg)
-    x1 = x0 + datagen.normal_rows(seed, 1, (T, d)).to(torch.float32)          # far from everything
-    x2 = torch.from_numpy(f1).to(torch.float32)
-    x = torch.stack([x0, x1, x2])
-    ref = orc.dp_search(mlong.oracle, x.double().numpy(), mlong.ocache, p0, p0, M)
-    assert list(ref["S"]) == [1, 0]                # layer 0 skipped, layer 1 applied by the search
-    res = eng.dp_search(x.cuda(), T * d, d, mlong.kv, p0, p0, T, M)
-    torch.cuda.synchronize()
-    assert eng.device_status() == 0
-    np.testing.assert_array_equal(res["S"].cpu().numpy(), ref["S"])
-    got = res["g_final"].cpu().numpy().reshape(T, d)
-    for r in range(T):                             # row by row: a wrong row must not hide among good ones
-        assert rel_l2(got[r:r + 1], f1[r:r + 1]) < 2e-2, r
-    D = res["D"].cpu().numpy()
-    np.testing.assert_allclose(D[~np.isnan(D)], ref["D"][~np.isnan(D)], atol=1e-3)
-
-
-@contextlib.contextmanager
-def scaled_keys(mlong, first, factor):
-    """Layer 1's cached keys from position `first` on times a power of two (exact in bf16 and float64), on
-    both sides.  With unit-variance keys a row's weights spread evenly over 8192 positions and the attention
-    output nearly vanishes in the layer output; larger keys concentrate them on a few positions, so that a
-    mistake in any tile of keys or values moves some row by far more than the tolerance."""
-    mlong.kv.k[1, first:] *= factor
-    mlong.ocache.k[1][first:] *= float(factor)
-    try:
-        yield
-    finally:
-        mlong.kv.k[1, first:] /= factor
-        mlong.ocache.k[1][first:] /= float(factor)
-
-
 @pytest.mark.parametrize("T", [12, 40])
 def test_search_returns_the_layer_output_it_computed(mlong, T):
     """T = 12: 48 (row, head) pairs per kv head, one 64-row item; T = 40: 160 pairs, a full 128-row
     block and a second one with 32 rows."""
     with scaled_keys(mlong, 0, 4):
-        _search_that_applies_layer_1(mlong, T, 74 + T)
+        search_that_applies_layer_1(mlong, C0, T, 74 + T)
 
 
 @pytest.mark.parametrize("lo_scale", [1, 2])
@@ -150,4 +109,4 @@ def test_search_with_keys_that_grow_along_the_context(mlong, lo_scale):
     a score of several hundred carries an absolute error near 1.)"""
     # (the step sits inside a run of keys, past its first 64-key tile: a run is one item's share of the context)
     with scaled_keys(mlong, 0, lo_scale), scaled_keys(mlong, C0 // 2 + 100, 4):
-        _search_that_applies_layer_1(mlong, 12, 91)
+        search_that_applies_layer_1(mlong, C0, 12, 91)

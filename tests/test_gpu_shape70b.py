@@ -1,7 +1,9 @@
 """Parity on the LLaMA3-70B layer shape (d = 8192, 64 / 8 heads of 128, FFN 28672, bf16) with the row
 counts of the 70B searches (40 candidate rows, a 1024-position cache), on a two-layer model so that the
 oracle can hold a layer in float64: sampled rows of one decoder layer, and one search whose single
-layer pass carries 40 rows (M = 2 states of T = 20 objective rows) compared cell by cell.
+layer pass carries 40 rows (M = 2 states of T = 20 objective rows) compared cell by cell; and a search
+over a 4096-position context (160 (row, head) pairs per kv head, eight query heads per kv head: two
+128-row blocks of the tensor-core attention) whose result is a layer output it computed itself.
 
 Inputs are seeded and synthetic, the same bytes on both sides (weights created on the device and copied
 to the host for the oracle; cache contents and states from seeded normal streams).  Tolerances: hidden
@@ -15,11 +17,12 @@ import torch
 import datagen
 from oracle import clasp_oracle as orc
 from oracle import from_torch
-from tests.util import rel_l2
+from tests.util import rel_l2, scaled_keys, search_that_applies_layer_1
 
 pytestmark = pytest.mark.gpu
 
 C0 = 1024
+C_LONG = 4096     # a context long enough for the search's tensor-core attention
 
 
 class Shape70B:
@@ -27,7 +30,7 @@ class Shape70B:
         import paper_2505_24196_b200 as clasp
         self.cfg = cfg = dataclasses.replace(datagen.CONFIGS["70b"], name="70b-l2", L=2, vocab=8192)
         dev = torch.device("cuda", 0)
-        self.ccfg = clasp.make_config(cfg, max_ctx=C0 + 64, max_rows=128, max_M=2, max_T=20, max_head_rows=8)
+        self.ccfg = clasp.make_config(cfg, max_ctx=C_LONG + 64, max_rows=128, max_M=2, max_T=20, max_head_rows=8)
         self.engine = clasp.Clasp(self.ccfg, device=dev)
         self.layers = [datagen.layer_weights(cfg, l, dev) for l in range(cfg.L)]
         self.head = datagen.head_weights(cfg, dev)
@@ -39,7 +42,7 @@ class Shape70B:
         cv = datagen.normal_rows(61, 1, shp).to(cfg.torch_dtype)
         self.kv.k.copy_(ck)
         self.kv.v.copy_(cv)
-        self.ocache = orc.KVCache(cfg, C0 + 64)
+        self.ocache = orc.KVCache(cfg, C_LONG + 64)
         self.ocache.k[:] = ck.double().numpy()
         self.ocache.v[:] = cv.double().numpy()
         # the oracle converts a layer to float64 when it asks for it (only layer 1 is ever applied)
@@ -88,3 +91,11 @@ def test_search_with_forty_rows_on_the_70b_shape(m70):
         np.testing.assert_array_equal(res["S"].cpu().numpy(), ref["S"])
         assert rel_l2(res["g_final"].cpu().numpy(), ref["g"][L, M]) < 2e-2
     assert int(res["S"].sum()) == M
+
+
+def test_search_over_a_long_context_on_the_70b_shape(m70):
+    """M = 1, T = 20, 4076 visible positions: g[L][M] is f_1(x_0), computed by the search over the cache
+    (keys scaled by 4 so that the attention carries weight in the layer output) and its own rows."""
+    with scaled_keys(m70, 0, 4):
+        search_that_applies_layer_1(m70, C_LONG, 20, 64)
+

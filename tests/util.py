@@ -2,6 +2,8 @@
 and for the CUDA library (device tensors).  No arithmetic of the method lives here."""
 from __future__ import annotations
 
+import contextlib
+
 import numpy as np
 import torch
 
@@ -132,3 +134,43 @@ def check_search_against_oracle(D, margin, S, g_final, ref, L: int, M: int, tol:
         if g_final is not None:
             assert close_hidden(g_final, ref["g"][L, M], tol)
     return n_checked
+
+
+def search_that_applies_layer_1(m, C0, T, seed):
+    """Hidden states x[0..2] such that the best state with one skipped layer is f_1(x_0): the search
+    must compute it (rows attend to the cache and to the rows before them) and return it as g[L][M]."""
+    cfg, eng = m.cfg, m.engine
+    L, d, M = cfg.L, cfg.d_model, 1
+    p0 = C0 - T
+    x0 = datagen.normal_rows(seed, 0, (T, d)).to(torch.float32)
+    w = m.oracle.layer(1)
+    f1, _, _ = orc.decoder_layer(x0.double().numpy(), w, m.ocache.k[1], m.ocache.v[1], p0, p0, cfg)
+    x1 = x0 + datagen.normal_rows(seed, 1, (T, d)).to(torch.float32)          # far from everything
+    x2 = torch.from_numpy(f1).to(torch.float32)
+    x = torch.stack([x0, x1, x2])
+    ref = orc.dp_search(m.oracle, x.double().numpy(), m.ocache, p0, p0, M)
+    assert list(ref["S"]) == [1, 0]                # layer 0 skipped, layer 1 applied by the search
+    res = eng.dp_search(x.cuda(), T * d, d, m.kv, p0, p0, T, M)
+    torch.cuda.synchronize()
+    assert eng.device_status() == 0
+    np.testing.assert_array_equal(res["S"].cpu().numpy(), ref["S"])
+    got = res["g_final"].cpu().numpy().reshape(T, d)
+    for r in range(T):                             # row by row: a wrong row must not hide among good ones
+        assert rel_l2(got[r:r + 1], f1[r:r + 1]) < 2e-2, r
+    D = res["D"].cpu().numpy()
+    np.testing.assert_allclose(D[~np.isnan(D)], ref["D"][~np.isnan(D)], atol=1e-3)
+
+
+@contextlib.contextmanager
+def scaled_keys(m, first, factor):
+    """Layer 1's cached keys from position `first` on times a power of two (exact in bf16 and float64), on
+    both sides.  With unit-variance keys a row's weights spread evenly over thousands of positions and the attention
+    output nearly vanishes in the layer output; larger keys concentrate them on a few positions, so that a
+    mistake in any tile of keys or values moves some row by far more than the tolerance."""
+    m.kv.k[1, first:] *= factor
+    m.ocache.k[1][first:] *= float(factor)
+    try:
+        yield
+    finally:
+        m.kv.k[1, first:] /= factor
+        m.ocache.k[1][first:] /= float(factor)

@@ -708,8 +708,11 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   // (measured on the 8B shape: it pays from about 4096 positions on, and from about 2048 when a kv head has 256 or more
   // (row, query head) pairs; below that the smaller ring costs the products more than the attention gains)
   const int att_pairs = Rmax * (c.n_q_heads / c.n_kv_heads);
-  const bool att_tc = c.head_dim == 128 && !(c.flags & CLASP_FLAG_NO_ATT_TC) &&
-                      (search_ctx >= pk::TC_MIN_CTX || (search_ctx >= pk::TC_MIN_CTX / 2 && att_pairs >= 256));
+  bool att_tc = c.head_dim == 128 && !(c.flags & CLASP_FLAG_NO_ATT_TC) &&
+                (search_ctx >= pk::TC_MIN_CTX || (search_ctx >= pk::TC_MIN_CTX / 2 && att_pairs >= 256));
+  // (that instantiation carries search jobs only: layer jobs with an Eq. 2 step and select jobs)
+  for (const pk::Job& J : ctx->e_jobs)
+    att_tc = att_tc && J.type != pk::JOB_HEAD && !(J.type == pk::JOB_LAYER && (J.uniform || !J.dp));
   // (row, query head) pairs of a kv head: up to 64 of them fit an M = 64 accumulator, which leaves the ring 24 KB more
   const int att_rows = att_pairs <= 64 ? 64 : pk::TC_ROWS;
   const int scratch_bytes = !att_tc ? pk::SCRATCH_BYTES : (att_rows == 64 ? pk::SCRATCH_TC64_BYTES : pk::SCRATCH_TC_BYTES);

@@ -752,7 +752,8 @@ __device__ void mma_issuer(const Params& p, Shared* sh, uint32_t ring_base, uint
 // ------------------------------------------------------------------ worker steps
 // TR: the step stamps are compiled in; HD: the model's head dimension (64 or 128).  The kernel is
 // sensitive to its code size, so an instantiation carries neither stamps it does not take nor the
-// attention code of the other head dimension; TC: with the tensor-core attention of long-context searches.
+// attention code of the other head dimension; TC: the instantiation for searches over long contexts (tensor-core
+// attention over the cache keys, Eq. 2 write-back dealt to all threads); it is launched for nothing else.
 template <bool TR, int HD, bool TC>
 struct Worker {
   const Params& p;
@@ -1199,6 +1200,30 @@ struct Worker {
   // for its o product, by a select-only job at its start.
   // from_epilogue: the down product's epilogue left the partials of this CTA in the tables and
   // the thread's layer outputs / skip candidates of its first row block in keep_y / keep_s.
+  // Eq. 2 step, rows past the two worker groups' first blocks: they come from global memory, and their
+  // (row, feature) pairs are dealt to all worker threads -- with many rows (several objective rows per state) a
+  // thread per feature would walk its row blocks one dependent load after the other.  to_operand: the chosen
+  // rows, normed, as the next layer's operand; else as g[i][.] for the next step (row r of the step is
+  // g[i][j][t] with j T + t = r + T).  Only in the instantiation for long contexts and many rows.
+  __device__ __forceinline__ void spread_rows(const Job& J, int f_lo, int nf, int rows, bool to_operand) const {
+    const int d = p.c.d, r_rest = 2 * RB, n_rest = max(rows - r_rest, 0) * nf;
+    float* const g_out = J.g_next + (long long)J.T * d;
+    const int gf_lo = (J.M - 1) * J.T;                              // first row of state M, if the step has it
+    float* const gf_out = (J.g_final && rows > gf_lo) ? J.g_final : nullptr;
+#pragma unroll 4
+    for (int idx = wtid; idx < n_rest; idx += WORKERS) {
+      const int rq = idx / nf;
+      const int r = r_rest + rq, ff = f_lo + (idx - rq * nf);
+      const float y = sh->choice_row[r] ? __ldcg(p.b.Gbuf + (long long)r * d + ff) : __ldcg(skip_row(J, r) + ff);
+      if (to_operand) {
+        p.b.xn_a[(long long)r * d + ff] = __float2bfloat16_rn(y * __ldg(J.norm_next + ff));
+      } else {
+        __stcg(g_out + (long long)r * d + ff, y);
+        if (gf_out && r >= gf_lo) gf_out[(long long)(r - gf_lo) * d + ff] = y;
+      }
+    }
+  }
+
   __device__ bool dp_step(const Job& J, int jb, bool from_epilogue, float (&keep_y)[RB], float (&keep_s)[RB]) {
     const Cfg& c = p.c;
     RedTables* T = tables();
@@ -1280,7 +1305,19 @@ struct Worker {
       y16[k] = 0.f;
       if (fv && r < rows) y16[k] = sh->choice_row[r] ? keep_y[k] : keep_s[k];
     }
-    if (J.norm_next && fv && !J.defer) {
+    if constexpr (TC) {
+      // (the instantiation for long contexts and many rows deals the rows past the first blocks to all threads)
+      if (J.norm_next && !J.defer) {
+        if (fv) {
+#pragma unroll
+          for (int k = 0; k < RB; ++k) {
+            const int r = group * RB + k;
+            if (r < rows) p.b.xn_a[(long long)r * c.d + f] = __float2bfloat16_rn(y16[k] * wn);
+          }
+        }
+        spread_rows(J, f_lo, f_hi - f_lo, rows, true);
+      }
+    } else if (J.norm_next && fv && !J.defer) {
       for (int cb = group; cb < ncb; cb += 2) {
 #pragma unroll
         for (int k = 0; k < RB; ++k) {
@@ -1299,7 +1336,19 @@ struct Worker {
     float* const g_out = J.g_next + (long long)J.T * c.d + f;
     const int gf_lo = (J.M - 1) * J.T;                              // first row of state M, if the step has it
     float* const gf_out = (J.g_final && rows > gf_lo) ? J.g_final + f : nullptr;
-    if (fv) {
+    if constexpr (TC) {
+      if (fv) {
+#pragma unroll
+        for (int k = 0; k < RB; ++k) {
+          const int r = group * RB + k;
+          if (r < rows) {
+            __stcg(g_out + (long long)r * c.d, y16[k]);
+            if (gf_out && r >= gf_lo) gf_out[(long long)(r - gf_lo) * c.d] = y16[k];
+          }
+        }
+      }
+      spread_rows(J, f_lo, f_hi - f_lo, rows, false);
+    } else if (fv) {
       for (int cb = group; cb < ncb; cb += 2) {
 #pragma unroll
         for (int k = 0; k < RB; ++k) {
@@ -2102,11 +2151,11 @@ struct Worker {
         mark(ph == G_QKV ? T_QKV : (ph == G_O ? T_O : (ph == G_GU ? T_GU : T_DOWN)));
         if (ph == G_QKV) {
           publish(F_QKV, jb + 1);
-          if (TC && c.att_tc && !J.uniform) {
+          if constexpr (TC) {   // (only launched for searches over long contexts: no forward-pass jobs)
             if (!attention_tc(J, jb)) return false;
             if (!attention_partials<true>(J, jb)) return false;
-          } else if (!attention_partials(J, jb)) {
-            return false;
+          } else {
+            if (!attention_partials(J, jb)) return false;
           }
           mark(T_ATT_PUB);
           if (!attention_merge(J, jb)) return false;

@@ -94,10 +94,11 @@ typedef struct clasp_config {
                                    GEMM, attention, norm, Eq. 2 select ...) instead of the
                                    persistent kernel that runs a whole call in one launch */
 
-#define CLASP_FLAG_NO_ATT_TC 16 /* diagnostics: searches over long contexts (about 4000 positions or more) keep the
-                                   attention over the cache keys on the warp-level multiply instead of
-                                   tcgen05 (the two sum a row's keys in different orders: results agree
-                                   to rounding, not bit for bit) */
+#define CLASP_FLAG_NO_ATT_TC 16 /* diagnostics: searches over long contexts (about 4000 visible positions or
+                                   more; about 1000 when a kv head serves 256 or more (row, query head)
+                                   pairs) keep the attention over the cache keys on the warp-level multiply
+                                   instead of tcgen05 (the two sum a row's keys in different orders:
+                                   results agree to rounding, not bit for bit) */
 
 /* Device pointers to the nine tensors of one decoder layer (borrowed). */
 typedef struct clasp_layer_weights {

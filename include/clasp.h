@@ -95,8 +95,8 @@ typedef struct clasp_config {
                                    persistent kernel that runs a whole call in one launch */
 
 #define CLASP_FLAG_NO_ATT_TC 16 /* diagnostics: searches over long contexts (about 4000 visible positions or
-                                   more; about 1000 when a kv head serves 256 or more (row, query head)
-                                   pairs) keep the attention over the cache keys on the warp-level multiply
+                                   more; 2500 when a kv head serves at most 64 (row, query head) pairs, 1000
+                                   when it serves 256 or more) keep the attention over the cache keys on the warp-level multiply
                                    instead of tcgen05 (the two sum a row's keys in different orders:
                                    results agree to rounding, not bit for bit) */
 

@@ -705,11 +705,15 @@ int engine_launch(clasp_ctx* ctx, int Rmax, int head_off, int search_ctx = -1) {
   CUDA_TRY(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
   // Searches over a long context run the attention over the cache keys on the tensor cores: that needs a
   // larger scratch area (taken from the weight ring) and runs of whole 64-key tiles.
-  // (measured on the 8B shape: it pays from about 4096 positions on, and from about 1024 when a kv head has 256 or more
+  // (measured on the 8B shape: it pays from about 4096 positions on, from about 2500 when a kv head's pairs fit one
+  // 64-row item -- those launches give up less of the ring --, and from about 1024 when a kv head has 256 or more
   // (row, query head) pairs; below that the smaller ring costs the products more than the attention gains)
   const int att_pairs = Rmax * (c.n_q_heads / c.n_kv_heads);
+  // (the 70B layer shape, whose products lose more to the smaller ring, breaks even at 2048 positions with 256 - 320 pairs)
+  const int wide_min = c.d_model >= 8192 ? 2 * pk::TC_MIN_CTX_WIDE : pk::TC_MIN_CTX_WIDE;
   bool att_tc = c.head_dim == 128 && !(c.flags & CLASP_FLAG_NO_ATT_TC) &&
-                (search_ctx >= pk::TC_MIN_CTX || (search_ctx >= pk::TC_MIN_CTX_WIDE && att_pairs >= 256));
+                (search_ctx >= pk::TC_MIN_CTX || (search_ctx >= wide_min && att_pairs >= 256) ||
+                 (search_ctx >= pk::TC_MIN_CTX_NARROW && att_pairs <= 64));
   // (that instantiation carries search jobs only: layer jobs with an Eq. 2 step and select jobs)
   for (const pk::Job& J : ctx->e_jobs)
     att_tc = att_tc && J.type != pk::JOB_HEAD && !(J.type == pk::JOB_LAYER && (J.uniform || !J.dp));

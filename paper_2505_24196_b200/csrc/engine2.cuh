@@ -57,6 +57,7 @@ constexpr int ATT_KEYS = 32;
 constexpr int SCRATCH_BYTES = 2 * ATT_KEYS * 136 * 2 + 2048;  // two padded K/V tiles + slack (>= 16 KB guard)
 constexpr int TC_MIN_CTX = 4000;              // search contexts from here on take the tensor-core attention
 constexpr int TC_MIN_CTX_WIDE = 1000;         // ... with 256 or more (row, query head) pairs per kv head: from here on
+constexpr int TC_MIN_CTX_NARROW = 2500;       // ... with at most 64 pairs per kv head (one 64-row item): from here on
 constexpr int TC_ROWS = 128;                  // (row, query head) pairs of one tensor-core attention item
 constexpr int SCRATCH_TC64_BYTES = 57 * 1024; // the same with 64 rows per item: q tile 16 KB, P tile 8 KB
 constexpr int SCRATCH_TC_BYTES = 81 * 1024;   // q tile 32 KB, K, V and P tiles 16 KB each (1024-aligned), 1 KB of per-row words
